@@ -1,0 +1,158 @@
+/* atb.h - C ABI of the asymmetric-tile-buffered BFP16 x BF16 GEMM library for NVIDIA B200 (sm_100a).
+ *
+ * The library computes C = A x B (Section 1 of "Can Asymmetric Tile Buffering Be Beneficial?")
+ * with A in BFP16 block floating point (Section 2.4: blocks of 8 values share one 8-bit
+ * exponent, 8-bit mantissas, 9 bytes per block), B in BF16, FP32 accumulation and BF16 output,
+ * tiled with asymmetric tile buffering (Section 3): the output tile keeps T_MC rows live while A
+ * is buffered only T_MA <= T_MC rows at a time.
+ *
+ * General rules
+ *   - Plain C.  Every pointer named *_dev is DEVICE memory owned by the caller (any allocator);
+ *     pointers without that suffix are HOST memory.  The library never allocates or frees device
+ *     memory and keeps no reference to caller memory after a call returns.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Device work is
+ *     asynchronous on that stream; the calls return as soon as it is enqueued.
+ *   - Argument errors are returned synchronously and nothing is launched.  No exception or abort
+ *     crosses this boundary.  atb_last_error_message() gives a per-thread detail string.
+ *   - The device must have compute capability 10.0; there is no fallback of any kind.
+ *
+ * BFP16 storage (the logical format is the paper's; the planar device layout is this library's)
+ *   - mantissa plane: int8  mant[M][K], row-major, two's complement in [-127, 127];
+ *   - exponent plane: uint8 exp[ceil(K/64)][M_pad][8], M_pad = M rounded up to a multiple of 32:
+ *     the 8 block exponents of row m that cover columns 64p .. 64p+63 sit in 8 consecutive bytes
+ *     at ((p * M_pad) + m) * 8.  Entries of padded rows / blocks are zero.
+ *   - value of element (m, k) = mant[m][k] * 2^(E - 133), E = exponent of block (m, k / 8).
+ */
+#ifndef ATB_H_
+#define ATB_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    ATB_OK = 0,
+    ATB_ERR_NULL_POINTER = 1,
+    ATB_ERR_BAD_SHAPE = 2,          /* M, N, K or a leading dimension is not acceptable        */
+    ATB_ERR_BAD_TILING = 3,         /* the (T_MA, T_MC, T_K, T_N) tuple is not supported        */
+    ATB_ERR_MISALIGNED = 4,         /* a pointer or stride breaks the 16-byte rules below       */
+    ATB_ERR_UNSUPPORTED_DEVICE = 5, /* current device is not compute capability 10.0            */
+    ATB_ERR_CUDA = 6,               /* a CUDA runtime / driver call failed (see the message)    */
+    ATB_ERR_BUFFER_TOO_SMALL = 7,   /* an output array given by the caller is too short         */
+    ATB_ERR_DEVICE_TIMEOUT = 8      /* a kernel gave up a bounded wait (reported by atb_device_status) */
+} atb_status_t;
+
+/* Name of a status code; never NULL. */
+const char* atb_status_string(atb_status_t status);
+/* Detail of the calling thread's most recent failing call ("" if none); never NULL. */
+const char* atb_last_error_message(void);
+
+/* Asymmetric tiling 4-tuple of Section 3: A is buffered T_MA x T_K, B T_K x T_N, C T_MC x T_N;
+ * rho = T_MC / T_MA >= 1, rho = 1 is conventional symmetric buffering. */
+typedef struct { int T_MA, T_MC, T_K, T_N; } atb_tiling_t;
+
+/* Sizes in bytes of the two BFP16 planes of an M x K matrix (K a multiple of 8). */
+size_t atb_bfp16_mant_bytes(int64_t M, int64_t K);   /* M * K                                  */
+size_t atb_bfp16_exp_bytes(int64_t M, int64_t K);    /* ceil(K/64) * roundup(M, 32) * 8        */
+
+/* BFP16 quantisation (format: Section 2.4; the paper leaves the algorithm open, so this is the
+ * library's definition).  For every row m and block kb (columns 8kb .. 8kb+7):
+ *   amax = largest |x| of the block, NaNs ignored;
+ *   E    = biased fp32 exponent field of amax, 0 if amax is zero or subnormal, at most 254;
+ *   m_k  = round-to-nearest-even(x_k / 2^(E-133)) saturated to [-127, 127]; NaN -> 0, +-Inf -> +-127.
+ * A_dev:    fp32 A[M][lda], row-major, lda >= K elements, 16-byte aligned, lda % 4 == 0.
+ * mant_dev: atb_bfp16_mant_bytes(M, K) bytes, 16-byte aligned.
+ * exp_dev:  atb_bfp16_exp_bytes(M, K) bytes, 16-byte aligned; padding entries are written as 0.
+ * Requires M >= 0, K >= 0, K % 8 == 0.  M == 0 or K == 0 is a no-op returning ATB_OK. */
+atb_status_t atb_quantize_bfp16(const float* A_dev, int64_t M, int64_t K, int64_t lda,
+                                int8_t* mant_dev, uint8_t* exp_dev, void* stream);
+
+/* C = dequant(A) x B with the asymmetric tile buffering schedule of Section 3 (output-stationary:
+ * per K-step the T_K x T_N tile of B is loaded once and rho = T_MC / T_MA slabs of A are streamed
+ * through it; the T_MC x T_N FP32 accumulator is written out once, after K / T_K steps).
+ * FP32 accumulation, one round-to-nearest-even to BF16 at the end.
+ *   A_mant_dev, A_exp_dev: the planes described above (16-byte aligned);
+ *   B_bf16_dev: bf16 B[K][ldb] row-major, ldb >= N, ldb % 8 == 0, 16-byte aligned;
+ *   C_bf16_dev: bf16 C[M][ldc] row-major, ldc >= N, ldc % 8 == 0, 16-byte aligned (written).
+ * Shapes: M, N >= 1 (any value; edge tiles are handled), N % 8 == 0, K >= 64 and K % 64 == 0.
+ * Tilings: T_MC in {128, 256}; T_N in {64, 128, 256}; T_K in {64, 128};
+ *          T_MA in {32, 64, 128, 256} with T_MA <= T_MC; (T_MC / 128) * T_N <= 512 (the FP32
+ *          accumulator must fit the 512 TMEM columns); the shared-memory rings must fit 227 KB.
+ *          atb_tiling_supported() tells in advance.
+ * For fixed (T_MC, T_K, T_N) the result is bit-identical for every T_MA.
+ * Errors: NULL_POINTER, BAD_SHAPE, BAD_TILING, MISALIGNED, UNSUPPORTED_DEVICE, CUDA. */
+atb_status_t atb_gemm(int64_t M, int64_t N, int64_t K, int T_MA, int T_MC, int T_K, int T_N,
+                      const int8_t* A_mant_dev, const uint8_t* A_exp_dev,
+                      const void* B_bf16_dev, int64_t ldb,
+                      void* C_bf16_dev, int64_t ldc, void* stream);
+
+/* 1 if atb_gemm accepts the tiling (kernel exists, TMEM and shared-memory budgets met), else 0.
+ * Host only; touches no device. */
+int atb_tiling_supported(int T_MA, int T_MC, int T_K, int T_N);
+
+/* Waits for `stream` and reports whether any kernel of this library launched by this process on
+ * the current device gave up a bounded wait since the last call (every wait on an mbarrier in the
+ * kernels has an iteration limit so that a fault cannot hang a shared GPU).  Returns ATB_OK,
+ * ATB_ERR_DEVICE_TIMEOUT (and clears the flag) or ATB_ERR_CUDA.  Debug / test helper: it
+ * synchronises. */
+atb_status_t atb_device_status(void* stream);
+
+/* Parameters of the analytical model of Sections 3-5.  One "unit" is what the paper calls a core
+ * (an AIE core there, an SM here). */
+typedef struct {
+    double peak_flops_per_cycle;  /* Perf_core^peak per unit, FLOP per cycle (Eq. 14-15)          */
+    double clock_hz;              /* cycles per second                                            */
+    int    n_units;               /* N_core of Eq. 12                                             */
+    double bw_bytes_per_s;        /* BW_offchip of Eq. 12                                         */
+    double a_bytes, b_bytes, c_bytes;              /* per-element byte costs in AI (Section 3.1)  */
+    double a_buf_bytes, b_buf_bytes, c_buf_bytes;  /* per-element byte costs in Eq. 1             */
+    double a_scratch_bytes;       /* bytes per A-slab element of one converted copy (0 = none)    */
+    double buf_capacity_bytes;    /* S of Eq. 1 for the A and B terms (+ the C term if acc_capacity_bytes == 0) */
+    double acc_capacity_bytes;    /* > 0: the C term c_buf*T_MC*T_N is budgeted here instead (TMEM) */
+    int    share_rows, share_cols;/* array-level sharing factors of Eq. 2 (4 and 8 in the paper)  */
+    double eta, eps_cycles, ii;   /* Eq. 13: Eff_micro = eta T_K / (eps + eta II T_K)             */
+    double delta_cycles;          /* per-slab switching cost of Eq. 14                            */
+} atb_hw_params_t;
+
+typedef struct {
+    atb_tiling_t t;
+    int    feasible;              /* Eq. 1 / Eq. 3 satisfied                                      */
+    double buf_bytes_used;        /* left-hand side of Eq. 1 (A, B and scratch terms; + C if not split) */
+    double acc_bytes_used;        /* C term                                                       */
+    double ai;                    /* Eq. 2, FLOP per byte                                         */
+    double eff_micro, eff_core;   /* Eq. 13, Eq. 15                                               */
+    double mem_bound_flops;       /* AI * BW                                                      */
+    double compute_bound_flops;   /* Eff_core * peak * N_core                                     */
+    double predicted_flops;       /* Eq. 12: the smaller of the two                               */
+} atb_tiling_score_t;
+
+/* Parameter presets: this library's B200 calibration, and the paper's XDNA2 evaluation
+ * (Section 5 and Table 2; precision_config 1, 2 or 3 selects the byte costs of Section 6.1). */
+void atb_hw_params_b200(atb_hw_params_t* hw);
+void atb_hw_params_xdna2(atb_hw_params_t* hw, int precision_config);
+
+/* Scores one tiling for problem depth K with the formulas of Sections 3 and 5 (Eq. 1, 2, 12-15).
+ * Pure host arithmetic; returns ATB_ERR_NULL_POINTER / ATB_ERR_BAD_TILING (non-positive sizes or
+ * T_MC not a multiple of T_MA). */
+atb_status_t atb_score_tiling(const atb_hw_params_t* hw, int64_t K, atb_tiling_t t,
+                              atb_tiling_score_t* out);
+
+/* Tiling selection (Section 5: the trade-off between arithmetic intensity, which wants small T_K
+ * and large rho, and core efficiency, which wants the opposite): enumerates the tilings atb_gemm
+ * supports, scores each with atb_score_tiling for this (M, N, K) - including the loss from
+ * partially filled waves of output tiles over n_units - and returns them best first.
+ *   hw:       NULL = atb_hw_params_b200().
+ *   best:     receives the top feasible tiling (may be NULL).
+ *   scores:   optional array of *n_scores entries, filled best first; *n_scores receives the
+ *             number written.  Pass scores = NULL, n_scores = NULL to get only `best`.
+ * Returns ATB_ERR_BAD_SHAPE if no supported tiling is feasible. */
+atb_status_t atb_select_tiling(int64_t M, int64_t N, int64_t K, const atb_hw_params_t* hw,
+                               atb_tiling_t* best, atb_tiling_score_t* scores, int* n_scores);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ATB_H_ */

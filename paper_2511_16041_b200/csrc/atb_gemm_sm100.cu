@@ -1,0 +1,620 @@
+// atb_gemm: C = dequant(A_bfp16) x B_bf16 with asymmetric tile buffering (Section 3), sm_100a.
+//
+// One persistent CTA per SM walks output tiles of T_MC x T_N.  Per K-step (output-stationary
+// schedule of Section 3.1) the T_K x T_N tile of B is brought into shared memory ONCE and
+// rho = T_MC / T_MA slabs of A are streamed through it; the FP32 accumulator of the whole
+// T_MC x T_N tile lives in tensor memory and is written out once, after K / T_K steps.
+//
+// Warp roles (448 threads):
+//   warp 0      TMA producer: B tiles and raw BFP16 A slabs (int8 mantissas + uint8 exponents)
+//   warp 1      UMMA issuer (one elected lane) and owner of the TMEM allocation
+//   warps 2-5   epilogue: tcgen05.ld -> round to bf16 -> global stores
+//   warps 6-13  dequantisers: raw slab -> bf16, K-major, 128-byte-swizzled operand in shared
+//               memory (exact: m * 2^(E-133) has at most 7 significant bits)
+// Rings, all guarded by mbarriers with bounded waits:
+//   B tiles          (n_b_stages)    producer -> UMMA          (freed by tcgen05.commit)
+//   raw A slabs      (n_raw_stages)  producer -> dequantisers  (freed by the dequantisers)
+//   bf16 A groups    (n_groups x 128 rows) dequantisers -> UMMA (freed by tcgen05.commit)
+//   accumulators     (acc_bufs x T_MC/128 row groups in TMEM)  UMMA -> epilogue
+// The UMMA shape is always 128 x T_N x 16.  A slab of T_MA < 128 rows is the unit of loading,
+// dequantising and signalling; 128 / T_MA consecutive slabs fill one 128-row operand group.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <cstdint>
+#include <mutex>
+
+#include "atb_internal.h"
+#include "sm100_ptx.cuh"
+
+namespace {
+
+using namespace sm100;
+
+constexpr int kThreads = 448;
+constexpr int kDequantWarps = 8;
+constexpr int kDequantThreads = kDequantWarps * 32;
+constexpr int kFirstEpilogueWarp = 2;
+constexpr int kFirstDequantWarp = 6;
+constexpr int kMaxStages = 16;
+constexpr uint32_t kSmemBudget = 232448;          // 227 KB of dynamic shared memory per CTA
+constexpr uint64_t kWaitTimeoutNs = 2000000000ull;  // every mbarrier wait gives up after 2 s
+
+// Set by a kernel whose bounded wait expired: (role << 8) | barrier kind.
+__device__ unsigned int g_gemm_error_flag = 0;
+
+struct GemmParams {
+    int64_t M, N, K, ldc;
+    __nv_bfloat16* C;
+    int m_tiles, n_tiles, k_steps;
+    int n_b_stages, n_groups, n_raw_stages, acc_bufs, tmem_cols;
+    unsigned int* error_flag;
+};
+
+struct Ring {
+    int stage = 0;
+    uint32_t phase = 0;
+    __device__ __forceinline__ void advance(int n) {
+        if (++stage == n) { stage = 0; phase ^= 1u; }
+    }
+};
+
+struct Ctx {
+    volatile uint32_t* abort_flag;
+    unsigned int* error_flag;
+};
+
+// Bounded mbarrier wait.  Returns false when the CTA is aborting or the wait timed out.
+__device__ __forceinline__ bool wait_bar(const Ctx& cx, uint32_t bar, uint32_t parity, unsigned code) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = global_timer_ns();
+    for (uint32_t spins = 0;; ++spins) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((spins & 63u) == 63u) {
+            if (*cx.abort_flag) return false;
+            if (global_timer_ns() - t0 > kWaitTimeoutNs) {
+                *cx.abort_flag = 1u;
+                atomicCAS(cx.error_flag, 0u, code);
+                return false;
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ void tile_coords(int tile, int m_tiles, int n_tiles, int& mt, int& nt) {
+    // Bands of 16 tile-rows, column-major inside a band: the CTAs of one wave share a few
+    // A row-panels and B column-panels in L2.
+    const int per_band = 16 * n_tiles;
+    const int band = tile / per_band, i = tile - band * per_band;
+    const int rows = min(16, m_tiles - band * 16);
+    mt = band * 16 + i % rows;
+    nt = i / rows;
+}
+
+template <int T_MA, int T_MC, int T_K, int T_N>
+struct Cfg {
+    static constexpr int G = T_MC / 128;                       // 128-row groups per output tile
+    static constexpr int RHO = T_MC / T_MA;                    // slabs per K-step
+    static constexpr int SPG = (T_MA < 128) ? 128 / T_MA : 1;  // slabs per group
+    static constexpr int GPS = (T_MA > 128) ? T_MA / 128 : 1;  // groups per slab
+    static constexpr uint32_t B_BYTES = T_K * T_N * 2;
+    static constexpr uint32_t B_BOX_BYTES = T_K * 128;         // one 64-column box of B
+    static constexpr uint32_t GROUP_BYTES = 128 * T_K * 2;
+    static constexpr uint32_t KHALF_BYTES = 128 * 128;         // 128 rows x 64 bf16
+    static constexpr uint32_t RAW_MANT_BYTES = T_MA * T_K;
+    static constexpr uint32_t RAW_EXP_BYTES = T_MA * T_K / 8;
+    static constexpr uint32_t RAW_BYTES = RAW_MANT_BYTES + RAW_EXP_BYTES;
+    static constexpr int BPR = T_K / 8;                        // blocks per slab row
+    static constexpr int DQ_ITERS = T_MA * BPR / kDequantThreads;
+    static_assert(T_MA * BPR % kDequantThreads == 0 && DQ_ITERS >= 1, "slab too small for the dequantisers");
+};
+
+// ---------------------------------------------------------------------------------------------
+// Dequantise one raw slab (T_MA rows x T_K columns) into its place in a bf16 operand group.
+// Thread t owns block (row r, block kb) = (t / BPR + i * 256 / BPR, t % BPR): the raw reads of a
+// warp are contiguous, and the 16-byte stores of 8 consecutive threads fill one 128-byte row.
+template <class C>
+__device__ __forceinline__ void dequant_slab(const uint8_t* raw_mant, const uint8_t* raw_exp,
+                                             uint32_t dst_base, int row_base, int t,
+                                             int T_MA_rows) {
+    const int kb = t % C::BPR;
+    const int r0 = t / C::BPR;
+    uint2 w[C::DQ_ITERS];
+    uint32_t e[C::DQ_ITERS];
+#pragma unroll
+    for (int i = 0; i < C::DQ_ITERS; ++i) {
+        const int r = r0 + i * (kDequantThreads / C::BPR);
+        w[i] = *reinterpret_cast<const uint2*>(raw_mant + (r * C::BPR + kb) * 8);
+        e[i] = raw_exp[(kb >> 3) * T_MA_rows * 8 + r * 8 + (kb & 7)];
+    }
+#pragma unroll
+    for (int i = 0; i < C::DQ_ITERS; ++i) {
+        const int r = r0 + i * (kDequantThreads / C::BPR);
+        const uint32_t E = e[i];
+        // scale 2^(E-133): a normal fp32 for E >= 7, an fp32 subnormal below.
+        const uint32_t s_bits = (E >= 7u) ? ((E - 6u) << 23) : (1u << (E + 16u));
+        const float s = __uint_as_float(s_bits);
+        const uint32_t u0 = w[i].x ^ 0x80808080u, u1 = w[i].y ^ 0x80808080u;   // m + 128 per byte
+        float f[8];
+        // 0x4B0000uu is the float 2^23 + u; (2^23 + u) * s - (2^23 + 128) * s = m * s exactly.
+        const float x0 = __uint_as_float(__byte_perm(u0, 0x4B000000u, 0x7650));
+        const float x1 = __uint_as_float(__byte_perm(u0, 0x4B000000u, 0x7651));
+        const float x2 = __uint_as_float(__byte_perm(u0, 0x4B000000u, 0x7652));
+        const float x3 = __uint_as_float(__byte_perm(u0, 0x4B000000u, 0x7653));
+        const float x4 = __uint_as_float(__byte_perm(u1, 0x4B000000u, 0x7650));
+        const float x5 = __uint_as_float(__byte_perm(u1, 0x4B000000u, 0x7651));
+        const float x6 = __uint_as_float(__byte_perm(u1, 0x4B000000u, 0x7652));
+        const float x7 = __uint_as_float(__byte_perm(u1, 0x4B000000u, 0x7653));
+        if (E < 238u) {
+            const float c = -8388736.0f * s;
+            f[0] = fmaf(x0, s, c); f[1] = fmaf(x1, s, c); f[2] = fmaf(x2, s, c); f[3] = fmaf(x3, s, c);
+            f[4] = fmaf(x4, s, c); f[5] = fmaf(x5, s, c); f[6] = fmaf(x6, s, c); f[7] = fmaf(x7, s, c);
+        } else {   // (2^23 + 128) * s would overflow: subtract first (exact), then scale (exact)
+            f[0] = (x0 - 8388736.0f) * s; f[1] = (x1 - 8388736.0f) * s;
+            f[2] = (x2 - 8388736.0f) * s; f[3] = (x3 - 8388736.0f) * s;
+            f[4] = (x4 - 8388736.0f) * s; f[5] = (x5 - 8388736.0f) * s;
+            f[6] = (x6 - 8388736.0f) * s; f[7] = (x7 - 8388736.0f) * s;
+        }
+        __nv_bfloat162 p0 = __floats2bfloat162_rn(f[0], f[1]);
+        __nv_bfloat162 p1 = __floats2bfloat162_rn(f[2], f[3]);
+        __nv_bfloat162 p2 = __floats2bfloat162_rn(f[4], f[5]);
+        __nv_bfloat162 p3 = __floats2bfloat162_rn(f[6], f[7]);
+        const int rr = row_base + r;
+        const uint32_t dst = dst_base + (rr >> 7) * C::GROUP_BYTES + (kb >> 3) * C::KHALF_BYTES +
+                             (rr & 127) * 128 + ((((kb & 7) ^ (rr & 7))) << 4);
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst),
+                     "r"(*reinterpret_cast<uint32_t*>(&p0)), "r"(*reinterpret_cast<uint32_t*>(&p1)),
+                     "r"(*reinterpret_cast<uint32_t*>(&p2)), "r"(*reinterpret_cast<uint32_t*>(&p3))
+                     : "memory");
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+template <int T_MA, int T_MC, int T_K, int T_N>
+__global__ void __launch_bounds__(kThreads, 1)
+atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_constant__ CUtensorMap tm_exp,
+                const __grid_constant__ CUtensorMap tm_b, const GemmParams p) {
+    using C = Cfg<T_MA, T_MC, T_K, T_N>;
+    extern __shared__ uint8_t smem_raw[];
+
+    // ---- carve shared memory (1024-byte aligned base: required by the 128-byte swizzle) ----
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* const smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+    const uint32_t b_base = smem_base;
+    const uint32_t deq_base = b_base + p.n_b_stages * C::B_BYTES;
+    const uint32_t raw_off = p.n_b_stages * C::B_BYTES + p.n_groups * C::GROUP_BYTES;
+    const uint32_t raw_base = smem_base + raw_off;
+    const uint32_t bar_off = raw_off + p.n_raw_stages * C::RAW_BYTES;
+    const uint32_t bar_base = smem_base + bar_off;          // 8-byte mbarriers
+    const int n_deq_stages = (T_MA <= 128) ? p.n_groups * C::SPG : p.n_groups / C::GPS;
+    const int n_acc = p.acc_bufs * C::G;
+    // barrier indices
+    const uint32_t b_full = bar_base, b_empty = b_full + 8 * p.n_b_stages;
+    const uint32_t raw_full = b_empty + 8 * p.n_b_stages, raw_empty = raw_full + 8 * p.n_raw_stages;
+    const uint32_t deq_full = raw_empty + 8 * p.n_raw_stages, deq_empty = deq_full + 8 * n_deq_stages;
+    const uint32_t acc_full = deq_empty + 8 * n_deq_stages, acc_empty = acc_full + 8 * n_acc;
+    const uint32_t misc = acc_empty + 8 * n_acc;             // [0]: TMEM base, [1]: abort flag
+    volatile uint32_t* const misc_gen = reinterpret_cast<volatile uint32_t*>(smem_gen + (misc - smem_base));
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    Ctx cx{misc_gen + 1, p.error_flag};
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < p.n_b_stages; ++i) { mbar_init(b_full + 8 * i, 1); mbar_init(b_empty + 8 * i, 1); }
+        for (int i = 0; i < p.n_raw_stages; ++i) { mbar_init(raw_full + 8 * i, 1); mbar_init(raw_empty + 8 * i, kDequantWarps); }
+        for (int i = 0; i < n_deq_stages; ++i) { mbar_init(deq_full + 8 * i, kDequantWarps); mbar_init(deq_empty + 8 * i, 1); }
+        for (int i = 0; i < n_acc; ++i) { mbar_init(acc_full + 8 * i, 1); mbar_init(acc_empty + 8 * i, 4); }
+        misc_gen[1] = 0u;
+        fence_mbar_init();
+        prefetch_tensormap(&tm_mant);
+        prefetch_tensormap(&tm_exp);
+        prefetch_tensormap(&tm_b);
+    }
+    if (warp == 1) {
+        tmem_alloc(misc, static_cast<uint32_t>(p.tmem_cols));
+        tmem_relinquish();
+    }
+    tcgen05_fence_before_sync();
+    __syncthreads();
+    tcgen05_fence_after_sync();
+    const uint32_t tmem_base = misc_gen[0];
+
+    const int total_tiles = p.m_tiles * p.n_tiles;
+
+    if (warp == 0) {
+        // ================================ TMA producer ================================
+        if (elect_one()) {
+            Ring rb, rr;
+            bool ok = true;
+            for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+                int mt, nt;
+                tile_coords(tile, p.m_tiles, p.n_tiles, mt, nt);
+                for (int k = 0; ok && k < p.k_steps; ++k) {
+                    if (!(ok = wait_bar(cx, b_empty + 8 * rb.stage, rb.phase ^ 1u, 0x001))) break;
+                    const uint32_t fb = b_full + 8 * rb.stage;
+                    mbar_arrive_expect_tx(fb, C::B_BYTES);
+#pragma unroll
+                    for (int j = 0; j < T_N / 64; ++j)
+                        tma_load_2d(b_base + rb.stage * C::B_BYTES + j * C::B_BOX_BYTES, &tm_b,
+                                    nt * T_N + j * 64, k * T_K, fb);
+                    rb.advance(p.n_b_stages);
+                    for (int s = 0; s < C::RHO; ++s) {
+                        if (!(ok = wait_bar(cx, raw_empty + 8 * rr.stage, rr.phase ^ 1u, 0x002))) break;
+                        const uint32_t fr = raw_full + 8 * rr.stage;
+                        const uint32_t dst = raw_base + rr.stage * C::RAW_BYTES;
+                        mbar_arrive_expect_tx(fr, C::RAW_BYTES);
+                        tma_load_2d(dst, &tm_mant, k * T_K, mt * T_MC + s * T_MA, fr);
+                        tma_load_2d(dst + C::RAW_MANT_BYTES, &tm_exp, mt * T_MC + s * T_MA, k * (T_K / 64), fr);
+                        rr.advance(p.n_raw_stages);
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ================================ UMMA issuer =================================
+        if (elect_one()) {
+            constexpr uint32_t idesc = umma_idesc_bf16_f32(128, T_N, false, true);
+            Ring rb, rd;
+            int it = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++it) {
+                const int acc_buf = it % p.acc_bufs;
+                const uint32_t acc_phase = static_cast<uint32_t>(it / p.acc_bufs) & 1u;
+                for (int k = 0; ok && k < p.k_steps; ++k) {
+                    if (!(ok = wait_bar(cx, b_full + 8 * rb.stage, rb.phase, 0x101))) break;
+                    const uint32_t bs = b_base + rb.stage * C::B_BYTES;
+                    for (int g = 0; g < C::G; ++g) {
+                        const int acc = acc_buf * C::G + g;
+                        if (k == 0 && !(ok = wait_bar(cx, acc_empty + 8 * acc, acc_phase ^ 1u, 0x102))) break;
+                        int group_slot;
+                        if (T_MA <= 128) {
+                            for (int i = 0; ok && i < C::SPG; ++i)
+                                ok = wait_bar(cx, deq_full + 8 * (rd.stage + i), rd.phase, 0x103);
+                            if (!ok) break;
+                            group_slot = rd.stage / C::SPG;
+                        } else {
+                            if ((g % C::GPS) == 0 && !(ok = wait_bar(cx, deq_full + 8 * rd.stage, rd.phase, 0x103))) break;
+                            group_slot = rd.stage * C::GPS + (g % C::GPS);
+                        }
+                        tcgen05_fence_after_sync();
+                        const uint32_t as = deq_base + group_slot * C::GROUP_BYTES;
+                        const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * T_N);
+#pragma unroll
+                        for (int kk = 0; kk < T_K / 16; ++kk) {
+                            const uint64_t a_desc = umma_smem_desc_sw128(as + (kk >> 2) * C::KHALF_BYTES + (kk & 3) * 32, 16, 1024);
+                            const uint64_t b_desc = umma_smem_desc_sw128(bs + kk * 2048, C::B_BOX_BYTES, 1024);
+                            umma_f16_ss(d_tmem, a_desc, b_desc, idesc, (k > 0 || kk > 0) ? 1u : 0u);
+                        }
+                        if (T_MA <= 128) {
+                            for (int i = 0; i < C::SPG; ++i) umma_commit(deq_empty + 8 * (rd.stage + i));
+                            for (int i = 0; i < C::SPG; ++i) rd.advance(n_deq_stages);
+                        } else if ((g % C::GPS) == C::GPS - 1) {
+                            umma_commit(deq_empty + 8 * rd.stage);
+                            rd.advance(n_deq_stages);
+                        }
+                        if (k == p.k_steps - 1) umma_commit(acc_full + 8 * acc);
+                    }
+                    if (!ok) break;
+                    umma_commit(b_empty + 8 * rb.stage);
+                    rb.advance(p.n_b_stages);
+                }
+            }
+        }
+    } else if (warp < kFirstDequantWarp) {
+        // ================================ epilogue ====================================
+        const int q = warp & 3;                       // TMEM lane quadrant this warp may access
+        int it = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++it) {
+            int mt, nt;
+            tile_coords(tile, p.m_tiles, p.n_tiles, mt, nt);
+            const int acc_buf = it % p.acc_bufs;
+            const uint32_t acc_phase = static_cast<uint32_t>(it / p.acc_bufs) & 1u;
+            for (int g = 0; g < C::G; ++g) {
+                const int acc = acc_buf * C::G + g;
+                if (!(ok = wait_bar(cx, acc_full + 8 * acc, acc_phase, 0x201))) break;
+                tcgen05_fence_after_sync();
+                const int64_t row = static_cast<int64_t>(mt) * T_MC + g * 128 + q * 32 + lane;
+                const int64_t col0 = static_cast<int64_t>(nt) * T_N;
+                const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + static_cast<uint32_t>(acc * T_N);
+#pragma unroll 1
+                for (int c = 0; c < T_N / 32; ++c) {
+                    uint32_t v[32];
+                    tmem_ld_32x32b_x32(t_addr + c * 32, v);
+                    tmem_ld_wait();
+                    if (row < p.M) {
+                        __nv_bfloat16* dst = p.C + row * p.ldc + col0 + c * 32;
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            if (col0 + c * 32 + j * 8 + 8 <= p.N) {
+                                uint32_t o[4];
+#pragma unroll
+                                for (int h = 0; h < 4; ++h) {
+                                    __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(v[j * 8 + 2 * h]),
+                                                                              __uint_as_float(v[j * 8 + 2 * h + 1]));
+                                    o[h] = *reinterpret_cast<uint32_t*>(&b2);
+                                }
+                                *reinterpret_cast<uint4*>(dst + j * 8) = make_uint4(o[0], o[1], o[2], o[3]);
+                            }
+                        }
+                    }
+                }
+                tcgen05_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(acc_empty + 8 * acc);
+            }
+        }
+    } else {
+        // ================================ dequantisers ================================
+        const int t = threadIdx.x - kFirstDequantWarp * 32;
+        Ring rr, rd;
+        bool ok = true;
+        for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+            for (int k = 0; ok && k < p.k_steps; ++k) {
+                for (int s = 0; s < C::RHO; ++s) {
+                    if (!(ok = wait_bar(cx, raw_full + 8 * rr.stage, rr.phase, 0x301))) break;
+                    if (!(ok = wait_bar(cx, deq_empty + 8 * rd.stage, rd.phase ^ 1u, 0x302))) break;
+                    const uint8_t* raw = smem_gen + raw_off + rr.stage * C::RAW_BYTES;
+                    uint32_t dst_base;
+                    int row_base;
+                    if (T_MA <= 128) {
+                        dst_base = deq_base + (rd.stage / C::SPG) * C::GROUP_BYTES;
+                        row_base = (rd.stage % C::SPG) * T_MA;
+                    } else {
+                        dst_base = deq_base + rd.stage * C::GPS * C::GROUP_BYTES;
+                        row_base = 0;
+                    }
+                    dequant_slab<C>(raw, raw + C::RAW_MANT_BYTES, dst_base, row_base, t, T_MA);
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) {
+                        mbar_arrive(deq_full + 8 * rd.stage);
+                        mbar_arrive(raw_empty + 8 * rr.stage);
+                    }
+                    rr.advance(p.n_raw_stages);
+                    rd.advance(n_deq_stages);
+                }
+            }
+        }
+    }
+
+    // ---- teardown: on the abort path give copies and MMAs in flight time to land first ----
+    if (*cx.abort_flag) {
+        for (int i = 0; i < 64; ++i) __nanosleep(20000);
+    }
+    tcgen05_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        tcgen05_fence_after_sync();
+        tmem_dealloc(tmem_base, static_cast<uint32_t>(p.tmem_cols));
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Host side
+// ---------------------------------------------------------------------------------------------
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                   CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                   CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    });
+    return fn;
+}
+
+bool make_map_2d(CUtensorMap* map, CUtensorMapDataType type, uint32_t elem_bytes, const void* base,
+                 uint64_t dim0, uint64_t dim1, uint64_t stride1_bytes, uint32_t box0, uint32_t box1,
+                 CUtensorMapSwizzle swizzle) {
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {dim0, dim1};
+    const cuuint64_t strides[1] = {stride1_bytes};
+    const cuuint32_t box[2] = {box0, box1};
+    const cuuint32_t estr[2] = {1, 1};
+    (void)elem_bytes;
+    return fn(map, type, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int T_MA, int T_MC, int T_K, int T_N>
+atb_status_t launch(const atb::GemmPlan& plan, int64_t M, int64_t N, int64_t K, const int8_t* mant,
+                    const uint8_t* exp, const void* B, int64_t ldb, void* Cout, int64_t ldc,
+                    int num_sms, unsigned int* error_flag, cudaStream_t stream) {
+    CUtensorMap tm_mant, tm_exp, tm_b;
+    const int64_t M_pad = atb::round_up(M, 32);
+    if (!make_map_2d(&tm_mant, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, mant, K, M, K, T_K, T_MA, CU_TENSOR_MAP_SWIZZLE_NONE))
+        return atb::fail(ATB_ERR_CUDA, "cuTensorMapEncodeTiled failed for the mantissa plane");
+    if (!make_map_2d(&tm_exp, CU_TENSOR_MAP_DATA_TYPE_UINT64, 8, exp, M_pad, atb::ceil_div(K, 64), M_pad * 8, T_MA,
+                     T_K / 64, CU_TENSOR_MAP_SWIZZLE_NONE))
+        return atb::fail(ATB_ERR_CUDA, "cuTensorMapEncodeTiled failed for the exponent plane");
+    if (!make_map_2d(&tm_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, B, N, K, ldb * 2, 64, T_K, CU_TENSOR_MAP_SWIZZLE_128B))
+        return atb::fail(ATB_ERR_CUDA, "cuTensorMapEncodeTiled failed for B");
+
+    GemmParams p;
+    p.M = M; p.N = N; p.K = K; p.ldc = ldc;
+    p.C = static_cast<__nv_bfloat16*>(Cout);
+    p.m_tiles = static_cast<int>(atb::ceil_div(M, T_MC));
+    p.n_tiles = static_cast<int>(atb::ceil_div(N, T_N));
+    p.k_steps = static_cast<int>(atb::ceil_div(K, T_K));
+    p.n_b_stages = plan.n_b_stages; p.n_groups = plan.n_groups; p.n_raw_stages = plan.n_raw_stages;
+    p.acc_bufs = plan.acc_bufs; p.tmem_cols = plan.tmem_cols;
+    p.error_flag = error_flag;
+
+    auto kernel = atb_gemm_kernel<T_MA, T_MC, T_K, T_N>;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(plan.smem_bytes));
+    if (e != cudaSuccess) return atb::fail(ATB_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
+    const int64_t tiles = static_cast<int64_t>(p.m_tiles) * p.n_tiles;
+    const int grid = static_cast<int>(tiles < num_sms ? tiles : num_sms);
+    kernel<<<grid, kThreads, plan.smem_bytes, stream>>>(tm_mant, tm_exp, tm_b, p);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return atb::fail(ATB_ERR_CUDA, "gemm launch: %s", cudaGetErrorString(e));
+    return ATB_OK;
+}
+
+struct DeviceInfo {
+    bool known = false;
+    int cc_major = 0, cc_minor = 0, num_sms = 0;
+    unsigned int* error_flag = nullptr;
+};
+DeviceInfo g_devices[64];
+std::mutex g_devices_mutex;
+
+atb_status_t device_info(DeviceInfo** out) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return atb::fail(ATB_ERR_CUDA, "cudaGetDevice: %s", cudaGetErrorString(e));
+    if (dev < 0 || dev >= 64) return atb::fail(ATB_ERR_UNSUPPORTED_DEVICE, "device ordinal %d out of range", dev);
+    std::lock_guard<std::mutex> lock(g_devices_mutex);
+    DeviceInfo& d = g_devices[dev];
+    if (!d.known) {
+        cudaDeviceGetAttribute(&d.cc_major, cudaDevAttrComputeCapabilityMajor, dev);
+        cudaDeviceGetAttribute(&d.cc_minor, cudaDevAttrComputeCapabilityMinor, dev);
+        cudaDeviceGetAttribute(&d.num_sms, cudaDevAttrMultiProcessorCount, dev);
+        if (d.cc_major == 10 && d.cc_minor == 0) {
+            e = cudaGetSymbolAddress(reinterpret_cast<void**>(&d.error_flag), g_gemm_error_flag);
+            if (e != cudaSuccess) return atb::fail(ATB_ERR_CUDA, "cudaGetSymbolAddress: %s", cudaGetErrorString(e));
+        }
+        d.known = true;
+    }
+    *out = &d;
+    return ATB_OK;
+}
+
+}  // namespace
+
+namespace atb {
+
+bool plan_gemm(int T_MA, int T_MC, int T_K, int T_N, GemmPlan* plan) {
+    if (!(T_MC == 128 || T_MC == 256)) return false;
+    if (!(T_N == 64 || T_N == 128 || T_N == 256)) return false;
+    if (!(T_K == 64 || T_K == 128)) return false;
+    if (!(T_MA == 32 || T_MA == 64 || T_MA == 128 || T_MA == 256) || T_MA > T_MC) return false;
+    const int G = T_MC / 128;
+    if (G * T_N > 512) return false;
+    const uint32_t b_bytes = T_K * T_N * 2, group_bytes = 128 * T_K * 2, raw_bytes = T_MA * T_K * 9 / 8;
+    const int gps = T_MA > 128 ? T_MA / 128 : 1;          // groups per slab
+    const int spg = T_MA < 128 ? 128 / T_MA : 1;          // slabs per group
+    int nb = 2, ng = 2 * gps, nr = 2;
+    auto total = [&](int b, int g, int r) {
+        const int n_deq = T_MA <= 128 ? g * spg : g / gps;
+        const uint32_t bars = 8u * (2 * b + 2 * r + 2 * n_deq + 2 * 2 * G) + 16u;
+        return 1024u + b * b_bytes + g * group_bytes + r * raw_bytes + bars;
+    };
+    if (total(nb, ng, nr) > kSmemBudget) return false;
+    // Grow the rings towards a target look-ahead, counted in 128-row x T_K operand groups:
+    // B tiles hide the TMA latency for G groups each, raw slabs for T_MA/128 groups each.
+    const double target_b = 8.0 * 64 / T_K, target_r = 6.0 * 64 / T_K, target_g = 4.0;
+    for (;;) {
+        const double cov_b = nb * G / target_b, cov_r = nr * (T_MA / 128.0) / target_r, cov_g = ng / target_g;
+        int pick = -1;
+        double best = 1.0;                               // stop once every ring meets its target
+        if (cov_b < best && nb < kMaxStages && total(nb + 1, ng, nr) <= kSmemBudget) { best = cov_b; pick = 0; }
+        if (cov_r < best && nr < kMaxStages && total(nb, ng, nr + 1) <= kSmemBudget) { best = cov_r; pick = 1; }
+        if (cov_g < best && ng + gps <= kMaxStages && total(nb, ng + gps, nr) <= kSmemBudget) { best = cov_g; pick = 2; }
+        if (pick < 0) break;
+        if (pick == 0) ++nb; else if (pick == 1) ++nr; else ng += gps;
+    }
+    plan->n_b_stages = nb;
+    plan->n_groups = ng;
+    plan->n_raw_stages = nr;
+    plan->acc_bufs = (2 * G * T_N <= 512) ? 2 : 1;
+    int cols = 32;
+    while (cols < plan->acc_bufs * G * T_N) cols <<= 1;
+    plan->tmem_cols = cols;
+    plan->smem_bytes = total(nb, ng, nr);
+    return true;
+}
+
+}  // namespace atb
+
+extern "C" int atb_tiling_supported(int T_MA, int T_MC, int T_K, int T_N) {
+    atb::GemmPlan plan;
+    return atb::plan_gemm(T_MA, T_MC, T_K, T_N, &plan) ? 1 : 0;
+}
+
+#define ATB_DISPATCH_TN(TMA_, TMC_, TK_)                                                               \
+    switch (T_N) {                                                                                     \
+        case 64:  return launch<TMA_, TMC_, TK_, 64>(plan, M, N, K, A_mant_dev, A_exp_dev, B_bf16_dev, ldb, C_bf16_dev, ldc, dev->num_sms, dev->error_flag, st);  \
+        case 128: return launch<TMA_, TMC_, TK_, 128>(plan, M, N, K, A_mant_dev, A_exp_dev, B_bf16_dev, ldb, C_bf16_dev, ldc, dev->num_sms, dev->error_flag, st); \
+        case 256: if constexpr ((TMC_ / 128) * 256 <= 512)                                             \
+                      return launch<TMA_, TMC_, TK_, 256>(plan, M, N, K, A_mant_dev, A_exp_dev, B_bf16_dev, ldb, C_bf16_dev, ldc, dev->num_sms, dev->error_flag, st); \
+                  break;                                                                               \
+    }                                                                                                  \
+    break;
+
+#define ATB_DISPATCH_TK(TMA_, TMC_)                      \
+    if (T_K == 64) { ATB_DISPATCH_TN(TMA_, TMC_, 64) }   \
+    else { ATB_DISPATCH_TN(TMA_, TMC_, 128) }
+
+extern "C" atb_status_t atb_gemm(int64_t M, int64_t N, int64_t K, int T_MA, int T_MC, int T_K, int T_N,
+                                 const int8_t* A_mant_dev, const uint8_t* A_exp_dev,
+                                 const void* B_bf16_dev, int64_t ldb, void* C_bf16_dev, int64_t ldc,
+                                 void* stream) {
+    atb::clear_error();
+    if (!A_mant_dev || !A_exp_dev || !B_bf16_dev || !C_bf16_dev)
+        return atb::fail(ATB_ERR_NULL_POINTER, "A_mant_dev, A_exp_dev, B_bf16_dev and C_bf16_dev must be non-NULL");
+    if (M < 1 || N < 1 || K < 64 || K % 64 != 0 || N % 8 != 0)
+        return atb::fail(ATB_ERR_BAD_SHAPE, "need M >= 1, N >= 8 with N %% 8 == 0, K >= 64 with K %% 64 == 0 (got %lld, %lld, %lld)",
+                         (long long)M, (long long)N, (long long)K);
+    if (M > (1ll << 30) || N > (1ll << 30) || K > (1ll << 30))
+        return atb::fail(ATB_ERR_BAD_SHAPE, "dimensions above 2^30 are not supported");
+    if (ldb < N || ldc < N || ldb % 8 != 0 || ldc % 8 != 0)
+        return atb::fail(ATB_ERR_BAD_SHAPE, "ldb=%lld and ldc=%lld must be >= N and multiples of 8", (long long)ldb, (long long)ldc);
+    if (!atb::aligned16(A_mant_dev) || !atb::aligned16(A_exp_dev) || !atb::aligned16(B_bf16_dev) || !atb::aligned16(C_bf16_dev))
+        return atb::fail(ATB_ERR_MISALIGNED, "all device pointers must be 16-byte aligned");
+    atb::GemmPlan plan;
+    if (T_MA <= 0 || T_MC <= 0 || T_MC % T_MA != 0 || !atb::plan_gemm(T_MA, T_MC, T_K, T_N, &plan))
+        return atb::fail(ATB_ERR_BAD_TILING, "tiling (T_MA=%d, T_MC=%d, T_K=%d, T_N=%d) is not supported", T_MA, T_MC, T_K, T_N);
+    DeviceInfo* dev = nullptr;
+    atb_status_t st_dev = device_info(&dev);
+    if (st_dev != ATB_OK) return st_dev;
+    if (dev->cc_major != 10 || dev->cc_minor != 0)
+        return atb::fail(ATB_ERR_UNSUPPORTED_DEVICE, "compute capability %d.%d; this library runs on 10.0 only", dev->cc_major, dev->cc_minor);
+    if (static_cast<int64_t>(atb::ceil_div(M, T_MC)) * atb::ceil_div(N, T_N) > (1ll << 30))
+        return atb::fail(ATB_ERR_BAD_SHAPE, "too many output tiles");
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+
+    switch (T_MC) {
+        case 128:
+            switch (T_MA) {
+                case 32:  ATB_DISPATCH_TK(32, 128)
+                case 64:  ATB_DISPATCH_TK(64, 128)
+                case 128: ATB_DISPATCH_TK(128, 128)
+            }
+            break;
+        case 256:
+            switch (T_MA) {
+                case 32:  ATB_DISPATCH_TK(32, 256)
+                case 64:  ATB_DISPATCH_TK(64, 256)
+                case 128: ATB_DISPATCH_TK(128, 256)
+                case 256: ATB_DISPATCH_TK(256, 256)
+            }
+            break;
+    }
+    return atb::fail(ATB_ERR_BAD_TILING, "no kernel for tiling (T_MA=%d, T_MC=%d, T_K=%d, T_N=%d)", T_MA, T_MC, T_K, T_N);
+}
+
+extern "C" atb_status_t atb_device_status(void* stream) {
+    atb::clear_error();
+    cudaError_t e = cudaStreamSynchronize(static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return atb::fail(ATB_ERR_CUDA, "cudaStreamSynchronize: %s", cudaGetErrorString(e));
+    unsigned int flag = 0;
+    e = cudaMemcpyFromSymbol(&flag, g_gemm_error_flag, sizeof flag);
+    if (e != cudaSuccess) return atb::fail(ATB_ERR_CUDA, "cudaMemcpyFromSymbol: %s", cudaGetErrorString(e));
+    if (flag != 0) {
+        const unsigned int zero = 0;
+        cudaMemcpyToSymbol(g_gemm_error_flag, &zero, sizeof zero);
+        return atb::fail(ATB_ERR_DEVICE_TIMEOUT, "a GEMM kernel gave up a bounded wait (code 0x%03x)", flag);
+    }
+    return ATB_OK;
+}

@@ -1,0 +1,31 @@
+// Internal helpers shared by the library's translation units (not part of the ABI).
+#pragma once
+#include <cstdarg>
+#include <cstdint>
+#include <cstdio>
+
+#include "atb.h"
+
+namespace atb {
+
+// Records the detail string of the calling thread's failing call and returns `status`.
+atb_status_t fail(atb_status_t status, const char* fmt, ...);
+void clear_error();
+
+inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
+inline int64_t round_up(int64_t a, int64_t b) { return ceil_div(a, b) * b; }
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Shared-memory plan of the GEMM kernel for one tiling (host side; the kernel receives it).
+struct GemmPlan {
+    int n_b_stages;      // B-tile ring depth
+    int n_groups;        // dequantised-A ring depth, in 128-row groups
+    int n_raw_stages;    // raw (BFP16) A-slab ring depth
+    int acc_bufs;        // accumulator buffers in TMEM (1 or 2)
+    int tmem_cols;       // allocated TMEM columns (power of two)
+    uint32_t smem_bytes; // dynamic shared memory of the launch
+};
+// Fills `plan`; false if the tiling is not supported or does not fit.
+bool plan_gemm(int T_MA, int T_MC, int T_K, int T_N, GemmPlan* plan);
+
+}  // namespace atb

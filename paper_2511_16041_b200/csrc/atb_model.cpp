@@ -1,0 +1,140 @@
+// Host-side analytical model of Sections 3-5 and the tiling selection built on it.
+// Pure host arithmetic in FP64; no CUDA calls.
+#include <algorithm>
+#include <cmath>
+#include <vector>
+
+#include "atb_internal.h"
+
+extern "C" {
+
+void atb_hw_params_b200(atb_hw_params_t* hw) {
+    if (!hw) return;
+    // One unit = one SM.  Dense BF16 tcgen05 peak: 8192 FLOP per cycle per SM.  The clock is the
+    // one a tensor-bound kernel settles at under the 1 kW power cap (about 1.35 GHz, which is
+    // what a measured 1.6 PFLOP/s over 148 SMs x 8192 FLOP/cycle implies), not the 1.965 GHz maximum.
+    hw->peak_flops_per_cycle = 8192.0;
+    hw->clock_hz = 1.35e9;
+    hw->n_units = 148;
+    // The level that feeds the SMs tile by tile is L2; every operand byte of a tile crosses it
+    // once per tile (the AI of Section 3.1 counts exactly these bytes).
+    hw->bw_bytes_per_s = 9.0e12;
+    hw->a_bytes = 1.125; hw->b_bytes = 2.0; hw->c_bytes = 2.0;
+    // Shared memory (Eq. 1, A and B terms): raw BFP16 slabs double-buffered at 9/8 B, one
+    // dequantised BF16 copy per slab (2 B, the "converted copy" term), B double-buffered.
+    hw->a_buf_bytes = 1.125; hw->b_buf_bytes = 2.0; hw->c_buf_bytes = 4.0;
+    hw->a_scratch_bytes = 2.0 * 2.0;          // the bf16 operand ring holds two groups per slab row
+    hw->buf_capacity_bytes = 227.0 * 1024.0;
+    hw->acc_capacity_bytes = 128.0 * 512.0 * 4.0;   // TMEM: 128 lanes x 512 columns x 4 B
+    hw->share_rows = 1; hw->share_cols = 1;
+    // Eq. 13: one UMMA covers K = 16 -> eta = 1/16 instructions per unit of T_K; issue interval
+    // II = 1 per instruction slot; eps = fixed per-slab cost, in the same instruction-slot units.
+    hw->eta = 1.0 / 16.0; hw->eps_cycles = 0.25; hw->ii = 1.0;
+    hw->delta_cycles = 150.0;                 // per-slab mbarrier round trip + commit, cycles
+}
+
+void atb_hw_params_xdna2(atb_hw_params_t* hw, int precision_config) {
+    if (!hw) return;
+    hw->peak_flops_per_cycle = 1024.0;        // 512 MAC per cycle per core (Section 2.4)
+    hw->clock_hz = 1.8e9;
+    hw->n_units = 32;
+    hw->bw_bytes_per_s = 65e9;                // Section 5
+    hw->buf_capacity_bytes = 63.0 * 1024.0;   // Eq. 3
+    hw->acc_capacity_bytes = 0.0;             // C lives in the same L1
+    hw->share_rows = 4; hw->share_cols = 8;   // Eq. 2
+    hw->eta = 1.0 / 8.0; hw->eps_cycles = 20.0; hw->ii = 1.0;
+    hw->delta_cycles = 50.0;                  // Section 5
+    hw->a_scratch_bytes = 0.0;
+    switch (precision_config) {
+        case 1:   // A, C in BF16, B in BFP16 (text: 1.25 B in AI; 9/8 B reproduces the buffer column)
+            hw->a_bytes = 2.0; hw->b_bytes = 1.25; hw->c_bytes = 2.0;
+            hw->a_buf_bytes = 2.0; hw->b_buf_bytes = 1.125; hw->c_buf_bytes = 2.0;
+            hw->a_scratch_bytes = 1.125;      // one BFP16-converted copy of the A slab
+            break;
+        case 3:   // all BFP16, BF16 accumulation
+            hw->a_bytes = hw->b_bytes = hw->c_bytes = 1.25;
+            hw->a_buf_bytes = hw->b_buf_bytes = 1.125; hw->c_buf_bytes = 2.125;
+            break;
+        default:  // 2: all BFP16
+            hw->a_bytes = hw->b_bytes = hw->c_bytes = 1.25;
+            hw->a_buf_bytes = hw->b_buf_bytes = hw->c_buf_bytes = 1.125;
+            break;
+    }
+}
+
+atb_status_t atb_score_tiling(const atb_hw_params_t* hw, int64_t K, atb_tiling_t t, atb_tiling_score_t* out) {
+    atb::clear_error();
+    if (!hw || !out) return atb::fail(ATB_ERR_NULL_POINTER, "hw and out must be non-NULL");
+    if (t.T_MA <= 0 || t.T_MC <= 0 || t.T_K <= 0 || t.T_N <= 0 || t.T_MC % t.T_MA != 0 || K <= 0)
+        return atb::fail(ATB_ERR_BAD_TILING, "need positive sizes and T_MC a multiple of T_MA");
+    const double rho = static_cast<double>(t.T_MC) / t.T_MA;
+    const double TMC = t.T_MC, TK = t.T_K, TN = t.T_N, TMA = t.T_MA;
+    out->t = t;
+    // Eq. 1 (left-hand side), with the optional converted-copy term.
+    const double ab = (2.0 * hw->a_buf_bytes / rho) * TMC * TK + 2.0 * hw->b_buf_bytes * TK * TN +
+                      hw->a_scratch_bytes * TMA * TK;
+    const double cb = hw->c_buf_bytes * TMC * TN;
+    if (hw->acc_capacity_bytes > 0.0) {
+        out->buf_bytes_used = ab;
+        out->acc_bytes_used = cb;
+        out->feasible = (ab <= hw->buf_capacity_bytes && cb <= hw->acc_capacity_bytes) ? 1 : 0;
+    } else {
+        out->buf_bytes_used = ab + cb;
+        out->acc_bytes_used = cb;
+        out->feasible = (ab + cb <= hw->buf_capacity_bytes) ? 1 : 0;
+    }
+    // Eq. 2
+    out->ai = 2.0 / (hw->a_bytes / (hw->share_cols * TN) + hw->b_bytes / (hw->share_rows * TMC) +
+                     hw->c_bytes / static_cast<double>(K));
+    // Eq. 13, Eq. 15
+    out->eff_micro = hw->eta * TK / (hw->eps_cycles + hw->eta * hw->ii * TK);
+    out->eff_core = 1.0 / (1.0 / out->eff_micro +
+                           hw->delta_cycles * rho * hw->peak_flops_per_cycle / (2.0 * TMC * TN * TK));
+    // Eq. 12
+    out->mem_bound_flops = out->ai * hw->bw_bytes_per_s;
+    out->compute_bound_flops = out->eff_core * hw->peak_flops_per_cycle * hw->clock_hz * hw->n_units;
+    out->predicted_flops = std::min(out->mem_bound_flops, out->compute_bound_flops);
+    return ATB_OK;
+}
+
+atb_status_t atb_select_tiling(int64_t M, int64_t N, int64_t K, const atb_hw_params_t* hw_in,
+                               atb_tiling_t* best, atb_tiling_score_t* scores, int* n_scores) {
+    atb::clear_error();
+    if (M < 1 || N < 1 || K < 1) return atb::fail(ATB_ERR_BAD_SHAPE, "M, N, K must be positive");
+    if ((scores == nullptr) != (n_scores == nullptr))
+        return atb::fail(ATB_ERR_NULL_POINTER, "scores and n_scores go together");
+    atb_hw_params_t hw;
+    if (hw_in) hw = *hw_in; else atb_hw_params_b200(&hw);
+
+    static const int kMC[] = {128, 256}, kN[] = {64, 128, 256}, kK[] = {64, 128}, kMA[] = {32, 64, 128, 256};
+    std::vector<atb_tiling_score_t> all;
+    for (int mc : kMC) for (int n : kN) for (int k : kK) for (int ma : kMA) {
+        if (ma > mc || !atb_tiling_supported(ma, mc, k, n)) continue;
+        atb_tiling_score_t s;
+        if (atb_score_tiling(&hw, K, atb_tiling_t{ma, mc, k, n}, &s) != ATB_OK) continue;
+        // Wave quantisation: tiles are spread over n_units; the last wave may be partly empty,
+        // and edge tiles compute padding.  Both scale the compute bound.
+        const double tiles = static_cast<double>(atb::ceil_div(M, mc)) * static_cast<double>(atb::ceil_div(N, n));
+        const double waves = std::ceil(tiles / hw.n_units);
+        const double useful = (static_cast<double>(M) * N) / (waves * hw.n_units * mc * n);
+        s.compute_bound_flops *= useful;
+        s.predicted_flops = std::min(s.mem_bound_flops, s.compute_bound_flops);
+        all.push_back(s);
+    }
+    std::stable_sort(all.begin(), all.end(), [](const atb_tiling_score_t& x, const atb_tiling_score_t& y) {
+        if (x.feasible != y.feasible) return x.feasible > y.feasible;
+        return x.predicted_flops > y.predicted_flops;
+    });
+    if (all.empty() || !all.front().feasible) return atb::fail(ATB_ERR_BAD_SHAPE, "no supported tiling is feasible");
+    if (best) *best = all.front().t;
+    if (scores) {
+        const int cap = *n_scores;
+        if (cap < 0) return atb::fail(ATB_ERR_BUFFER_TOO_SMALL, "negative capacity");
+        const int n = std::min<int>(cap, static_cast<int>(all.size()));
+        for (int i = 0; i < n; ++i) scores[i] = all[i];
+        *n_scores = n;
+    }
+    return ATB_OK;
+}
+
+}  // extern "C"
