@@ -1,0 +1,348 @@
+#!/usr/bin/env python3
+"""Benchmark of the asymmetric-tile-buffered BFP16 x BF16 GEMM hot path on B200.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+One *step* is one pass of the whole hot path over one batch of seeded synthetic input that is
+already resident in HBM: quantise A (fp32 -> BFP16 planes), pick the tiling with the host model,
+run the GEMM.  ``value`` is 2*M*N*K per step time, summed over ranks (weak scaling: every rank
+runs the full workload on its own A; no data-path collective).  ``roofline`` is about the GEMM
+kernel alone: its algorithmic FLOPs over its own CUDA-event time inside the same timed region,
+against the measured dense-BF16 cuBLAS peak.  ``e2e`` repeats the step with host buffers: pinned
+host A and B are copied to the device and C is copied back inside the timed region.
+``cpu_baseline`` times the FP64 oracle on the host cores on a bounded row sample (a reported
+baseline, not a target).  ``--impl reference`` times that oracle alone.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "ATB GEMM TFLOPS (1xB200) at 8192^3 BFP16xBF16"
+DEFAULT_WORKLOAD = "cfg3_8192"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# dram__bytes_read.sum + dram__bytes_write.sum per GEMM launch, from the ncu capture summarised in
+# profiles/ (None until a capture of that workload exists).
+NCU_TRAFFIC_BYTES = {}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            d = json.load(f)
+        return {k: float(d[k]) for k in FALLBACK_PEAKS}, "measured"
+    except Exception:
+        return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler:
+    """Polls SM clock and throttle reasons through NVML (read only) while the timed region runs."""
+
+    REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown",
+               0x40: "hw_thermal_slowdown", 0x80: "hw_power_brake_slowdown"}
+
+    def __init__(self, index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            self._h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self._nv = None
+
+    def _run(self):
+        nv = self._nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM))
+                mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self._h) if hasattr(
+                    nv, "nvmlDeviceGetCurrentClocksEventReasons") else nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h)
+                for bit, name in self.REASONS.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(0.002)
+
+    def start(self):
+        if self._nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+        return {"sm_mhz": statistics.median(self.samples) if self.samples else None,
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def physical_gpu_index(local_rank: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_rank])
+        except Exception:
+            return local_rank
+    return local_rank
+
+
+def cpu_oracle_sample(name: str, target_seconds: float):
+    """Times the FP64 oracle GEMM (as it stands) on a bounded row sample of workload `name`."""
+    import oracle
+    from paper_2511_16041_b200 import inputs
+    c = inputs.CONFIGS[name]
+    N, K = c["N"], c["K"]
+    Bb = inputs.make_B_bits(K, N, c["b_scale"])
+    probe = min(c["M"], 64)
+    A = inputs.make_A(c["A"], probe, K)
+    mant, exp = oracle.quantize_bfp16(A)
+    t0 = time.perf_counter()
+    oracle.gemm(mant, exp, Bb)
+    t_probe = time.perf_counter() - t0
+    # the probe pays the fixed B conversion; size the sample from a second, larger probe
+    rows2 = min(c["M"], 256)
+    A = inputs.make_A(c["A"], rows2, K)
+    mant, exp = oracle.quantize_bfp16(A)
+    t0 = time.perf_counter()
+    oracle.gemm(mant, exp, Bb)
+    t2 = time.perf_counter() - t0
+    per_row = max((t2 - t_probe) / max(rows2 - probe, 1), 1e-6)
+    rows = int(min(c["M"], max(rows2, (target_seconds - t_probe) / per_row)))
+    rows -= rows % 8
+    A = inputs.make_A(c["A"], rows, K)
+    t0 = time.perf_counter()
+    mant, exp = oracle.quantize_bfp16(A)
+    oracle.gemm(mant, exp, Bb)
+    dt = time.perf_counter() - t0
+    return {"value": 2.0 * rows * N * K / dt / 1e12, "unit": "TFLOPS", "cores": oracle.num_threads(),
+            "kind": "oracle", "seconds": round(dt, 3),
+            "sample": f"first {rows} of {c['M']} rows of {name} (all {N} columns, K={K}): oracle quantise + FP64 GEMM and |a||b| sum"}
+
+
+def run_reference(args):
+    """--impl reference: the oracle, as it stands, on the host cores; one bounded sample per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    import oracle
+    from paper_2511_16041_b200 import inputs
+    name = args.workload
+    c = inputs.CONFIGS[name]
+    M, N, K = c["M"], c["N"], c["K"]
+    rows = min(M, 256)
+    A = inputs.make_A(c["A"], rows, K)
+    Bb = inputs.make_B_bits(K, N, c["b_scale"])
+    times = []
+    for i in range(args.warmup + args.steps):
+        t0 = time.perf_counter()
+        mant, exp = oracle.quantize_bfp16(A)
+        oracle.gemm(mant, exp, Bb)
+        dt = time.perf_counter() - t0
+        if i >= args.warmup:
+            times.append(dt)
+    ms = 1e3 * sum(times) / len(times)
+    value = 2.0 * rows * N * K / (ms * 1e-3) / 1e12
+    sample = f"{rows} of {M} rows of {name} per step (all {N} columns, K={K})"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": "TFLOPS", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": name, "M": M, "N": N, "K": K, "sampled_rows_per_step": rows},
+            "cpu_baseline": {"value": value, "unit": "TFLOPS", "cores": oracle.num_threads(), "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": value, "unit": "TFLOPS", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+    return 0
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    import paper_2511_16041_b200 as atb
+    from paper_2511_16041_b200 import inputs
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback of the hot path")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    atb.load_library()
+
+    name = args.workload
+    c = inputs.CONFIGS[name]
+    M, N, K = c["M"], c["N"], c["K"]
+    seed = inputs.BASE_SEED + rank                       # each rank owns different rows of a taller A
+    A_host = torch.from_numpy(inputs.make_A(c["A"], M, K, seed)).pin_memory()
+    B_host = torch.from_numpy(inputs.make_B_bits(K, N, c["b_scale"]).view(np.int16)).pin_memory()
+    C_host = torch.empty((M, N), dtype=torch.int16).pin_memory()
+
+    stream = torch.cuda.Stream(dev)
+    A_dev = A_host.to(dev)
+    B_dev = B_host.to(dev).view(torch.bfloat16)
+    mant = torch.empty((M, K), dtype=torch.int8, device=dev)
+    plane = torch.empty(atb.atb_bfp16_exp_bytes(M, K), dtype=torch.uint8, device=dev)
+    C_dev = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
+    torch.cuda.synchronize()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    tiling_used = []
+
+    def step(ev=None):
+        """Whole hot path on device-resident input: quantise -> select tiling -> GEMM."""
+        atb.atb_quantize_bfp16(A_dev, mant, plane, stream=stream)
+        if args.tiling:
+            t = tuple(args.tiling)
+        else:
+            t, _ = atb.atb_select_tiling(M, N, K, max_scores=1)
+        if ev is not None:
+            ev[0].record(stream)
+        atb.atb_gemm(M, N, K, *t, mant, plane, B_dev, C_dev, stream=stream)
+        if ev is not None:
+            ev[1].record(stream)
+        if not tiling_used:
+            tiling_used.append(tuple(t))
+
+    def step_e2e():
+        """Same, from pinned host buffers and back to the host."""
+        with torch.cuda.stream(stream):
+            A_dev.copy_(A_host, non_blocking=True)
+            B_dev.view(torch.int16).copy_(B_host, non_blocking=True)
+        step()
+        with torch.cuda.stream(stream):
+            C_host.copy_(C_dev.view(torch.int16), non_blocking=True)
+        stream.synchronize()
+
+    # ---------------- device-resident timing ----------------
+    for _ in range(max(args.warmup, 3)):
+        step()
+    atb.atb_device_status(stream)
+    sampler = ClockSampler(physical_gpu_index(local_rank))
+    gemm_events = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+                   for _ in range(args.steps)]
+    t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    sampler.start()
+    t_begin.record(stream)
+    for i in range(args.steps):
+        step(gemm_events[i])
+    t_end.record(stream)
+    stream.synchronize()
+    barrier()
+    clocks = sampler.stop()
+    atb.atb_device_status(stream)
+    total_ms = t_begin.elapsed_time(t_end)
+    gemm_ms = sum(a.elapsed_time(b) for a, b in gemm_events) / args.steps
+
+    # ---------------- end-to-end timing (host buffers) ----------------
+    e2e_steps = max(2, min(args.steps, 5))
+    step_e2e()
+    barrier()
+    t0 = time.perf_counter()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(e2e_steps):
+        step_e2e()
+    e1.record(stream)
+    stream.synchronize()
+    barrier()
+    e2e_ms = max(e0.elapsed_time(e1), 1e3 * (time.perf_counter() - t0)) / e2e_steps
+
+    # ---------------- quantiser alone (HBM roofline) ----------------
+    q0, q1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    q0.record(stream)
+    for _ in range(10):
+        atb.atb_quantize_bfp16(A_dev, mant, plane, stream=stream)
+    q1.record(stream)
+    stream.synchronize()
+    quant_ms = q0.elapsed_time(q1) / 10
+
+    # max over ranks
+    times = torch.tensor([total_ms, gemm_ms, e2e_ms, quant_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    total_ms, gemm_ms, e2e_ms, quant_ms = [float(x) for x in times.cpu()]
+
+    if rank == 0:
+        peaks, peak_src = load_peaks()
+        flops = 2.0 * M * N * K
+        ms_per_step = total_ms / args.steps
+        value = world * flops / (ms_per_step * 1e-3) / 1e12
+        achieved = flops / (gemm_ms * 1e-3) / 1e12
+        T_MA, T_MC, T_K, T_N = tiling_used[0]
+        line = {
+            "metric": METRIC, "value": value, "unit": "TFLOPS", "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": name, "M": M, "N": N, "K": K,
+                       "A": f"BFP16 quantised on device from seeded {c['A']} fp32", "B": "bf16, seeded normal",
+                       "tiling": {"T_MA": T_MA, "T_MC": T_MC, "T_K": T_K, "T_N": T_N,
+                                  "chosen_by": "flag" if args.tiling else "atb_select_tiling"},
+                       "step": "atb_quantize_bfp16 + atb_select_tiling + atb_gemm",
+                       "l2": "inputs larger than L2 (A fp32 %d MB, B %d MB, C %d MB per step)" % (
+                           M * K * 4 >> 20, K * N * 2 >> 20, M * N * 2 >> 20),
+                       "parallelism": "replicas, one full GEMM per GPU" if world > 1 else "single GPU"},
+            "clocks": clocks,
+            "e2e": {"value": world * flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOPS",
+                    "h2d_bytes_per_step": A_host.numel() * 4 + B_host.numel() * 2,
+                    "d2h_bytes_per_step": C_host.numel() * 2, "ms_per_step": e2e_ms},
+            "gpu_launches": 2 * args.steps,
+            "roofline": {"bound": "tensor", "kernel": "atb_gemm_kernel", "achieved": achieved,
+                         "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"],
+                         "peak_source": f"{peak_src} cuBLAS bf16 burst",
+                         "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"],
+                         "kernel_ms": gemm_ms, "traffic": NCU_TRAFFIC_BYTES.get(name)},
+            "quantize": {"bound": "hbm", "achieved": M * K * 5.125 / (quant_ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
+                         "unit": "GB/s", "frac": M * K * 5.125 / (quant_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                         "kernel_ms": quant_ms},
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            line["cpu_baseline"] = cpu_oracle_sample(name, args.cpu_seconds)
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
+    ap.add_argument("--tiling", type=int, nargs=4, metavar=("T_MA", "T_MC", "T_K", "T_N"), default=None)
+    ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

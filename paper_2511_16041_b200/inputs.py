@@ -22,11 +22,15 @@ config shape (M, N, K)             A (fp32, then BFP16)          B (bf16)
 """
 from __future__ import annotations
 
+import os
+from concurrent.futures import ThreadPoolExecutor
+
 import numpy as np
 
 BASE_SEED = 251116041
 TAG_A, TAG_B, TAG_MASK = 1, 2, 3
-_CHUNK = 1 << 22
+_CHUNK = 1 << 20
+_THREADS = min(16, os.cpu_count() or 1)
 _U64 = np.uint64
 
 
@@ -50,12 +54,22 @@ def _bits(seed: int, tag: int, start: int, count: int) -> np.ndarray:
         return _splitmix64(idx * _U64(0xD1342543DE82EF95) + _key(seed, tag))
 
 
-def _fill(shape, fn) -> np.ndarray:
+def _fill(shape, fn, dtype=np.float32) -> np.ndarray:
+    """out[i] = fn(start, count)[i - start], chunk by chunk (chunks are independent: threads)."""
     n = int(np.prod(shape))
-    out = np.empty(n, np.float32)
-    for s in range(0, n, _CHUNK):
+    out = np.empty(n, dtype)
+
+    def work(s):
         c = min(_CHUNK, n - s)
         out[s:s + c] = fn(s, c)
+
+    starts = range(0, n, _CHUNK)
+    if _THREADS > 1 and n > _CHUNK:
+        with ThreadPoolExecutor(_THREADS) as pool:
+            list(pool.map(work, starts))
+    else:
+        for s in starts:
+            work(s)
     return out.reshape(shape)
 
 
@@ -81,13 +95,10 @@ def laplace(seed: int, tag: int, shape) -> np.ndarray:
 
 def bernoulli(seed: int, tag: int, shape, p: float) -> np.ndarray:
     """Boolean mask, each entry True with probability p."""
-    n = int(np.prod(shape))
-    out = np.empty(n, bool)
-    for s in range(0, n, _CHUNK):
-        c = min(_CHUNK, n - s)
+    def fn(s, c):
         z = _bits(seed, tag, s, c)
-        out[s:s + c] = (z >> _U64(11)).astype(np.float64) * 2.0 ** -53 < p
-    return out.reshape(shape)
+        return (z >> _U64(11)).astype(np.float64) * 2.0 ** -53 < p
+    return _fill(shape, fn, bool)
 
 
 def to_bf16_bits(x: np.ndarray) -> np.ndarray:

@@ -1,0 +1,72 @@
+"""The C-ABI library loads without a GPU and exports every function include/atb.h declares."""
+import ctypes
+import os
+import re
+
+import paper_2511_16041_b200 as atb
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "atb.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(atb_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    lib = atb.load_library()
+    names = declared_functions()
+    assert "atb_gemm" in names and "atb_quantize_bfp16" in names and "atb_select_tiling" in names
+    for n in names:
+        assert hasattr(lib, n), n
+    assert sorted(atb.EXPORTED_SYMBOLS) == names
+
+
+def test_binding_has_the_same_names():
+    for n in declared_functions():
+        assert callable(getattr(atb, n)), n
+
+
+def test_status_strings_and_sizes():
+    assert atb.atb_status_string(0) == "ATB_OK"
+    assert atb.atb_status_string(8) == "ATB_ERR_DEVICE_TIMEOUT"
+    assert atb.atb_status_string(99) == "ATB_ERR_UNKNOWN"
+    assert atb.atb_bfp16_mant_bytes(100, 72) == 7200
+    assert atb.atb_bfp16_exp_bytes(100, 72) == 2 * 128 * 8
+    assert atb.atb_bfp16_exp_bytes(8192, 8192) == 8192 * 8192 // 8
+    assert atb.atb_bfp16_exp_bytes(0, 64) == 0
+
+
+def test_tiling_supported_rules():
+    ok = atb.atb_tiling_supported
+    assert ok(64, 128, 64, 128) and ok(128, 256, 64, 256) and ok(256, 256, 64, 256) and ok(32, 256, 64, 256)
+    assert not ok(256, 128, 64, 128)          # T_MA > T_MC
+    assert not ok(64, 192, 64, 128)           # T_MC not 128 / 256
+    assert not ok(64, 128, 32, 128)           # T_K
+    assert not ok(64, 128, 64, 96)            # T_N
+    # asymmetric buffering is what makes the deep K-step fit next to a 256-wide B tile
+    assert not ok(256, 256, 128, 256) and not ok(128, 256, 128, 256)
+    assert ok(64, 256, 128, 256) and ok(32, 256, 128, 256)
+
+
+def test_layout_helpers_roundtrip():
+    import numpy as np
+    rng = np.random.default_rng(0)
+    for (M, K) in [(100, 72), (32, 64), (33, 128), (1, 8)]:
+        e = rng.integers(0, 255, size=(M, K // 8)).astype(np.uint8)
+        plane = atb.logical_to_exp_plane(e, M, K)
+        assert plane.size == atb.atb_bfp16_exp_bytes(M, K)
+        assert np.array_equal(atb.exp_plane_to_logical(plane, M, K), e)
+        # documented address rule: ((p * M_pad) + m) * 8 + (kb % 8)
+        m_pad = -(-M // 32) * 32
+        for (m, kb) in [(0, 0), (M - 1, K // 8 - 1), (M // 2, (K // 8) // 2)]:
+            assert plane[((kb // 8) * m_pad + m) * 8 + kb % 8] == e[m, kb]
+
+
+def test_argument_validation_needs_no_gpu():
+    lib = atb.load_library()
+    assert lib.atb_quantize_bfp16(None, 8, 12, 12, None, None, None) == 2       # K % 8
+    assert lib.atb_quantize_bfp16(None, 0, 64, 64, None, None, None) == 0       # empty: no-op
+    assert lib.atb_gemm(128, 128, 64, 64, 128, 64, 128, None, None, None, 128, None, 128, None) == 1
+    assert atb.atb_last_error_message() != ""

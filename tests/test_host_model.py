@@ -1,0 +1,80 @@
+"""The library's host-side model (C++) against the oracle's restatement of Sections 3-5."""
+import math
+import os
+
+import pytest
+
+import paper_2511_16041_b200 as atb
+from oracle import model
+from tests.test_oracle_model import rows, _printed
+
+
+@pytest.mark.parametrize("r", rows(), ids=lambda r: f"{r['cfg']}-{r['T_MC']}x{r['T_K']}x{r['T_N']}-rho{r['rho']}")
+def test_xdna2_preset_reproduces_table2(r):
+    cfg = int(r["cfg"][1])
+    hw = atb.atb_hw_params_xdna2(cfg)
+    T_MA = r["T_MC"] // r["rho"]
+    s = atb.atb_score_tiling(hw, r["K"], (T_MA, r["T_MC"], r["T_K"], r["T_N"]))
+    assert abs(s.ai - r["ai"]) <= 0.5
+    assert abs(s.mem_bound_flops / 1e12 - r["mem"]) <= 0.075
+    if r["buf"] != "-":
+        assert _printed(s.buf_bytes_used / 1024, r["buf"])
+        assert s.feasible == 1
+        if r["rho"] > 1:
+            sym = atb.atb_score_tiling(hw, r["K"], (r["T_MC"], r["T_MC"], r["T_K"], r["T_N"]))
+            assert sym.feasible == 0
+
+
+def test_score_matches_oracle_formulas():
+    for hw in (atb.atb_hw_params_b200(), atb.atb_hw_params_xdna2(1), atb.atb_hw_params_xdna2(3)):
+        for t in [(32, 256, 64, 256), (128, 128, 128, 64), (64, 256, 128, 128), (256, 256, 64, 256)]:
+            for K in (256, 4096, 16384):
+                s = atb.atb_score_tiling(hw, K, t)
+                T_MA, T_MC, T_K, T_N = t
+                ai = model.ai_array(T_MC, T_N, K, hw.a_bytes, hw.b_bytes, hw.c_bytes, hw.share_rows, hw.share_cols)
+                em = model.eff_micro(T_K, hw.eta, hw.eps_cycles, hw.ii)
+                ec = model.eff_core(T_MA, T_MC, T_K, T_N, hw.peak_flops_per_cycle, em, hw.delta_cycles)
+                assert math.isclose(s.ai, ai, rel_tol=1e-12)
+                assert math.isclose(s.eff_micro, em, rel_tol=1e-12)
+                assert math.isclose(s.eff_core, ec, rel_tol=1e-12)
+                perf = model.perf_array(ai, hw.bw_bytes_per_s, ec, hw.peak_flops_per_cycle * hw.clock_hz, hw.n_units)
+                assert math.isclose(s.predicted_flops, perf, rel_tol=1e-12)
+                c_term = hw.c_buf_bytes * T_MC * T_N
+                buf = model.buffer_bytes(T_MA, T_MC, T_K, T_N, hw.a_buf_bytes, hw.b_buf_bytes, 0.0, hw.a_scratch_bytes)
+                if hw.acc_capacity_bytes > 0:
+                    assert math.isclose(s.buf_bytes_used, buf, rel_tol=1e-12)
+                    assert math.isclose(s.acc_bytes_used, c_term, rel_tol=1e-12)
+                else:
+                    assert math.isclose(s.buf_bytes_used, buf + c_term, rel_tol=1e-12)
+
+
+def test_select_tiling_orders_and_filters():
+    best, scores = atb.atb_select_tiling(8192, 8192, 8192)
+    assert atb.atb_tiling_supported(*best)
+    assert len(scores) >= 20
+    feas = [s for s in scores if s.feasible]
+    assert feas and all(a.predicted_flops >= b.predicted_flops for a, b in zip(feas, feas[1:]))
+    assert (scores[0].t.T_MA, scores[0].t.T_MC, scores[0].t.T_K, scores[0].t.T_N) == tuple(best)
+    for s in scores:                                   # only tilings the kernel accepts are proposed
+        assert atb.atb_tiling_supported(s.t.T_MA, s.t.T_MC, s.t.T_K, s.t.T_N)
+        assert s.predicted_flops <= min(s.mem_bound_flops, s.compute_bound_flops) * (1 + 1e-12)
+    # trade-off of Section 5: at fixed (T_MC, T_K, T_N) a larger rho never raises the compute bound,
+    # and AI does not depend on T_MA or T_K
+    by = {(s.t.T_MA, s.t.T_MC, s.t.T_K, s.t.T_N): s for s in scores}
+    assert by[(32, 256, 64, 256)].compute_bound_flops < by[(256, 256, 64, 256)].compute_bound_flops
+    assert by[(32, 256, 64, 256)].ai == by[(256, 256, 64, 256)].ai == by[(64, 256, 128, 256)].ai
+
+
+def test_select_tiling_small_problem_prefers_more_tiles():
+    # 1024 x 1024 has 16 tiles of 256 x 256 on 148 SMs: wave quantisation must show in the score
+    best, scores = atb.atb_select_tiling(1024, 1024, 8192)
+    big = [s for s in scores if (s.t.T_MC, s.t.T_N) == (256, 256)][0]
+    small = [s for s in scores if (s.t.T_MC, s.t.T_N) == (128, 64)][0]
+    assert small.compute_bound_flops > big.compute_bound_flops
+
+
+def test_select_tiling_errors():
+    lib = atb.load_library()
+    assert lib.atb_select_tiling(0, 8, 64, None, None, None, None) == 2
+    with pytest.raises(atb.AtbError):
+        atb.atb_score_tiling(atb.atb_hw_params_b200(), 64, (48, 128, 64, 128))
