@@ -119,6 +119,9 @@ CONFIGS = {
     "cfg3_8192": dict(M=8192, N=8192, K=8192, A="laplace", B="normal", b_scale=1.0),
     "cfg4_ffn_up": dict(M=16384, N=14336, K=4096, A="outlier", B="normal", b_scale=None),
     "cfg4_ffn_down": dict(M=16384, N=4096, K=14336, A="outlier", B="normal", b_scale=None),
+    # shallow-K cut of the headline shape: same tiles per wave, a quarter of the K-steps; small
+    # enough for a multi-pass profiler capture while operands + output still exceed the L2
+    "prof_8192x8192x2048": dict(M=8192, N=8192, K=2048, A="laplace", B="normal", b_scale=1.0),
 }
 
 

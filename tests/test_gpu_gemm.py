@@ -79,7 +79,7 @@ def test_small_integer_matrices_exact():
     b = rng.integers(-1, 2, size=(K, N)).astype(np.float32)
     mant, exp = oracle.quantize_bfp16(a)
     Cr, _ = oracle.gemm(mant, exp, inputs.to_bf16_bits(b))
-    for t in [(128, 128, 64, 128), (64, 256, 64, 256), (256, 256, 128, 64)]:
+    for t in [(128, 128, 64, 128), (64, 256, 64, 256), (64, 256, 128, 64)]:
         Cg = run_gemm(mant, exp, inputs.to_bf16_bits(b), t)
         assert np.array_equal(inputs.bf16_bits_to_f32(Cg).astype(np.float64), Cr), t
 
