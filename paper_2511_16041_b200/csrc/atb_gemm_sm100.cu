@@ -5,11 +5,11 @@
 // rho = T_MC / T_MA slabs of A are streamed through it; the FP32 accumulator of the whole
 // T_MC x T_N tile lives in tensor memory and is written out once, after K / T_K steps.
 //
-// Warp roles (448 threads):
+// Warp roles (704 threads):
 //   warp 0      TMA producer: B tiles and raw BFP16 A slabs (int8 mantissas + uint8 exponents)
 //   warp 1      UMMA issuer (one elected lane) and owner of the TMEM allocation
 //   warps 2-5   epilogue: tcgen05.ld -> round to bf16 -> global stores
-//   warps 6-13  dequantisers: raw slab -> bf16, K-major, 128-byte-swizzled operand in shared
+//   warps 6-21  dequantisers (two groups of 8 warps taking alternate slabs): raw slab -> bf16, K-major, 128-byte-swizzled operand in shared
 //               memory (exact: m * 2^(E-133) has at most 7 significant bits)
 // Rings, all guarded by mbarriers with bounded waits:
 //   B tiles          (n_b_stages)    producer -> UMMA          (freed by tcgen05.commit)
@@ -32,9 +32,11 @@ namespace {
 
 using namespace sm100;
 
-constexpr int kThreads = 448;
-constexpr int kDequantWarps = 8;
-constexpr int kDequantThreads = kDequantWarps * 32;
+constexpr int kDequantGroups = 2;                  // slabs alternate between the groups
+constexpr int kGroupWarps = 8;
+constexpr int kGroupThreads = kGroupWarps * 32;
+constexpr int kDequantWarps = kDequantGroups * kGroupWarps;
+constexpr int kThreads = (6 + kDequantWarps) * 32;
 constexpr int kFirstEpilogueWarp = 2;
 constexpr int kFirstDequantWarp = 6;
 constexpr int kMaxStages = 16;
@@ -105,68 +107,85 @@ struct Cfg {
     static constexpr uint32_t RAW_MANT_BYTES = T_MA * T_K;
     static constexpr uint32_t RAW_EXP_BYTES = T_MA * T_K / 8;
     static constexpr uint32_t RAW_BYTES = RAW_MANT_BYTES + RAW_EXP_BYTES;
-    static constexpr int BPR = T_K / 8;                        // blocks per slab row
-    static constexpr int DQ_ITERS = T_MA * BPR / kDequantThreads;
-    static_assert(T_MA * BPR % kDequantThreads == 0 && DQ_ITERS >= 1, "slab too small for the dequantisers");
+    static constexpr int SLOTS_PER_ROW = T_K / 16;             // a slot = 2 blocks = 16 mantissa bytes
+    static constexpr int SLOTS = T_MA * SLOTS_PER_ROW;
+    static constexpr int DQ_ITERS = (SLOTS + kGroupThreads - 1) / kGroupThreads;
+    static constexpr int ROWS_PER_ITER = kGroupThreads / SLOTS_PER_ROW;
 };
 
 // ---------------------------------------------------------------------------------------------
 // Dequantise one raw slab (T_MA rows x T_K columns) into its place in a bf16 operand group.
-// Thread t owns block (row r, block kb) = (t / BPR + i * 256 / BPR, t % BPR): the raw reads of a
-// warp are contiguous, and the 16-byte stores of 8 consecutive threads fill one 128-byte row.
+// One group of 256 threads works on a slab.  Thread t owns slot (row r, pair p) = (t / SPR + i *
+// 256 / SPR, t % SPR), a slot being two blocks: 16 mantissa bytes (one 16-byte load; the loads of
+// a warp are contiguous), two exponent bytes, and two 16-byte stores into the swizzled row.
+//
+// Per element: the byte u = m + 128 is dropped into the mantissa of the float 2^23 (bit pattern
+// 0x4B0000uu = 2^23 + u); subtracting 2^23 + 128 leaves m exactly, and the product with the
+// block scale 2^(E-133) (taken from a 256-entry table: normal for E >= 7, fp32-subnormal below) is
+// exact for every E.  The result has at most 7 significant bits, so its low 16 bits are zero and
+// the bf16 value is the upper half of the word.
+__device__ __forceinline__ uint64_t pack_f32x2(uint32_t lo, uint32_t hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+    return r;
+}
+
+// bf16x2 of (m0, m1) * scale for bytes `sel0`, `sel0 + 1` of the biased word u.
+__device__ __forceinline__ uint32_t dequant_pair(uint32_t u, uint32_t sel0, uint64_t neg_magic2, uint64_t scale2) {
+    const uint32_t x0 = __byte_perm(u, 0x4B000000u, 0x7650u + sel0);
+    const uint32_t x1 = __byte_perm(u, 0x4B000000u, 0x7651u + sel0);
+    uint64_t d, r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(pack_f32x2(x0, x1)), "l"(neg_magic2));
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(d), "l"(scale2));
+    uint32_t f0, f1;
+    asm("mov.b64 {%0, %1}, %2;" : "=r"(f0), "=r"(f1) : "l"(r));
+    return __byte_perm(f0, f1, 0x7632);
+}
+
 template <class C>
-__device__ __forceinline__ void dequant_slab(const uint8_t* raw_mant, const uint8_t* raw_exp,
-                                             uint32_t dst_base, int row_base, int t,
-                                             int T_MA_rows) {
-    const int kb = t % C::BPR;
-    const int r0 = t / C::BPR;
-    uint2 w[C::DQ_ITERS];
+__device__ __forceinline__ void dequant_slab(uint32_t raw_mant, uint32_t raw_exp, uint32_t scale_lut,
+                                             uint32_t dst_base, int row_base, int t, int T_MA_rows) {
+    const int p = t % C::SLOTS_PER_ROW;                 // blocks 2p, 2p + 1 of the row
+    const int r0 = t / C::SLOTS_PER_ROW;
+    const int kb = 2 * p;
+    uint4 w[C::DQ_ITERS];
     uint32_t e[C::DQ_ITERS];
 #pragma unroll
     for (int i = 0; i < C::DQ_ITERS; ++i) {
-        const int r = r0 + i * (kDequantThreads / C::BPR);
-        w[i] = *reinterpret_cast<const uint2*>(raw_mant + (r * C::BPR + kb) * 8);
-        e[i] = raw_exp[(kb >> 3) * T_MA_rows * 8 + r * 8 + (kb & 7)];
+        const int r = r0 + i * C::ROWS_PER_ITER;
+        if (C::SLOTS % kGroupThreads == 0 || r < T_MA_rows) {
+            asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                         : "=r"(w[i].x), "=r"(w[i].y), "=r"(w[i].z), "=r"(w[i].w)
+                         : "r"(raw_mant + (r * C::SLOTS_PER_ROW + p) * 16));
+            uint16_t e2;
+            asm volatile("ld.shared.u16 %0, [%1];" : "=h"(e2)
+                         : "r"(raw_exp + (kb >> 3) * T_MA_rows * 8 + r * 8 + (kb & 7)));
+            e[i] = e2;
+        }
     }
+    const uint64_t neg_magic2 = pack_f32x2(0xCB000080u, 0xCB000080u);    // -(2^23 + 128), twice
 #pragma unroll
     for (int i = 0; i < C::DQ_ITERS; ++i) {
-        const int r = r0 + i * (kDequantThreads / C::BPR);
-        const uint32_t E = e[i];
-        // scale 2^(E-133): a normal fp32 for E >= 7, an fp32 subnormal below.
-        const uint32_t s_bits = (E >= 7u) ? ((E - 6u) << 23) : (1u << (E + 16u));
-        const float s = __uint_as_float(s_bits);
-        const uint32_t u0 = w[i].x ^ 0x80808080u, u1 = w[i].y ^ 0x80808080u;   // m + 128 per byte
-        float f[8];
-        // 0x4B0000uu is the float 2^23 + u; (2^23 + u) * s - (2^23 + 128) * s = m * s exactly.
-        const float x0 = __uint_as_float(__byte_perm(u0, 0x4B000000u, 0x7650));
-        const float x1 = __uint_as_float(__byte_perm(u0, 0x4B000000u, 0x7651));
-        const float x2 = __uint_as_float(__byte_perm(u0, 0x4B000000u, 0x7652));
-        const float x3 = __uint_as_float(__byte_perm(u0, 0x4B000000u, 0x7653));
-        const float x4 = __uint_as_float(__byte_perm(u1, 0x4B000000u, 0x7650));
-        const float x5 = __uint_as_float(__byte_perm(u1, 0x4B000000u, 0x7651));
-        const float x6 = __uint_as_float(__byte_perm(u1, 0x4B000000u, 0x7652));
-        const float x7 = __uint_as_float(__byte_perm(u1, 0x4B000000u, 0x7653));
-        if (E < 238u) {
-            const float c = -8388736.0f * s;
-            f[0] = fmaf(x0, s, c); f[1] = fmaf(x1, s, c); f[2] = fmaf(x2, s, c); f[3] = fmaf(x3, s, c);
-            f[4] = fmaf(x4, s, c); f[5] = fmaf(x5, s, c); f[6] = fmaf(x6, s, c); f[7] = fmaf(x7, s, c);
-        } else {   // (2^23 + 128) * s would overflow: subtract first (exact), then scale (exact)
-            f[0] = (x0 - 8388736.0f) * s; f[1] = (x1 - 8388736.0f) * s;
-            f[2] = (x2 - 8388736.0f) * s; f[3] = (x3 - 8388736.0f) * s;
-            f[4] = (x4 - 8388736.0f) * s; f[5] = (x5 - 8388736.0f) * s;
-            f[6] = (x6 - 8388736.0f) * s; f[7] = (x7 - 8388736.0f) * s;
+        const int r = r0 + i * C::ROWS_PER_ITER;
+        if (C::SLOTS % kGroupThreads == 0 || r < T_MA_rows) {
+            uint32_t s0, s1;
+            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(s0) : "r"(scale_lut + (e[i] & 0xFFu) * 4));
+            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(s1) : "r"(scale_lut + (e[i] >> 8) * 4));
+            const uint64_t sc0 = pack_f32x2(s0, s0), sc1 = pack_f32x2(s1, s1);
+            const uint32_t u0 = w[i].x ^ 0x80808080u, u1 = w[i].y ^ 0x80808080u;
+            const uint32_t u2 = w[i].z ^ 0x80808080u, u3 = w[i].w ^ 0x80808080u;
+            const int rr = row_base + r;
+            const uint32_t row_addr = dst_base + (rr >> 7) * C::GROUP_BYTES + (kb >> 3) * C::KHALF_BYTES + (rr & 127) * 128;
+            const uint32_t sw = static_cast<uint32_t>(rr & 7);
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row_addr + ((((kb & 7)) ^ sw) << 4)),
+                         "r"(dequant_pair(u0, 0, neg_magic2, sc0)), "r"(dequant_pair(u0, 2, neg_magic2, sc0)),
+                         "r"(dequant_pair(u1, 0, neg_magic2, sc0)), "r"(dequant_pair(u1, 2, neg_magic2, sc0))
+                         : "memory");
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row_addr + ((((kb & 7) + 1) ^ sw) << 4)),
+                         "r"(dequant_pair(u2, 0, neg_magic2, sc1)), "r"(dequant_pair(u2, 2, neg_magic2, sc1)),
+                         "r"(dequant_pair(u3, 0, neg_magic2, sc1)), "r"(dequant_pair(u3, 2, neg_magic2, sc1))
+                         : "memory");
         }
-        __nv_bfloat162 p0 = __floats2bfloat162_rn(f[0], f[1]);
-        __nv_bfloat162 p1 = __floats2bfloat162_rn(f[2], f[3]);
-        __nv_bfloat162 p2 = __floats2bfloat162_rn(f[4], f[5]);
-        __nv_bfloat162 p3 = __floats2bfloat162_rn(f[6], f[7]);
-        const int rr = row_base + r;
-        const uint32_t dst = dst_base + (rr >> 7) * C::GROUP_BYTES + (kb >> 3) * C::KHALF_BYTES +
-                             (rr & 127) * 128 + ((((kb & 7) ^ (rr & 7))) << 4);
-        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst),
-                     "r"(*reinterpret_cast<uint32_t*>(&p0)), "r"(*reinterpret_cast<uint32_t*>(&p1)),
-                     "r"(*reinterpret_cast<uint32_t*>(&p2)), "r"(*reinterpret_cast<uint32_t*>(&p3))
-                     : "memory");
     }
 }
 
@@ -195,6 +214,7 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
     const uint32_t deq_full = raw_empty + 8 * p.n_raw_stages, deq_empty = deq_full + 8 * n_deq_stages;
     const uint32_t acc_full = deq_empty + 8 * n_deq_stages, acc_empty = acc_full + 8 * n_acc;
     const uint32_t misc = acc_empty + 8 * n_acc;             // [0]: TMEM base, [1]: abort flag
+    const uint32_t scale_lut = misc + 16;                    // 256 floats: 2^(E-133)
     volatile uint32_t* const misc_gen = reinterpret_cast<volatile uint32_t*>(smem_gen + (misc - smem_base));
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -202,8 +222,8 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < p.n_b_stages; ++i) { mbar_init(b_full + 8 * i, 1); mbar_init(b_empty + 8 * i, 1); }
-        for (int i = 0; i < p.n_raw_stages; ++i) { mbar_init(raw_full + 8 * i, 1); mbar_init(raw_empty + 8 * i, kDequantWarps); }
-        for (int i = 0; i < n_deq_stages; ++i) { mbar_init(deq_full + 8 * i, kDequantWarps); mbar_init(deq_empty + 8 * i, 1); }
+        for (int i = 0; i < p.n_raw_stages; ++i) { mbar_init(raw_full + 8 * i, 1); mbar_init(raw_empty + 8 * i, kGroupWarps); }
+        for (int i = 0; i < n_deq_stages; ++i) { mbar_init(deq_full + 8 * i, kGroupWarps); mbar_init(deq_empty + 8 * i, 1); }
         for (int i = 0; i < n_acc; ++i) { mbar_init(acc_full + 8 * i, 1); mbar_init(acc_empty + 8 * i, 4); }
         misc_gen[1] = 0u;
         fence_mbar_init();
@@ -214,6 +234,11 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
     if (warp == 1) {
         tmem_alloc(misc, static_cast<uint32_t>(p.tmem_cols));
         tmem_relinquish();
+    }
+    if (threadIdx.x >= kFirstDequantWarp * 32 && threadIdx.x < kFirstDequantWarp * 32 + 256) {
+        const uint32_t E = threadIdx.x - kFirstDequantWarp * 32;
+        const uint32_t bits = (E >= 7u) ? ((E - 6u) << 23) : (1u << (E + 16u));
+        asm volatile("st.shared.b32 [%0], %1;" ::"r"(scale_lut + E * 4), "r"(E == 255u ? 0u : bits) : "memory");
     }
     tcgen05_fence_before_sync();
     __syncthreads();
@@ -347,15 +372,21 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
         }
     } else {
         // ================================ dequantisers ================================
-        const int t = threadIdx.x - kFirstDequantWarp * 32;
+        const int t = (threadIdx.x - kFirstDequantWarp * 32) % kGroupThreads;
+        const int my_group = (threadIdx.x - kFirstDequantWarp * 32) / kGroupThreads;
         Ring rr, rd;
+        for (int i = 0; i < my_group; ++i) { rr.advance(p.n_raw_stages); rd.advance(n_deq_stages); }
+        int turn = 0;                                   // slab sequence number modulo the group count
         bool ok = true;
         for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
             for (int k = 0; ok && k < p.k_steps; ++k) {
                 for (int s = 0; s < C::RHO; ++s) {
+                    const bool mine = (turn == my_group);
+                    if (++turn == kDequantGroups) turn = 0;
+                    if (!mine) continue;
                     if (!(ok = wait_bar(cx, raw_full + 8 * rr.stage, rr.phase, 0x301))) break;
                     if (!(ok = wait_bar(cx, deq_empty + 8 * rd.stage, rd.phase ^ 1u, 0x302))) break;
-                    const uint8_t* raw = smem_gen + raw_off + rr.stage * C::RAW_BYTES;
+                    const uint32_t raw = raw_base + rr.stage * C::RAW_BYTES;
                     uint32_t dst_base;
                     int row_base;
                     if (T_MA <= 128) {
@@ -365,15 +396,14 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
                         dst_base = deq_base + rd.stage * C::GPS * C::GROUP_BYTES;
                         row_base = 0;
                     }
-                    dequant_slab<C>(raw, raw + C::RAW_MANT_BYTES, dst_base, row_base, t, T_MA);
+                    dequant_slab<C>(raw, raw + C::RAW_MANT_BYTES, scale_lut, dst_base, row_base, t, T_MA);
                     fence_proxy_async_smem();
                     __syncwarp();
                     if (lane == 0) {
                         mbar_arrive(deq_full + 8 * rd.stage);
                         mbar_arrive(raw_empty + 8 * rr.stage);
                     }
-                    rr.advance(p.n_raw_stages);
-                    rd.advance(n_deq_stages);
+                    for (int i = 0; i < kDequantGroups; ++i) { rr.advance(p.n_raw_stages); rd.advance(n_deq_stages); }
                 }
             }
         }
@@ -507,7 +537,7 @@ bool plan_gemm(int T_MA, int T_MC, int T_K, int T_N, GemmPlan* plan) {
     int nb = 2, ng = 2 * gps, nr = 2;
     auto total = [&](int b, int g, int r) {
         const int n_deq = T_MA <= 128 ? g * spg : g / gps;
-        const uint32_t bars = 8u * (2 * b + 2 * r + 2 * n_deq + 2 * 2 * G) + 16u;
+        const uint32_t bars = 8u * (2 * b + 2 * r + 2 * n_deq + 2 * 2 * G) + 16u + 1024u;
         return 1024u + b * b_bytes + g * group_bytes + r * raw_bytes + bars;
     };
     if (total(nb, ng, nr) > kSmemBudget) return false;
