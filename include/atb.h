@@ -78,7 +78,7 @@ atb_status_t atb_quantize_bfp16(const float* A_dev, int64_t M, int64_t K, int64_
  *   B_bf16_dev: bf16 B[K][ldb] row-major, ldb >= N, ldb % 8 == 0, 16-byte aligned;
  *   C_bf16_dev: bf16 C[M][ldc] row-major, ldc >= N, ldc % 8 == 0, 16-byte aligned (written).
  * Shapes: M, N >= 1 (any value; edge tiles are handled), N % 8 == 0, K >= 64 and K % 64 == 0.
- * Tilings: T_MC in {128, 256}; T_N in {64, 128, 256}; T_K in {64, 128};
+ * Tilings: T_MC in {128, 256}; T_N in {64, 128, 256, 512}; T_K in {64, 128};
  *          T_MA in {32, 64, 128, 256} with T_MA <= T_MC; (T_MC / 128) * T_N <= 512 (the FP32
  *          accumulator must fit the 512 TMEM columns); the shared-memory rings must fit 227 KB.
  *          atb_tiling_supported() tells in advance.
@@ -92,6 +92,21 @@ atb_status_t atb_gemm(int64_t M, int64_t N, int64_t K, int T_MA, int T_MC, int T
 /* 1 if atb_gemm accepts the tiling (kernel exists, TMEM and shared-memory budgets met), else 0.
  * Host only; touches no device. */
 int atb_tiling_supported(int T_MA, int T_MC, int T_K, int T_N);
+
+/* How atb_gemm lays a tiling out on the SM (host only; for documentation, tests and tuning).
+ * The rings are the B200 counterpart of the buffers of Eq. 1: B tiles of T_K x T_N, raw BFP16 A
+ * slabs of T_MA x T_K, and dequantised BF16 A in 128-row groups of T_K columns. */
+typedef struct {
+    int n_b_stages;      /* depth of the B-tile ring                                              */
+    int n_raw_stages;    /* depth of the raw A-slab ring (a multiple of dequant_groups)           */
+    int n_a_groups;      /* depth of the dequantised-A ring, in 128-row groups                    */
+    int dequant_groups;  /* groups the 16 dequantiser warps are split into; slabs take turns      */
+    int acc_buffers;     /* T_MC x T_N FP32 accumulators resident in TMEM (1 or 2)                */
+    int tmem_columns;    /* TMEM columns allocated (power of two <= 512)                          */
+    int smem_bytes;      /* dynamic shared memory of the launch                                   */
+} atb_plan_t;
+/* Returns ATB_ERR_BAD_TILING if atb_gemm does not support the tiling. */
+atb_status_t atb_tiling_plan(int T_MA, int T_MC, int T_K, int T_N, atb_plan_t* plan);
 
 /* Waits for `stream` and reports whether any kernel of this library launched by this process on
  * the current device gave up a bounded wait since the last call (every wait on an mbarrier in the

@@ -15,7 +15,7 @@ import os
 from typing import NamedTuple
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libatb.so")
+LIB_PATH = os.environ.get("ATB_LIBRARY_PATH") or os.path.join(_HERE, "libatb.so")
 _lib = None
 
 ATB_OK = 0
@@ -51,6 +51,11 @@ class atb_tiling_score_t(ctypes.Structure):
                                                "mem_bound_flops", "compute_bound_flops", "predicted_flops")]
 
 
+class atb_plan_t(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int) for n in ("n_b_stages", "n_raw_stages", "n_a_groups", "dequant_groups",
+                                            "acc_buffers", "tmem_columns", "smem_bytes")]
+
+
 class Tiling(NamedTuple):
     T_MA: int
     T_MC: int
@@ -60,7 +65,7 @@ class Tiling(NamedTuple):
 
 EXPORTED_SYMBOLS = [
     "atb_status_string", "atb_last_error_message", "atb_bfp16_mant_bytes", "atb_bfp16_exp_bytes",
-    "atb_quantize_bfp16", "atb_gemm", "atb_tiling_supported", "atb_device_status",
+    "atb_quantize_bfp16", "atb_gemm", "atb_tiling_supported", "atb_tiling_plan", "atb_device_status",
     "atb_hw_params_b200", "atb_hw_params_xdna2", "atb_score_tiling", "atb_select_tiling",
 ]
 
@@ -88,6 +93,8 @@ def load_library():
     lib.atb_gemm.argtypes = [i64, i64, i64, ci, ci, ci, ci, vp, vp, vp, i64, vp, i64, vp]
     lib.atb_tiling_supported.restype = ci
     lib.atb_tiling_supported.argtypes = [ci, ci, ci, ci]
+    lib.atb_tiling_plan.restype = ci
+    lib.atb_tiling_plan.argtypes = [ci, ci, ci, ci, ctypes.POINTER(atb_plan_t)]
     lib.atb_device_status.restype = ci
     lib.atb_device_status.argtypes = [vp]
     lib.atb_hw_params_b200.restype = None
@@ -142,6 +149,12 @@ def atb_bfp16_exp_bytes(M: int, K: int) -> int:
 
 def atb_tiling_supported(T_MA: int, T_MC: int, T_K: int, T_N: int) -> bool:
     return bool(load_library().atb_tiling_supported(T_MA, T_MC, T_K, T_N))
+
+
+def atb_tiling_plan(T_MA: int, T_MC: int, T_K: int, T_N: int) -> atb_plan_t:
+    plan = atb_plan_t()
+    _check(load_library().atb_tiling_plan(T_MA, T_MC, T_K, T_N, ctypes.byref(plan)))
+    return plan
 
 
 # ------------------------------------------------------------------ device calls

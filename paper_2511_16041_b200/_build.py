@@ -37,6 +37,7 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
               "-I", os.path.join(ROOT, "include"), "-I", CSRC]
     if verbose:
         common += ["-Xptxas", "-v"]
+    common += os.environ.get("ATB_NVCC_FLAGS", "").split()
     procs = []
     for src in SOURCES:
         obj = os.path.join(CSRC, os.path.splitext(src)[0] + ".o")

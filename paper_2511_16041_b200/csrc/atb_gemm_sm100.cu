@@ -28,15 +28,28 @@
 #include "atb_internal.h"
 #include "sm100_ptx.cuh"
 
+#ifndef ATB_PACK_F2FP
+#define ATB_PACK_F2FP 0
+#endif
+
 namespace {
 
 using namespace sm100;
 
-constexpr int kDequantGroups = 2;                  // slabs alternate between the groups
-constexpr int kGroupWarps = 8;
-constexpr int kGroupThreads = kGroupWarps * 32;
-constexpr int kDequantWarps = kDequantGroups * kGroupWarps;
+constexpr int kDequantWarps = 16;
 constexpr int kThreads = (6 + kDequantWarps) * 32;
+// The dequantiser warps work in groups; slabs are dealt to the groups in turn, so that several
+// slabs are in flight and every thread has a few 16-element slots per barrier round trip.
+// Ring depths are multiples of the group count: a ring stage is then always served by the same
+// group, which keeps each mbarrier's phases strictly in order for its waiters.
+__host__ __device__ constexpr int dq_groups(int T_MA, int T_K, int T_N) {
+#ifdef ATB_DQ_GROUPS
+    return ATB_DQ_GROUPS;
+#else
+    // two groups for big slabs, and where a double-buffered B tile already takes 128 KB
+    return (T_MA * T_K >= 256 * 64 || T_K * T_N >= 128 * 256) ? 2 : 4;
+#endif
+}
 constexpr int kFirstEpilogueWarp = 2;
 constexpr int kFirstDequantWarp = 6;
 constexpr int kMaxStages = 16;
@@ -68,12 +81,15 @@ struct Ctx {
 };
 
 // Bounded mbarrier wait.  Returns false when the CTA is aborting or the wait timed out.
+// The first probes are immediate; after that the thread lets the hardware suspend it for up to
+// `kSuspendNs` per probe, so that waiting roles do not take issue slots from the dequantisers.
+constexpr uint32_t kSuspendNs = 20000;
 __device__ __forceinline__ bool wait_bar(const Ctx& cx, uint32_t bar, uint32_t parity, unsigned code) {
     if (mbar_try_wait(bar, parity)) return true;
     const uint64_t t0 = global_timer_ns();
     for (uint32_t spins = 0;; ++spins) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((spins & 63u) == 63u) {
+        if (mbar_try_wait_suspend(bar, parity, kSuspendNs)) return true;
+        if ((spins & 7u) == 7u) {
             if (*cx.abort_flag) return false;
             if (global_timer_ns() - t0 > kWaitTimeoutNs) {
                 *cx.abort_flag = 1u;
@@ -100,6 +116,8 @@ struct Cfg {
     static constexpr int RHO = T_MC / T_MA;                    // slabs per K-step
     static constexpr int SPG = (T_MA < 128) ? 128 / T_MA : 1;  // slabs per group
     static constexpr int GPS = (T_MA > 128) ? T_MA / 128 : 1;  // groups per slab
+    static constexpr int N_MMA = T_N > 256 ? 256 : T_N;        // UMMA N extent; T_N / N_MMA instructions side by side
+    static constexpr int N_CHUNKS = T_N / N_MMA;
     static constexpr uint32_t B_BYTES = T_K * T_N * 2;
     static constexpr uint32_t B_BOX_BYTES = T_K * 128;         // one 64-column box of B
     static constexpr uint32_t GROUP_BYTES = 128 * T_K * 2;
@@ -109,14 +127,17 @@ struct Cfg {
     static constexpr uint32_t RAW_BYTES = RAW_MANT_BYTES + RAW_EXP_BYTES;
     static constexpr int SLOTS_PER_ROW = T_K / 16;             // a slot = 2 blocks = 16 mantissa bytes
     static constexpr int SLOTS = T_MA * SLOTS_PER_ROW;
-    static constexpr int DQ_ITERS = (SLOTS + kGroupThreads - 1) / kGroupThreads;
-    static constexpr int ROWS_PER_ITER = kGroupThreads / SLOTS_PER_ROW;
+    static constexpr int DQ_GROUPS = dq_groups(T_MA, T_K, T_N);
+    static constexpr int GROUP_WARPS = kDequantWarps / DQ_GROUPS;
+    static constexpr int GROUP_THREADS = GROUP_WARPS * 32;
+    static constexpr int DQ_ITERS = (SLOTS + GROUP_THREADS - 1) / GROUP_THREADS;
+    static constexpr int ROWS_PER_ITER = GROUP_THREADS / SLOTS_PER_ROW;
 };
 
 // ---------------------------------------------------------------------------------------------
 // Dequantise one raw slab (T_MA rows x T_K columns) into its place in a bf16 operand group.
-// One group of 256 threads works on a slab.  Thread t owns slot (row r, pair p) = (t / SPR + i *
-// 256 / SPR, t % SPR), a slot being two blocks: 16 mantissa bytes (one 16-byte load; the loads of
+// One group of dequantiser warps (GROUP_THREADS threads) works on a slab.  Thread t owns slot (row r, pair p) = (t / SPR + i *
+// GROUP_THREADS / SPR, t % SPR), a slot being two blocks: 16 mantissa bytes (one 16-byte load; the loads of
 // a warp are contiguous), two exponent bytes, and two 16-byte stores into the swizzled row.
 //
 // Per element: the byte u = m + 128 is dropped into the mantissa of the float 2^23 (bit pattern
@@ -139,7 +160,13 @@ __device__ __forceinline__ uint32_t dequant_pair(uint32_t u, uint32_t sel0, uint
     asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(d), "l"(scale2));
     uint32_t f0, f1;
     asm("mov.b64 {%0, %1}, %2;" : "=r"(f0), "=r"(f1) : "l"(r));
+#if ATB_PACK_F2FP
+    uint32_t pk;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(pk) : "f"(__uint_as_float(f1)), "f"(__uint_as_float(f0)));
+    return pk;
+#else
     return __byte_perm(f0, f1, 0x7632);
+#endif
 }
 
 template <class C>
@@ -153,7 +180,7 @@ __device__ __forceinline__ void dequant_slab(uint32_t raw_mant, uint32_t raw_exp
 #pragma unroll
     for (int i = 0; i < C::DQ_ITERS; ++i) {
         const int r = r0 + i * C::ROWS_PER_ITER;
-        if (C::SLOTS % kGroupThreads == 0 || r < T_MA_rows) {
+        if (C::SLOTS % C::GROUP_THREADS == 0 || r < T_MA_rows) {
             asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
                          : "=r"(w[i].x), "=r"(w[i].y), "=r"(w[i].z), "=r"(w[i].w)
                          : "r"(raw_mant + (r * C::SLOTS_PER_ROW + p) * 16));
@@ -167,7 +194,7 @@ __device__ __forceinline__ void dequant_slab(uint32_t raw_mant, uint32_t raw_exp
 #pragma unroll
     for (int i = 0; i < C::DQ_ITERS; ++i) {
         const int r = r0 + i * C::ROWS_PER_ITER;
-        if (C::SLOTS % kGroupThreads == 0 || r < T_MA_rows) {
+        if (C::SLOTS % C::GROUP_THREADS == 0 || r < T_MA_rows) {
             uint32_t s0, s1;
             asm volatile("ld.shared.b32 %0, [%1];" : "=r"(s0) : "r"(scale_lut + (e[i] & 0xFFu) * 4));
             asm volatile("ld.shared.b32 %0, [%1];" : "=r"(s1) : "r"(scale_lut + (e[i] >> 8) * 4));
@@ -222,8 +249,8 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < p.n_b_stages; ++i) { mbar_init(b_full + 8 * i, 1); mbar_init(b_empty + 8 * i, 1); }
-        for (int i = 0; i < p.n_raw_stages; ++i) { mbar_init(raw_full + 8 * i, 1); mbar_init(raw_empty + 8 * i, kGroupWarps); }
-        for (int i = 0; i < n_deq_stages; ++i) { mbar_init(deq_full + 8 * i, kGroupWarps); mbar_init(deq_empty + 8 * i, 1); }
+        for (int i = 0; i < p.n_raw_stages; ++i) { mbar_init(raw_full + 8 * i, 1); mbar_init(raw_empty + 8 * i, C::GROUP_WARPS); }
+        for (int i = 0; i < n_deq_stages; ++i) { mbar_init(deq_full + 8 * i, C::GROUP_WARPS); mbar_init(deq_empty + 8 * i, 1); }
         for (int i = 0; i < n_acc; ++i) { mbar_init(acc_full + 8 * i, 1); mbar_init(acc_empty + 8 * i, 4); }
         misc_gen[1] = 0u;
         fence_mbar_init();
@@ -279,7 +306,7 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
     } else if (warp == 1) {
         // ================================ UMMA issuer =================================
         if (elect_one()) {
-            constexpr uint32_t idesc = umma_idesc_bf16_f32(128, T_N, false, true);
+            constexpr uint32_t idesc = umma_idesc_bf16_f32(128, C::N_MMA, false, true);
             Ring rb, rd;
             int it = 0;
             bool ok = true;
@@ -306,10 +333,14 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
                         const uint32_t as = deq_base + group_slot * C::GROUP_BYTES;
                         const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * T_N);
 #pragma unroll
-                        for (int kk = 0; kk < T_K / 16; ++kk) {
-                            const uint64_t a_desc = umma_smem_desc_sw128(as + (kk >> 2) * C::KHALF_BYTES + (kk & 3) * 32, 16, 1024);
-                            const uint64_t b_desc = umma_smem_desc_sw128(bs + kk * 2048, C::B_BOX_BYTES, 1024);
-                            umma_f16_ss(d_tmem, a_desc, b_desc, idesc, (k > 0 || kk > 0) ? 1u : 0u);
+                        for (int nc = 0; nc < C::N_CHUNKS; ++nc) {
+#pragma unroll
+                            for (int kk = 0; kk < T_K / 16; ++kk) {
+                                const uint64_t a_desc = umma_smem_desc_sw128(as + (kk >> 2) * C::KHALF_BYTES + (kk & 3) * 32, 16, 1024);
+                                const uint64_t b_desc = umma_smem_desc_sw128(bs + nc * (C::N_MMA / 64) * C::B_BOX_BYTES + kk * 2048,
+                                                                             C::B_BOX_BYTES, 1024);
+                                umma_f16_ss(d_tmem + nc * C::N_MMA, a_desc, b_desc, idesc, (k > 0 || kk > 0) ? 1u : 0u);
+                            }
                         }
                         if (T_MA <= 128) {
                             for (int i = 0; i < C::SPG; ++i) umma_commit(deq_empty + 8 * (rd.stage + i));
@@ -372,8 +403,8 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
         }
     } else {
         // ================================ dequantisers ================================
-        const int t = (threadIdx.x - kFirstDequantWarp * 32) % kGroupThreads;
-        const int my_group = (threadIdx.x - kFirstDequantWarp * 32) / kGroupThreads;
+        const int t = (threadIdx.x - kFirstDequantWarp * 32) % C::GROUP_THREADS;
+        const int my_group = (threadIdx.x - kFirstDequantWarp * 32) / C::GROUP_THREADS;
         Ring rr, rd;
         for (int i = 0; i < my_group; ++i) { rr.advance(p.n_raw_stages); rd.advance(n_deq_stages); }
         int turn = 0;                                   // slab sequence number modulo the group count
@@ -382,7 +413,7 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
             for (int k = 0; ok && k < p.k_steps; ++k) {
                 for (int s = 0; s < C::RHO; ++s) {
                     const bool mine = (turn == my_group);
-                    if (++turn == kDequantGroups) turn = 0;
+                    if (++turn == C::DQ_GROUPS) turn = 0;
                     if (!mine) continue;
                     if (!(ok = wait_bar(cx, raw_full + 8 * rr.stage, rr.phase, 0x301))) break;
                     if (!(ok = wait_bar(cx, deq_empty + 8 * rd.stage, rd.phase ^ 1u, 0x302))) break;
@@ -403,7 +434,7 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
                         mbar_arrive(deq_full + 8 * rd.stage);
                         mbar_arrive(raw_empty + 8 * rr.stage);
                     }
-                    for (int i = 0; i < kDequantGroups; ++i) { rr.advance(p.n_raw_stages); rd.advance(n_deq_stages); }
+                    for (int i = 0; i < C::DQ_GROUPS; ++i) { rr.advance(p.n_raw_stages); rd.advance(n_deq_stages); }
                 }
             }
         }
@@ -526,7 +557,7 @@ namespace atb {
 
 bool plan_gemm(int T_MA, int T_MC, int T_K, int T_N, GemmPlan* plan) {
     if (!(T_MC == 128 || T_MC == 256)) return false;
-    if (!(T_N == 64 || T_N == 128 || T_N == 256)) return false;
+    if (!(T_N == 64 || T_N == 128 || T_N == 256 || T_N == 512)) return false;
     if (!(T_K == 64 || T_K == 128)) return false;
     if (!(T_MA == 32 || T_MA == 64 || T_MA == 128 || T_MA == 256) || T_MA > T_MC) return false;
     const int G = T_MC / 128;
@@ -534,12 +565,18 @@ bool plan_gemm(int T_MA, int T_MC, int T_K, int T_N, GemmPlan* plan) {
     const uint32_t b_bytes = T_K * T_N * 2, group_bytes = 128 * T_K * 2, raw_bytes = T_MA * T_K * 9 / 8;
     const int gps = T_MA > 128 ? T_MA / 128 : 1;          // groups per slab
     const int spg = T_MA < 128 ? 128 / T_MA : 1;          // slabs per group
-    int nb = 2, ng = 2 * gps, nr = 2;
+    // The raw-slab ring and the ring of dequantised slab stages come in multiples of the
+    // dequantiser group count (see dq_groups); the bf16 ring itself is counted in 128-row groups.
+    const int dqg = dq_groups(T_MA, T_K, T_N);
+    const int nr_step = dqg;
+    const int ng_step = T_MA <= 128 ? (dqg >= spg ? dqg / spg : 1) : dqg * gps;
     auto total = [&](int b, int g, int r) {
         const int n_deq = T_MA <= 128 ? g * spg : g / gps;
         const uint32_t bars = 8u * (2 * b + 2 * r + 2 * n_deq + 2 * 2 * G) + 16u + 1024u;
         return 1024u + b * b_bytes + g * group_bytes + r * raw_bytes + bars;
     };
+    int nb = 2, ng = ng_step, nr = nr_step;
+    if (ng < 2) ng = 2 * ng_step;
     if (total(nb, ng, nr) > kSmemBudget) return false;
     // Grow the rings towards a target look-ahead, counted in 128-row x T_K operand groups:
     // B tiles hide the TMA latency for G groups each, raw slabs for T_MA/128 groups each.
@@ -549,11 +586,12 @@ bool plan_gemm(int T_MA, int T_MC, int T_K, int T_N, GemmPlan* plan) {
         int pick = -1;
         double best = 1.0;                               // stop once every ring meets its target
         if (cov_b < best && nb < kMaxStages && total(nb + 1, ng, nr) <= kSmemBudget) { best = cov_b; pick = 0; }
-        if (cov_r < best && nr < kMaxStages && total(nb, ng, nr + 1) <= kSmemBudget) { best = cov_r; pick = 1; }
-        if (cov_g < best && ng + gps <= kMaxStages && total(nb, ng + gps, nr) <= kSmemBudget) { best = cov_g; pick = 2; }
+        if (cov_r < best && nr + nr_step <= kMaxStages && total(nb, ng, nr + nr_step) <= kSmemBudget) { best = cov_r; pick = 1; }
+        if (cov_g < best && ng + ng_step <= kMaxStages && total(nb, ng + ng_step, nr) <= kSmemBudget) { best = cov_g; pick = 2; }
         if (pick < 0) break;
-        if (pick == 0) ++nb; else if (pick == 1) ++nr; else ng += gps;
+        if (pick == 0) ++nb; else if (pick == 1) nr += nr_step; else ng += ng_step;
     }
+    plan->dq_groups = dqg;
     plan->n_b_stages = nb;
     plan->n_groups = ng;
     plan->n_raw_stages = nr;
@@ -572,12 +610,31 @@ extern "C" int atb_tiling_supported(int T_MA, int T_MC, int T_K, int T_N) {
     return atb::plan_gemm(T_MA, T_MC, T_K, T_N, &plan) ? 1 : 0;
 }
 
+extern "C" atb_status_t atb_tiling_plan(int T_MA, int T_MC, int T_K, int T_N, atb_plan_t* out) {
+    atb::clear_error();
+    if (!out) return atb::fail(ATB_ERR_NULL_POINTER, "out must be non-NULL");
+    atb::GemmPlan plan;
+    if (T_MA <= 0 || T_MC <= 0 || T_MC % T_MA != 0 || !atb::plan_gemm(T_MA, T_MC, T_K, T_N, &plan))
+        return atb::fail(ATB_ERR_BAD_TILING, "tiling (T_MA=%d, T_MC=%d, T_K=%d, T_N=%d) is not supported", T_MA, T_MC, T_K, T_N);
+    out->n_b_stages = plan.n_b_stages;
+    out->n_raw_stages = plan.n_raw_stages;
+    out->n_a_groups = plan.n_groups;
+    out->dequant_groups = plan.dq_groups;
+    out->acc_buffers = plan.acc_bufs;
+    out->tmem_columns = plan.tmem_cols;
+    out->smem_bytes = static_cast<int>(plan.smem_bytes);
+    return ATB_OK;
+}
+
 #define ATB_DISPATCH_TN(TMA_, TMC_, TK_)                                                               \
     switch (T_N) {                                                                                     \
         case 64:  return launch<TMA_, TMC_, TK_, 64>(plan, M, N, K, A_mant_dev, A_exp_dev, B_bf16_dev, ldb, C_bf16_dev, ldc, dev->num_sms, dev->error_flag, st);  \
         case 128: return launch<TMA_, TMC_, TK_, 128>(plan, M, N, K, A_mant_dev, A_exp_dev, B_bf16_dev, ldb, C_bf16_dev, ldc, dev->num_sms, dev->error_flag, st); \
         case 256: if constexpr ((TMC_ / 128) * 256 <= 512)                                             \
                       return launch<TMA_, TMC_, TK_, 256>(plan, M, N, K, A_mant_dev, A_exp_dev, B_bf16_dev, ldb, C_bf16_dev, ldc, dev->num_sms, dev->error_flag, st); \
+                  break;                                                                               \
+        case 512: if constexpr ((TMC_ / 128) * 512 <= 512 && TK_ == 64)                                \
+                      return launch<TMA_, TMC_, TK_, 512>(plan, M, N, K, A_mant_dev, A_exp_dev, B_bf16_dev, ldb, C_bf16_dev, ldc, dev->num_sms, dev->error_flag, st); \
                   break;                                                                               \
     }                                                                                                  \
     break;

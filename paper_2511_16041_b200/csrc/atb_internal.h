@@ -21,6 +21,7 @@ struct GemmPlan {
     int n_b_stages;      // B-tile ring depth
     int n_groups;        // dequantised-A ring depth, in 128-row groups
     int n_raw_stages;    // raw (BFP16) A-slab ring depth
+    int dq_groups;       // dequantiser warp groups (ring depths are multiples of it)
     int acc_bufs;        // accumulator buffers in TMEM (1 or 2)
     int tmem_cols;       // allocated TMEM columns (power of two)
     uint32_t smem_bytes; // dynamic shared memory of the launch
