@@ -102,6 +102,26 @@ def physical_gpu_index(local_rank: int) -> int:
     return local_rank
 
 
+def rank_seed(base_seed: int, rank: int) -> int:
+    """Each rank multiplies its own rows of a taller A: a different seed per rank, same B."""
+    return base_seed + rank
+
+
+def max_over_ranks(values, device, world: int):
+    """Element-wise maximum of per-rank timings over all ranks (identity for one rank)."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t.cpu()]
+
+
+def aggregate_tflops(flops_per_rank: float, world: int, ms_per_step: float) -> float:
+    """Whole-job throughput: every rank does `flops_per_rank` per step in the slowest rank's time."""
+    return world * flops_per_rank / (ms_per_step * 1e-3) / 1e12
+
+
 def cpu_oracle_sample(name: str, target_seconds: float):
     """Times the FP64 oracle GEMM (as it stands) on a bounded row sample of workload `name`."""
     import oracle
@@ -191,7 +211,7 @@ def run_ours(args):
     name = args.workload
     c = inputs.CONFIGS[name]
     M, N, K = c["M"], c["N"], c["K"]
-    seed = inputs.BASE_SEED + rank                       # each rank owns different rows of a taller A
+    seed = rank_seed(inputs.BASE_SEED, rank)
     A_host = torch.from_numpy(inputs.make_A(c["A"], M, K, seed)).pin_memory()
     B_host = torch.from_numpy(inputs.make_B_bits(K, N, c["b_scale"]).view(np.int16)).pin_memory()
     C_host = torch.empty((M, N), dtype=torch.int16).pin_memory()
@@ -281,17 +301,13 @@ def run_ours(args):
     stream.synchronize()
     quant_ms = q0.elapsed_time(q1) / 10
 
-    # max over ranks
-    times = torch.tensor([total_ms, gemm_ms, e2e_ms, quant_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    total_ms, gemm_ms, e2e_ms, quant_ms = [float(x) for x in times.cpu()]
+    total_ms, gemm_ms, e2e_ms, quant_ms = max_over_ranks([total_ms, gemm_ms, e2e_ms, quant_ms], dev, world)
 
     if rank == 0:
         peaks, peak_src = load_peaks()
         flops = 2.0 * M * N * K
         ms_per_step = total_ms / args.steps
-        value = world * flops / (ms_per_step * 1e-3) / 1e12
+        value = aggregate_tflops(flops, world, ms_per_step)
         achieved = flops / (gemm_ms * 1e-3) / 1e12
         T_MA, T_MC, T_K, T_N = tiling_used[0]
         line = {
@@ -307,7 +323,7 @@ def run_ours(args):
                            M * K * 4 >> 20, K * N * 2 >> 20, M * N * 2 >> 20),
                        "parallelism": "replicas, one full GEMM per GPU" if world > 1 else "single GPU"},
             "clocks": clocks,
-            "e2e": {"value": world * flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOPS",
+            "e2e": {"value": aggregate_tflops(flops, world, e2e_ms), "unit": "TFLOPS",
                     "h2d_bytes_per_step": A_host.numel() * 4 + B_host.numel() * 2,
                     "d2h_bytes_per_step": C_host.numel() * 2, "ms_per_step": e2e_ms},
             "gpu_launches": 2 * args.steps,
