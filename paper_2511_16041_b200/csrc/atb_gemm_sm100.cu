@@ -8,7 +8,7 @@
 // Warp roles (704 threads):
 //   warp 0      TMA producer: B tiles and raw BFP16 A slabs (int8 mantissas + uint8 exponents)
 //   warp 1      UMMA issuer (one elected lane) and owner of the TMEM allocation
-//   warps 2-5   epilogue: tcgen05.ld -> round to bf16 -> global stores
+//   warps 2-5   epilogue: tcgen05.ld -> round to bf16 -> swizzled shared-memory box -> TMA store
 //   warps 6-21  dequantisers (two groups of 8 warps taking alternate slabs): raw slab -> bf16, K-major, 128-byte-swizzled operand in shared
 //               memory (exact: m * 2^(E-133) has at most 7 significant bits)
 // Rings, all guarded by mbarriers with bounded waits:
@@ -27,10 +27,6 @@
 
 #include "atb_internal.h"
 #include "sm100_ptx.cuh"
-
-#ifndef ATB_PACK_F2FP
-#define ATB_PACK_F2FP 0
-#endif
 
 namespace {
 
@@ -53,6 +49,7 @@ __host__ __device__ constexpr int dq_groups(int T_MA, int T_K, int T_N) {
 constexpr int kFirstEpilogueWarp = 2;
 constexpr int kFirstDequantWarp = 6;
 constexpr int kMaxStages = 16;
+constexpr uint32_t kEpilogueBoxBytes = 32 * 128;   // 32 rows x 64 bf16 columns
 constexpr uint32_t kSmemBudget = 232448;          // 227 KB of dynamic shared memory per CTA
 constexpr uint64_t kWaitTimeoutNs = 2000000000ull;  // every mbarrier wait gives up after 2 s
 
@@ -160,13 +157,7 @@ __device__ __forceinline__ uint32_t dequant_pair(uint32_t u, uint32_t sel0, uint
     asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(d), "l"(scale2));
     uint32_t f0, f1;
     asm("mov.b64 {%0, %1}, %2;" : "=r"(f0), "=r"(f1) : "l"(r));
-#if ATB_PACK_F2FP
-    uint32_t pk;
-    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(pk) : "f"(__uint_as_float(f1)), "f"(__uint_as_float(f0)));
-    return pk;
-#else
     return __byte_perm(f0, f1, 0x7632);
-#endif
 }
 
 template <class C>
@@ -220,7 +211,8 @@ __device__ __forceinline__ void dequant_slab(uint32_t raw_mant, uint32_t raw_exp
 template <int T_MA, int T_MC, int T_K, int T_N>
 __global__ void __launch_bounds__(kThreads, 1)
 atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_constant__ CUtensorMap tm_exp,
-                const __grid_constant__ CUtensorMap tm_b, const GemmParams p) {
+                const __grid_constant__ CUtensorMap tm_b, const __grid_constant__ CUtensorMap tm_c,
+                const GemmParams p) {
     using C = Cfg<T_MA, T_MC, T_K, T_N>;
     extern __shared__ uint8_t smem_raw[];
 
@@ -231,7 +223,9 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
     const uint32_t deq_base = b_base + p.n_b_stages * C::B_BYTES;
     const uint32_t raw_off = p.n_b_stages * C::B_BYTES + p.n_groups * C::GROUP_BYTES;
     const uint32_t raw_base = smem_base + raw_off;
-    const uint32_t bar_off = raw_off + p.n_raw_stages * C::RAW_BYTES;
+    // epilogue staging: one 32-row x 64-column bf16 box (4 KB, 128-byte swizzle) per epilogue warp
+    const uint32_t stage_off = (raw_off + p.n_raw_stages * C::RAW_BYTES + 1023u) & ~1023u;
+    const uint32_t bar_off = stage_off + 4u * kEpilogueBoxBytes;
     const uint32_t bar_base = smem_base + bar_off;          // 8-byte mbarriers
     const int n_deq_stages = (T_MA <= 128) ? p.n_groups * C::SPG : p.n_groups / C::GPS;
     const int n_acc = p.acc_bufs * C::G;
@@ -257,6 +251,7 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
         prefetch_tensormap(&tm_mant);
         prefetch_tensormap(&tm_exp);
         prefetch_tensormap(&tm_b);
+        prefetch_tensormap(&tm_c);
     }
     if (warp == 1) {
         tmem_alloc(misc, static_cast<uint32_t>(p.tmem_cols));
@@ -371,29 +366,40 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
                 const int acc = acc_buf * C::G + g;
                 if (!(ok = wait_bar(cx, acc_full + 8 * acc, acc_phase, 0x201))) break;
                 tcgen05_fence_after_sync();
-                const int64_t row = static_cast<int64_t>(mt) * T_MC + g * 128 + q * 32 + lane;
-                const int64_t col0 = static_cast<int64_t>(nt) * T_N;
+                const int row0 = mt * T_MC + g * 128 + q * 32;          // first of this warp's 32 rows
+                const int col0 = nt * T_N;
                 const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + static_cast<uint32_t>(acc * T_N);
+                const uint32_t box = smem_base + stage_off + static_cast<uint32_t>(warp - kFirstEpilogueWarp) * kEpilogueBoxBytes;
+                const uint32_t my_row = box + lane * 128;
+                const uint32_t sw = static_cast<uint32_t>(lane & 7);
 #pragma unroll 1
-                for (int c = 0; c < T_N / 32; ++c) {
-                    uint32_t v[32];
-                    tmem_ld_32x32b_x32(t_addr + c * 32, v);
-                    tmem_ld_wait();
-                    if (row < p.M) {
-                        __nv_bfloat16* dst = p.C + row * p.ldc + col0 + c * 32;
+                for (int c = 0; c < T_N / 64; ++c) {
+                    // the previous TMA store of this warp must have finished reading the box
+                    if (lane == 0) tma_store_wait_read<0>();
+                    __syncwarp();
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        uint32_t v[32];
+                        tmem_ld_32x32b_x32(t_addr + c * 64 + h * 32, v);
+                        tmem_ld_wait();
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {
-                            if (col0 + c * 32 + j * 8 + 8 <= p.N) {
-                                uint32_t o[4];
+                            uint32_t o[4];
 #pragma unroll
-                                for (int h = 0; h < 4; ++h) {
-                                    __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(v[j * 8 + 2 * h]),
-                                                                              __uint_as_float(v[j * 8 + 2 * h + 1]));
-                                    o[h] = *reinterpret_cast<uint32_t*>(&b2);
-                                }
-                                *reinterpret_cast<uint4*>(dst + j * 8) = make_uint4(o[0], o[1], o[2], o[3]);
+                            for (int e = 0; e < 4; ++e) {
+                                __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(v[j * 8 + 2 * e]),
+                                                                          __uint_as_float(v[j * 8 + 2 * e + 1]));
+                                o[e] = *reinterpret_cast<uint32_t*>(&b2);
                             }
+                            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(my_row + ((static_cast<uint32_t>(h * 4 + j) ^ sw) << 4)),
+                                         "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]) : "memory");
                         }
+                    }
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0 && row0 < p.M && col0 + c * 64 < p.N) {   // rows / columns past the edge are clipped
+                        tma_store_2d(&tm_c, box, col0 + c * 64, row0);
+                        tma_store_commit();
                     }
                 }
                 tcgen05_fence_before_sync();
@@ -401,6 +407,7 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
                 if (lane == 0) mbar_arrive(acc_empty + 8 * acc);
             }
         }
+        if (lane == 0) tma_store_wait_all<0>();
     } else {
         // ================================ dequantisers ================================
         const int t = (threadIdx.x - kFirstDequantWarp * 32) % C::GROUP_THREADS;
@@ -491,7 +498,7 @@ template <int T_MA, int T_MC, int T_K, int T_N>
 atb_status_t launch(const atb::GemmPlan& plan, int64_t M, int64_t N, int64_t K, const int8_t* mant,
                     const uint8_t* exp, const void* B, int64_t ldb, void* Cout, int64_t ldc,
                     int num_sms, unsigned int* error_flag, cudaStream_t stream) {
-    CUtensorMap tm_mant, tm_exp, tm_b;
+    CUtensorMap tm_mant, tm_exp, tm_b, tm_c;
     const int64_t M_pad = atb::round_up(M, 32);
     if (!make_map_2d(&tm_mant, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, mant, K, M, K, T_K, T_MA, CU_TENSOR_MAP_SWIZZLE_NONE))
         return atb::fail(ATB_ERR_CUDA, "cuTensorMapEncodeTiled failed for the mantissa plane");
@@ -500,6 +507,8 @@ atb_status_t launch(const atb::GemmPlan& plan, int64_t M, int64_t N, int64_t K, 
         return atb::fail(ATB_ERR_CUDA, "cuTensorMapEncodeTiled failed for the exponent plane");
     if (!make_map_2d(&tm_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, B, N, K, ldb * 2, 64, T_K, CU_TENSOR_MAP_SWIZZLE_128B))
         return atb::fail(ATB_ERR_CUDA, "cuTensorMapEncodeTiled failed for B");
+    if (!make_map_2d(&tm_c, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Cout, N, M, ldc * 2, 64, 32, CU_TENSOR_MAP_SWIZZLE_128B))
+        return atb::fail(ATB_ERR_CUDA, "cuTensorMapEncodeTiled failed for C");
 
     GemmParams p;
     p.M = M; p.N = N; p.K = K; p.ldc = ldc;
@@ -516,7 +525,7 @@ atb_status_t launch(const atb::GemmPlan& plan, int64_t M, int64_t N, int64_t K, 
     if (e != cudaSuccess) return atb::fail(ATB_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
     const int64_t tiles = static_cast<int64_t>(p.m_tiles) * p.n_tiles;
     const int grid = static_cast<int>(tiles < num_sms ? tiles : num_sms);
-    kernel<<<grid, kThreads, plan.smem_bytes, stream>>>(tm_mant, tm_exp, tm_b, p);
+    kernel<<<grid, kThreads, plan.smem_bytes, stream>>>(tm_mant, tm_exp, tm_b, tm_c, p);
     e = cudaGetLastError();
     if (e != cudaSuccess) return atb::fail(ATB_ERR_CUDA, "gemm launch: %s", cudaGetErrorString(e));
     return ATB_OK;
@@ -573,7 +582,7 @@ bool plan_gemm(int T_MA, int T_MC, int T_K, int T_N, GemmPlan* plan) {
     auto total = [&](int b, int g, int r) {
         const int n_deq = T_MA <= 128 ? g * spg : g / gps;
         const uint32_t bars = 8u * (2 * b + 2 * r + 2 * n_deq + 2 * 2 * G) + 16u + 1024u;
-        return 1024u + b * b_bytes + g * group_bytes + r * raw_bytes + bars;
+        return 1024u + b * b_bytes + g * group_bytes + r * raw_bytes + 1024u + 4u * kEpilogueBoxBytes + bars;
     };
     int nb = 2, ng = ng_step, nr = nr_step;
     if (ng < 2) ng = 2 * ng_step;
