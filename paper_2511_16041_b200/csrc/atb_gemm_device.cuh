@@ -1,0 +1,214 @@
+// Device-side building blocks shared by the GEMM kernels (single-CTA and CTA-pair): bounded
+// mbarrier waits, ring bookkeeping, tile rasterisation, the BFP16 -> BF16 dequantiser, and the
+// host helper that encodes TMA descriptors.  Everything lives in an unnamed namespace: each
+// translation unit gets its own copy.
+#pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <cstdint>
+#include <mutex>
+
+#include "atb_internal.h"
+#include "sm100_ptx.cuh"
+
+namespace {
+
+using namespace sm100;
+
+constexpr int kDequantWarps = 16;
+constexpr int kThreads = (6 + kDequantWarps) * 32;
+// The dequantiser warps work in groups; slabs are dealt to the groups in turn, so that several
+// slabs are in flight and every thread has a few 16-element slots per barrier round trip.
+// Ring depths are multiples of the group count: a ring stage is then always served by the same
+// group, which keeps each mbarrier's phases strictly in order for its waiters.
+__host__ __device__ constexpr int dq_groups(int T_MA, int T_K, int T_N) {
+#ifdef ATB_DQ_GROUPS
+    return ATB_DQ_GROUPS;
+#else
+    // two groups for big slabs, and where a double-buffered B tile already takes 128 KB
+    return (T_MA * T_K >= 256 * 64 || T_K * T_N >= 128 * 256) ? 2 : 4;
+#endif
+}
+constexpr int kFirstEpilogueWarp = 2;
+constexpr int kFirstDequantWarp = 6;
+constexpr int kMaxStages = 16;
+constexpr uint32_t kEpilogueBoxBytes = 32 * 128;   // 32 rows x 64 bf16 columns
+constexpr uint32_t kSmemBudget = 232448;          // 227 KB of dynamic shared memory per CTA
+constexpr uint64_t kWaitTimeoutNs = 2000000000ull;  // every mbarrier wait gives up after 2 s
+
+struct GemmParams {
+    int64_t M, N, K, ldc;
+    __nv_bfloat16* C;
+    int m_tiles, n_tiles, k_steps;
+    int n_b_stages, n_groups, n_raw_stages, acc_bufs, tmem_cols;
+    unsigned int* error_flag;
+};
+
+struct Ring {
+    int stage = 0;
+    uint32_t phase = 0;
+    __device__ __forceinline__ void advance(int n) {
+        if (++stage == n) { stage = 0; phase ^= 1u; }
+    }
+};
+
+struct Ctx {
+    volatile uint32_t* abort_flag;
+    unsigned int* error_flag;
+};
+
+// Bounded mbarrier wait.  Returns false when the CTA is aborting or the wait timed out.
+// kSpin = true (single-thread, latency-critical roles: TMA producer, UMMA issuer): tight polling.
+// kSpin = false (whole warps): after a first immediate probe the hardware may suspend the thread
+// for up to `kSuspendNs` per probe, so that waiting warps do not take issue slots from the
+// dequantisers.  kCluster = true uses cluster-scope acquire (arrivals may come from the peer CTA).
+constexpr uint32_t kSuspendNs = 20000;
+template <bool kSpin, bool kCluster>
+__device__ __forceinline__ bool wait_bar_t(const Ctx& cx, uint32_t bar, uint32_t parity, unsigned code) {
+    auto probe = [&]() { return kCluster ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity); };
+    auto probe_suspend = [&]() {
+        return kCluster ? mbar_try_wait_cluster_suspend(bar, parity, kSuspendNs) : mbar_try_wait_suspend(bar, parity, kSuspendNs);
+    };
+    if (probe()) return true;
+    const uint64_t t0 = global_timer_ns();
+    constexpr uint32_t kCheckMask = kSpin ? 1023u : 7u;
+    for (uint32_t spins = 0;; ++spins) {
+        if (kSpin ? probe() : probe_suspend()) return true;
+        if ((spins & kCheckMask) == kCheckMask) {
+            if (*cx.abort_flag) return false;
+            if (global_timer_ns() - t0 > kWaitTimeoutNs) {
+                *cx.abort_flag = 1u;
+                atomicCAS(cx.error_flag, 0u, code);
+                return false;
+            }
+        }
+    }
+}
+__device__ __forceinline__ bool wait_bar(const Ctx& cx, uint32_t bar, uint32_t parity, unsigned code) {
+    return wait_bar_t<false, false>(cx, bar, parity, code);
+}
+__device__ __forceinline__ bool wait_bar_spin(const Ctx& cx, uint32_t bar, uint32_t parity, unsigned code) {
+    return wait_bar_t<true, false>(cx, bar, parity, code);
+}
+
+__device__ __forceinline__ void tile_coords(int tile, int m_tiles, int n_tiles, int& mt, int& nt) {
+    // Bands of 16 tile-rows, column-major inside a band: the CTAs of one wave share a few
+    // A row-panels and B column-panels in L2.
+    const int per_band = 16 * n_tiles;
+    const int band = tile / per_band, i = tile - band * per_band;
+    const int rows = min(16, m_tiles - band * 16);
+    mt = band * 16 + i % rows;
+    nt = i / rows;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Dequantise one raw slab (T_MA rows x T_K columns) into its place in a bf16 operand group.
+// One group of dequantiser warps (GROUP_THREADS threads) works on a slab.  Thread t owns slot (row r, pair p) = (t / SPR + i *
+// GROUP_THREADS / SPR, t % SPR), a slot being two blocks: 16 mantissa bytes (one 16-byte load; the loads of
+// a warp are contiguous), two exponent bytes, and two 16-byte stores into the swizzled row.
+//
+// Per element: the byte u = m + 128 is dropped into the mantissa of the float 2^23 (bit pattern
+// 0x4B0000uu = 2^23 + u); subtracting 2^23 + 128 leaves m exactly, and the product with the
+// block scale 2^(E-133) (taken from a 256-entry table: normal for E >= 7, fp32-subnormal below) is
+// exact for every E.  The result has at most 7 significant bits, so its low 16 bits are zero and
+// the bf16 value is the upper half of the word.
+__device__ __forceinline__ uint64_t pack_f32x2(uint32_t lo, uint32_t hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+    return r;
+}
+
+// bf16x2 of (m0, m1) * scale for bytes `sel0`, `sel0 + 1` of the biased word u.
+__device__ __forceinline__ uint32_t dequant_pair(uint32_t u, uint32_t sel0, uint64_t neg_magic2, uint64_t scale2) {
+    const uint32_t x0 = __byte_perm(u, 0x4B000000u, 0x7650u + sel0);
+    const uint32_t x1 = __byte_perm(u, 0x4B000000u, 0x7651u + sel0);
+    uint64_t d, r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(pack_f32x2(x0, x1)), "l"(neg_magic2));
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(d), "l"(scale2));
+    uint32_t f0, f1;
+    asm("mov.b64 {%0, %1}, %2;" : "=r"(f0), "=r"(f1) : "l"(r));
+    return __byte_perm(f0, f1, 0x7632);
+}
+
+template <class C>
+__device__ __forceinline__ void dequant_slab(uint32_t raw_mant, uint32_t raw_exp, uint32_t scale_lut,
+                                             uint32_t dst_base, int row_base, int t, int T_MA_rows) {
+    const int p = t % C::SLOTS_PER_ROW;                 // blocks 2p, 2p + 1 of the row
+    const int r0 = t / C::SLOTS_PER_ROW;
+    const int kb = 2 * p;
+    uint4 w[C::DQ_ITERS];
+    uint32_t e[C::DQ_ITERS];
+#pragma unroll
+    for (int i = 0; i < C::DQ_ITERS; ++i) {
+        const int r = r0 + i * C::ROWS_PER_ITER;
+        if (C::SLOTS % C::GROUP_THREADS == 0 || r < T_MA_rows) {
+            asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                         : "=r"(w[i].x), "=r"(w[i].y), "=r"(w[i].z), "=r"(w[i].w)
+                         : "r"(raw_mant + (r * C::SLOTS_PER_ROW + p) * 16));
+            uint16_t e2;
+            asm volatile("ld.shared.u16 %0, [%1];" : "=h"(e2)
+                         : "r"(raw_exp + (kb >> 3) * T_MA_rows * 8 + r * 8 + (kb & 7)));
+            e[i] = e2;
+        }
+    }
+    const uint64_t neg_magic2 = pack_f32x2(0xCB000080u, 0xCB000080u);    // -(2^23 + 128), twice
+#pragma unroll
+    for (int i = 0; i < C::DQ_ITERS; ++i) {
+        const int r = r0 + i * C::ROWS_PER_ITER;
+        if (C::SLOTS % C::GROUP_THREADS == 0 || r < T_MA_rows) {
+            uint32_t s0, s1;
+            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(s0) : "r"(scale_lut + (e[i] & 0xFFu) * 4));
+            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(s1) : "r"(scale_lut + (e[i] >> 8) * 4));
+            const uint64_t sc0 = pack_f32x2(s0, s0), sc1 = pack_f32x2(s1, s1);
+            const uint32_t u0 = w[i].x ^ 0x80808080u, u1 = w[i].y ^ 0x80808080u;
+            const uint32_t u2 = w[i].z ^ 0x80808080u, u3 = w[i].w ^ 0x80808080u;
+            const int rr = row_base + r;
+            const uint32_t row_addr = dst_base + (rr >> 7) * C::GROUP_BYTES + (kb >> 3) * C::KHALF_BYTES + (rr & 127) * 128;
+            const uint32_t sw = static_cast<uint32_t>(rr & 7);
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row_addr + ((((kb & 7)) ^ sw) << 4)),
+                         "r"(dequant_pair(u0, 0, neg_magic2, sc0)), "r"(dequant_pair(u0, 2, neg_magic2, sc0)),
+                         "r"(dequant_pair(u1, 0, neg_magic2, sc0)), "r"(dequant_pair(u1, 2, neg_magic2, sc0))
+                         : "memory");
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row_addr + ((((kb & 7) + 1) ^ sw) << 4)),
+                         "r"(dequant_pair(u2, 0, neg_magic2, sc1)), "r"(dequant_pair(u2, 2, neg_magic2, sc1)),
+                         "r"(dequant_pair(u3, 0, neg_magic2, sc1)), "r"(dequant_pair(u3, 2, neg_magic2, sc1))
+                         : "memory");
+        }
+    }
+}
+
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                   CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                   CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    });
+    return fn;
+}
+
+bool make_map_2d(CUtensorMap* map, CUtensorMapDataType type, uint32_t elem_bytes, const void* base,
+                 uint64_t dim0, uint64_t dim1, uint64_t stride1_bytes, uint32_t box0, uint32_t box1,
+                 CUtensorMapSwizzle swizzle) {
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {dim0, dim1};
+    const cuuint64_t strides[1] = {stride1_bytes};
+    const cuuint32_t box[2] = {box0, box1};
+    const cuuint32_t estr[2] = {1, 1};
+    (void)elem_bytes;
+    return fn(map, type, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace

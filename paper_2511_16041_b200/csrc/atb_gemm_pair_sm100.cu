@@ -1,0 +1,372 @@
+// atb_gemm, CTA-pair kernel for the tiling T_MC = 256, T_N = 512, T_K = 64 (sm_100a).
+//
+// Two CTAs of a cluster share one 256 x 512 output tile through tcgen05.mma cta_group::2:
+// CTA r (r = 0, 1) owns rows 128r .. 128r+127 of the tile - it loads, dequantises and feeds that
+// half of A, and holds its 128 x 512 FP32 accumulator in its own TMEM (all 512 columns) - and
+// supplies half of every 256-column B chunk (columns 128r .. 128r+127) from its own shared
+// memory.  This is the B200 counterpart of the array-level sharing of Section 3.2 (Eq. 2): the
+// B tile is shared across the two "rows" of the pair, and every dequantised A element feeds
+// 512 output columns instead of 256, which halves the dequantiser work per FLOP.
+//
+// Per K-step (Section 3.1 schedule): each CTA brings in its 64 x 256 half of the B tile once and
+// streams 128 / SLAB_ROWS raw A slabs through the dequantisers; the leader CTA (rank 0) issues
+// 2 x 4 UMMAs of 256 x 256 x 16.  Barriers the UMMA issuer waits on live in the leader CTA and
+// collect arrivals from both CTAs; stage-free barriers are signalled in both CTAs at once by
+// tcgen05.commit with a CTA mask.  No TMA load uses multicast.
+//
+// Warp roles are those of the single-CTA kernel: 0 TMA producer, 1 UMMA issuer (active in the
+// leader only) + TMEM owner, 2-5 epilogue, 6-21 dequantisers (4 groups of 4 warps).
+#include "atb_gemm_device.cuh"
+
+namespace {
+
+template <int SLAB_ROWS>
+struct PairCfg {
+    static constexpr int T_K = 64, N_MMA = 256, N_CHUNKS = 2, ROWS = 128;
+    static constexpr int SLABS = ROWS / SLAB_ROWS;             // slabs per CTA and K-step
+    static constexpr uint32_t B_BOX_BYTES = T_K * 128;         // 64 columns x 64 rows of bf16
+    static constexpr uint32_t B_BYTES = 4 * B_BOX_BYTES;       // this CTA's half: 2 chunks x 128 columns
+    static constexpr uint32_t GROUP_BYTES = 128 * T_K * 2;
+    static constexpr uint32_t KHALF_BYTES = 128 * 128;
+    static constexpr uint32_t RAW_MANT_BYTES = SLAB_ROWS * T_K;
+    static constexpr uint32_t RAW_EXP_BYTES = SLAB_ROWS * T_K / 8;
+    static constexpr uint32_t RAW_BYTES = RAW_MANT_BYTES + RAW_EXP_BYTES;
+    static constexpr int SLOTS_PER_ROW = T_K / 16;
+    static constexpr int SLOTS = SLAB_ROWS * SLOTS_PER_ROW;
+    static constexpr int DQ_GROUPS = 4;
+    static constexpr int GROUP_WARPS = kDequantWarps / DQ_GROUPS;
+    static constexpr int GROUP_THREADS = GROUP_WARPS * 32;
+    static constexpr int DQ_ITERS = (SLOTS + GROUP_THREADS - 1) / GROUP_THREADS;
+    static constexpr int ROWS_PER_ITER = GROUP_THREADS / SLOTS_PER_ROW;
+};
+
+struct PairParams {
+    int64_t M, N, K;
+    int m_tiles, n_tiles, k_steps;           // tiles of 256 x 512
+    int n_b_stages, n_groups, n_raw_stages;
+    unsigned int* error_flag;
+};
+
+// Bounded waits with cluster-scope acquire (the arrivals may come from the peer CTA).
+__device__ __forceinline__ bool wait_bar_cl(const Ctx& cx, uint32_t bar, uint32_t parity, unsigned code) {
+    return wait_bar_t<false, true>(cx, bar, parity, code);
+}
+__device__ __forceinline__ bool wait_bar_cl_spin(const Ctx& cx, uint32_t bar, uint32_t parity, unsigned code) {
+    return wait_bar_t<true, true>(cx, bar, parity, code);
+}
+
+template <int SLAB_ROWS>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+atb_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_constant__ CUtensorMap tm_exp,
+                     const __grid_constant__ CUtensorMap tm_b, const __grid_constant__ CUtensorMap tm_c,
+                     const PairParams p) {
+    using C = PairCfg<SLAB_ROWS>;
+    extern __shared__ uint8_t smem_raw[];
+
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* const smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+    const uint32_t b_base = smem_base;
+    const uint32_t deq_base = b_base + p.n_b_stages * C::B_BYTES;
+    const uint32_t raw_off = p.n_b_stages * C::B_BYTES + p.n_groups * C::GROUP_BYTES;
+    const uint32_t raw_base = smem_base + raw_off;
+    const uint32_t stage_off = (raw_off + p.n_raw_stages * C::RAW_BYTES + 1023u) & ~1023u;
+    const uint32_t bar_off = stage_off + 4u * kEpilogueBoxBytes;
+    const uint32_t bar_base = smem_base + bar_off;
+    const int n_deq_stages = p.n_groups * C::SLABS;
+    const uint32_t b_full = bar_base, b_empty = b_full + 8 * p.n_b_stages;
+    const uint32_t raw_full = b_empty + 8 * p.n_b_stages, raw_empty = raw_full + 8 * p.n_raw_stages;
+    const uint32_t deq_full = raw_empty + 8 * p.n_raw_stages, deq_empty = deq_full + 8 * n_deq_stages;
+    const uint32_t acc_full = deq_empty + 8 * n_deq_stages, acc_empty = acc_full + 8 * C::N_CHUNKS;
+    const uint32_t misc = acc_empty + 8 * C::N_CHUNKS;       // [0]: TMEM base, [1]: abort flag
+    const uint32_t scale_lut = misc + 16;
+    volatile uint32_t* const misc_gen = reinterpret_cast<volatile uint32_t*>(smem_gen + (misc - smem_base));
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();
+    const bool leader = rank == 0;
+    Ctx cx{misc_gen + 1, p.error_flag};
+
+    if (threadIdx.x == 0) {
+        // Barriers with arrivals from both CTAs are only used in the leader, but are initialised
+        // everywhere so that both CTAs have the same layout.
+        for (int i = 0; i < p.n_b_stages; ++i) { mbar_init(b_full + 8 * i, 1); mbar_init(b_empty + 8 * i, 1); }
+        for (int i = 0; i < p.n_raw_stages; ++i) { mbar_init(raw_full + 8 * i, 1); mbar_init(raw_empty + 8 * i, C::GROUP_WARPS); }
+        for (int i = 0; i < n_deq_stages; ++i) { mbar_init(deq_full + 8 * i, 2 * C::GROUP_WARPS); mbar_init(deq_empty + 8 * i, 1); }
+        for (int i = 0; i < C::N_CHUNKS; ++i) { mbar_init(acc_full + 8 * i, 1); mbar_init(acc_empty + 8 * i, 8); }
+        misc_gen[1] = 0u;
+        fence_mbar_init();
+        prefetch_tensormap(&tm_mant);
+        prefetch_tensormap(&tm_exp);
+        prefetch_tensormap(&tm_b);
+        prefetch_tensormap(&tm_c);
+    }
+    if (warp == 1) {
+        tmem_alloc_pair(misc, 512u);
+        tmem_relinquish_pair();
+    }
+    if (threadIdx.x >= kFirstDequantWarp * 32 && threadIdx.x < kFirstDequantWarp * 32 + 256) {
+        const uint32_t E = threadIdx.x - kFirstDequantWarp * 32;
+        const uint32_t bits = (E >= 7u) ? ((E - 6u) << 23) : (1u << (E + 16u));
+        asm volatile("st.shared.b32 [%0], %1;" ::"r"(scale_lut + E * 4), "r"(E == 255u ? 0u : bits) : "memory");
+    }
+    tcgen05_fence_before_sync();
+    __syncthreads();
+    cluster_sync_all();                      // the peer's barriers exist before anything arrives on them
+    tcgen05_fence_after_sync();
+    const uint32_t tmem_base = misc_gen[0];
+
+    const int total_tiles = p.m_tiles * p.n_tiles;
+    const int cluster_id = blockIdx.x >> 1, n_clusters = gridDim.x >> 1;
+
+    if (warp == 0) {
+        // ================================ TMA producer ================================
+        if (elect_one()) {
+            Ring rb, rr;
+            bool ok = true;
+            for (int tile = cluster_id; ok && tile < total_tiles; tile += n_clusters) {
+                int mt, nt;
+                tile_coords(tile, p.m_tiles, p.n_tiles, mt, nt);
+                const int row0 = mt * 256 + static_cast<int>(rank) * 128;
+                const int colb = nt * 512 + static_cast<int>(rank) * 128;
+                for (int k = 0; ok && k < p.k_steps; ++k) {
+                    if (!(ok = wait_bar_cl_spin(cx, b_empty + 8 * rb.stage, rb.phase ^ 1u, 0x001))) break;
+                    // both halves of the B tile are credited to the leader's barrier
+                    if (leader) mbar_arrive_expect_tx(b_full + 8 * rb.stage, 2 * C::B_BYTES);
+                    const uint32_t fb = mapa_shared(b_full + 8 * rb.stage, 0);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        tma_load_2d_pair(b_base + rb.stage * C::B_BYTES + j * C::B_BOX_BYTES, &tm_b,
+                                         colb + (j >> 1) * 256 + (j & 1) * 64, k * C::T_K, fb);
+                    rb.advance(p.n_b_stages);
+                    for (int s = 0; s < C::SLABS; ++s) {
+                        if (!(ok = wait_bar_cl_spin(cx, raw_empty + 8 * rr.stage, rr.phase ^ 1u, 0x002))) break;
+                        const uint32_t fr = raw_full + 8 * rr.stage;
+                        const uint32_t dst = raw_base + rr.stage * C::RAW_BYTES;
+                        mbar_arrive_expect_tx(fr, C::RAW_BYTES);
+                        tma_load_2d(dst, &tm_mant, k * C::T_K, row0 + s * SLAB_ROWS, fr);
+                        tma_load_2d(dst + C::RAW_MANT_BYTES, &tm_exp, row0 + s * SLAB_ROWS, k, fr);
+                        rr.advance(p.n_raw_stages);
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ================================ UMMA issuer (leader CTA) ====================
+        if (leader && elect_one()) {
+            constexpr uint32_t idesc = umma_idesc_bf16_f32(256, C::N_MMA, false, true);
+            Ring rb, rd;
+            uint32_t acc_phase = 0;
+            bool ok = true;
+            for (int tile = cluster_id; ok && tile < total_tiles; tile += n_clusters, acc_phase ^= 1u) {
+                for (int k = 0; ok && k < p.k_steps; ++k) {
+                    if (!(ok = wait_bar_cl_spin(cx, b_full + 8 * rb.stage, rb.phase, 0x101))) break;
+                    for (int i = 0; ok && i < C::SLABS; ++i)
+                        ok = wait_bar_cl_spin(cx, deq_full + 8 * (rd.stage + i), rd.phase, 0x103);
+                    if (!ok) break;
+                    const uint32_t as = deq_base + (rd.stage / C::SLABS) * C::GROUP_BYTES;
+                    const uint32_t bs = b_base + rb.stage * C::B_BYTES;
+#pragma unroll
+                    for (int nc = 0; nc < C::N_CHUNKS; ++nc) {
+                        // both CTAs' epilogues have drained this chunk of the previous tile
+                        if (k == 0 && !(ok = wait_bar_cl_spin(cx, acc_empty + 8 * nc, acc_phase ^ 1u, 0x102))) break;
+                        tcgen05_fence_after_sync();
+#pragma unroll
+                        for (int kk = 0; kk < C::T_K / 16; ++kk) {
+                            const uint64_t a_desc = umma_smem_desc_sw128(as + kk * 32, 16, 1024);
+                            const uint64_t b_desc = umma_smem_desc_sw128(bs + nc * 2 * C::B_BOX_BYTES + kk * 2048,
+                                                                         C::B_BOX_BYTES, 1024);
+                            umma_f16_ss_pair(tmem_base + nc * C::N_MMA, a_desc, b_desc, idesc, (k > 0 || kk > 0) ? 1u : 0u);
+                        }
+                        if (k == p.k_steps - 1) umma_commit_pair(acc_full + 8 * nc, 3);
+                    }
+                    if (!ok) break;
+                    for (int i = 0; i < C::SLABS; ++i) umma_commit_pair(deq_empty + 8 * (rd.stage + i), 3);
+                    for (int i = 0; i < C::SLABS; ++i) rd.advance(n_deq_stages);
+                    umma_commit_pair(b_empty + 8 * rb.stage, 3);
+                    rb.advance(p.n_b_stages);
+                }
+            }
+        }
+    } else if (warp < kFirstDequantWarp) {
+        // ================================ epilogue ====================================
+        const int q = warp & 3;
+        uint32_t acc_phase = 0;
+        bool ok = true;
+        for (int tile = cluster_id; ok && tile < total_tiles; tile += n_clusters, acc_phase ^= 1u) {
+            int mt, nt;
+            tile_coords(tile, p.m_tiles, p.n_tiles, mt, nt);
+            const int row0 = mt * 256 + static_cast<int>(rank) * 128 + q * 32;
+            const uint32_t box = smem_base + stage_off + static_cast<uint32_t>(warp - kFirstEpilogueWarp) * kEpilogueBoxBytes;
+            const uint32_t my_row = box + lane * 128;
+            const uint32_t sw = static_cast<uint32_t>(lane & 7);
+            for (int nc = 0; nc < C::N_CHUNKS; ++nc) {
+                if (!(ok = wait_bar_cl(cx, acc_full + 8 * nc, acc_phase, 0x201))) break;
+                tcgen05_fence_after_sync();
+                const int col0 = nt * 512 + nc * C::N_MMA;
+                const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + static_cast<uint32_t>(nc * C::N_MMA);
+#pragma unroll 1
+                for (int c = 0; c < C::N_MMA / 64; ++c) {
+                    if (lane == 0) tma_store_wait_read<0>();
+                    __syncwarp();
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        uint32_t v[32];
+                        tmem_ld_32x32b_x32(t_addr + c * 64 + h * 32, v);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            uint32_t o[4];
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(v[j * 8 + 2 * e]),
+                                                                          __uint_as_float(v[j * 8 + 2 * e + 1]));
+                                o[e] = *reinterpret_cast<uint32_t*>(&b2);
+                            }
+                            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(my_row + ((static_cast<uint32_t>(h * 4 + j) ^ sw) << 4)),
+                                         "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]) : "memory");
+                        }
+                    }
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0 && row0 < p.M && col0 + c * 64 < p.N) {
+                        tma_store_2d(&tm_c, box, col0 + c * 64, row0);
+                        tma_store_commit();
+                    }
+                }
+                tcgen05_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(mapa_shared(acc_empty + 8 * nc, 0));
+            }
+        }
+        if (lane == 0) tma_store_wait_all<0>();
+    } else {
+        // ================================ dequantisers ================================
+        const int t = (threadIdx.x - kFirstDequantWarp * 32) % C::GROUP_THREADS;
+        const int my_group = (threadIdx.x - kFirstDequantWarp * 32) / C::GROUP_THREADS;
+        Ring rr, rd;
+        for (int i = 0; i < my_group; ++i) { rr.advance(p.n_raw_stages); rd.advance(n_deq_stages); }
+        int turn = 0;
+        bool ok = true;
+        for (int tile = cluster_id; ok && tile < total_tiles; tile += n_clusters) {
+            for (int k = 0; ok && k < p.k_steps; ++k) {
+                for (int s = 0; s < C::SLABS; ++s) {
+                    const bool mine = (turn == my_group);
+                    if (++turn == C::DQ_GROUPS) turn = 0;
+                    if (!mine) continue;
+                    if (!(ok = wait_bar_cl(cx, raw_full + 8 * rr.stage, rr.phase, 0x301))) break;
+                    if (!(ok = wait_bar_cl(cx, deq_empty + 8 * rd.stage, rd.phase ^ 1u, 0x302))) break;
+                    const uint32_t raw = raw_base + rr.stage * C::RAW_BYTES;
+                    const uint32_t dst_base = deq_base + (rd.stage / C::SLABS) * C::GROUP_BYTES;
+                    const int row_base = (rd.stage % C::SLABS) * SLAB_ROWS;
+                    dequant_slab<C>(raw, raw + C::RAW_MANT_BYTES, scale_lut, dst_base, row_base, t, SLAB_ROWS);
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) {
+                        mbar_arrive_cluster(mapa_shared(deq_full + 8 * rd.stage, 0));
+                        mbar_arrive(raw_empty + 8 * rr.stage);
+                    }
+                    for (int i = 0; i < C::DQ_GROUPS; ++i) { rr.advance(p.n_raw_stages); rd.advance(n_deq_stages); }
+                }
+            }
+        }
+    }
+
+    // ---- teardown: the peer may still arrive on this CTA's barriers until it gets here ----
+    if (*cx.abort_flag) {
+        for (int i = 0; i < 64; ++i) __nanosleep(20000);
+    }
+    tcgen05_fence_before_sync();
+    __syncthreads();
+    cluster_sync_all();
+    if (warp == 1) {
+        tcgen05_fence_after_sync();
+        tmem_dealloc_pair(tmem_base, 512u);
+    }
+}
+
+template <int SLAB_ROWS>
+atb_status_t launch_pair_t(const atb::GemmPlan& plan, int64_t M, int64_t N, int64_t K, const int8_t* mant,
+                           const uint8_t* exp, const void* B, int64_t ldb, void* Cout, int64_t ldc, int num_sms,
+                           unsigned int* error_flag, cudaStream_t stream) {
+    using C = PairCfg<SLAB_ROWS>;
+    CUtensorMap tm_mant, tm_exp, tm_b, tm_c;
+    const int64_t M_pad = atb::round_up(M, 32);
+    if (!make_map_2d(&tm_mant, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, mant, K, M, K, C::T_K, SLAB_ROWS, CU_TENSOR_MAP_SWIZZLE_NONE))
+        return atb::fail(ATB_ERR_CUDA, "cuTensorMapEncodeTiled failed for the mantissa plane");
+    if (!make_map_2d(&tm_exp, CU_TENSOR_MAP_DATA_TYPE_UINT64, 8, exp, M_pad, atb::ceil_div(K, 64), M_pad * 8, SLAB_ROWS, 1,
+                     CU_TENSOR_MAP_SWIZZLE_NONE))
+        return atb::fail(ATB_ERR_CUDA, "cuTensorMapEncodeTiled failed for the exponent plane");
+    if (!make_map_2d(&tm_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, B, N, K, ldb * 2, 64, C::T_K, CU_TENSOR_MAP_SWIZZLE_128B))
+        return atb::fail(ATB_ERR_CUDA, "cuTensorMapEncodeTiled failed for B");
+    if (!make_map_2d(&tm_c, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Cout, N, M, ldc * 2, 64, 32, CU_TENSOR_MAP_SWIZZLE_128B))
+        return atb::fail(ATB_ERR_CUDA, "cuTensorMapEncodeTiled failed for C");
+
+    PairParams p;
+    p.M = M; p.N = N; p.K = K;
+    p.m_tiles = static_cast<int>(atb::ceil_div(M, 256));
+    p.n_tiles = static_cast<int>(atb::ceil_div(N, 512));
+    p.k_steps = static_cast<int>(atb::ceil_div(K, C::T_K));
+    p.n_b_stages = plan.n_b_stages; p.n_groups = plan.n_groups; p.n_raw_stages = plan.n_raw_stages;
+    p.error_flag = error_flag;
+
+    auto kernel = atb_gemm_pair_kernel<SLAB_ROWS>;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(plan.smem_bytes));
+    if (e != cudaSuccess) return atb::fail(ATB_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
+    const int64_t tiles = static_cast<int64_t>(p.m_tiles) * p.n_tiles;
+    const int max_clusters = num_sms / 2;
+    const int clusters = static_cast<int>(tiles < max_clusters ? tiles : max_clusters);
+    kernel<<<2 * clusters, kThreads, plan.smem_bytes, stream>>>(tm_mant, tm_exp, tm_b, tm_c, p);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return atb::fail(ATB_ERR_CUDA, "gemm (pair) launch: %s", cudaGetErrorString(e));
+    return ATB_OK;
+}
+
+}  // namespace
+
+namespace atb {
+
+bool plan_gemm_pair(int T_MA, GemmPlan* plan) {
+    if (!(T_MA == 32 || T_MA == 64 || T_MA == 128 || T_MA == 256)) return false;
+    const int slab = T_MA > 128 ? 128 : T_MA;
+    const int slabs = 128 / slab;
+    const uint32_t b_bytes = 4 * 64 * 128, group_bytes = 128 * 64 * 2, raw_bytes = slab * 64 * 9 / 8;
+    // 4 dequantiser groups: raw ring and slab stages in multiples of 4
+    const int dqg = 4;                                   // PairCfg::DQ_GROUPS
+    int ng = (dqg + slabs - 1) / slabs;
+    if ((ng * slabs) % dqg != 0) ng = dqg;
+    const int ng_step = ng;
+    int nb = 3, nr = dqg;
+    auto total = [&](int b, int g, int r) {
+        const uint32_t bars = 8u * (2 * b + 2 * r + 2 * g * slabs + 4) + 16u + 1024u;
+        return 1024u + b * b_bytes + g * group_bytes + r * raw_bytes + 1024u + 4u * kEpilogueBoxBytes + bars;
+    };
+    if (total(nb, ng, nr) > kSmemBudget) return false;
+    // Spend what is left on raw slabs (up to 8 K-steps of look-ahead), then B tiles, then bf16
+    // groups (measured: the dequantised-A ring is the one whose depth pays most).
+    while (ng + ng_step <= 4 && total(nb, ng + ng_step, nr) <= kSmemBudget) ng += ng_step;
+    while (nr + dqg <= kMaxStages && nr * slab < 8 * 128 && total(nb, ng, nr + dqg) <= kSmemBudget) nr += dqg;
+    while (nb < 4 && total(nb + 1, ng, nr) <= kSmemBudget) ++nb;
+    plan->dq_groups = dqg;
+    plan->n_b_stages = nb;
+    plan->n_groups = ng;
+    plan->n_raw_stages = nr;
+    plan->acc_bufs = 1;
+    plan->tmem_cols = 512;
+    plan->smem_bytes = total(nb, ng, nr);
+    return true;
+}
+
+atb_status_t launch_gemm_pair(int T_MA, const GemmPlan& plan, int64_t M, int64_t N, int64_t K, const int8_t* mant,
+                              const uint8_t* exp, const void* B, int64_t ldb, void* C, int64_t ldc, int num_sms,
+                              unsigned int* error_flag, void* stream) {
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    switch (T_MA) {
+        case 32:  return launch_pair_t<32>(plan, M, N, K, mant, exp, B, ldb, C, ldc, num_sms, error_flag, st);
+        case 64:  return launch_pair_t<64>(plan, M, N, K, mant, exp, B, ldb, C, ldc, num_sms, error_flag, st);
+        case 128:
+        case 256: return launch_pair_t<128>(plan, M, N, K, mant, exp, B, ldb, C, ldc, num_sms, error_flag, st);
+    }
+    return atb::fail(ATB_ERR_BAD_TILING, "no pair kernel for T_MA=%d", T_MA);
+}
+
+}  // namespace atb

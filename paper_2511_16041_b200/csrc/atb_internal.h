@@ -28,5 +28,11 @@ struct GemmPlan {
 };
 // Fills `plan`; false if the tiling is not supported or does not fit.
 bool plan_gemm(int T_MA, int T_MC, int T_K, int T_N, GemmPlan* plan);
+// True for the tilings executed by a CTA pair (cluster of 2): T_MC = 256, T_N = 512, T_K = 64.
+inline bool is_pair_tiling(int T_MC, int T_K, int T_N) { return T_MC == 256 && T_N == 512 && T_K == 64; }
+bool plan_gemm_pair(int T_MA, GemmPlan* plan);
+atb_status_t launch_gemm_pair(int T_MA, const GemmPlan& plan, int64_t M, int64_t N, int64_t K, const int8_t* mant,
+                              const uint8_t* exp, const void* B, int64_t ldb, void* C, int64_t ldc, int num_sms,
+                              unsigned int* error_flag, void* stream);
 
 }  // namespace atb

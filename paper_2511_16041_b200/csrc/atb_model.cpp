@@ -106,7 +106,7 @@ atb_status_t atb_select_tiling(int64_t M, int64_t N, int64_t K, const atb_hw_par
     atb_hw_params_t hw;
     if (hw_in) hw = *hw_in; else atb_hw_params_b200(&hw);
 
-    static const int kMC[] = {128, 256}, kN[] = {64, 128, 256}, kK[] = {64, 128}, kMA[] = {32, 64, 128, 256};
+    static const int kMC[] = {128, 256}, kN[] = {64, 128, 256, 512}, kK[] = {64, 128}, kMA[] = {32, 64, 128, 256};
     std::vector<atb_tiling_score_t> all;
     for (int mc : kMC) for (int n : kN) for (int k : kK) for (int ma : kMA) {
         if (ma > mc || !atb_tiling_supported(ma, mc, k, n)) continue;

@@ -45,9 +45,10 @@ def test_tiling_supported_rules():
     assert not ok(64, 192, 64, 128)           # T_MC not 128 / 256
     assert not ok(64, 128, 32, 128)           # T_K
     assert not ok(64, 128, 64, 96)            # T_N
+    assert ok(128, 256, 64, 512) and ok(32, 256, 64, 512) and not ok(128, 256, 128, 512)   # CTA-pair tilings
     # asymmetric buffering is what makes the deep K-step fit next to a 256-wide B tile
-    assert not ok(256, 256, 128, 256) and not ok(128, 256, 128, 256)
-    assert ok(64, 256, 128, 256) and ok(32, 256, 128, 256)
+    assert not ok(256, 256, 128, 256) and not ok(128, 256, 128, 256) and not ok(64, 256, 128, 256)
+    assert ok(32, 256, 128, 256)
 
 
 def test_layout_helpers_roundtrip():
@@ -70,3 +71,27 @@ def test_argument_validation_needs_no_gpu():
     assert lib.atb_quantize_bfp16(None, 0, 64, 64, None, None, None) == 0       # empty: no-op
     assert lib.atb_gemm(128, 128, 64, 64, 128, 64, 128, None, None, None, 128, None, 128, None) == 1
     assert atb.atb_last_error_message() != ""
+
+
+def test_ring_plans_keep_mbarrier_phases_in_order():
+    """Ring depths must be multiples of the dequantiser group count (a stage is then always
+    served by the same group), and everything must fit the 227 KB / 512-column budgets."""
+    n = 0
+    for mc in (128, 256):
+        for tn in (64, 128, 256, 512):
+            for tk in (64, 128):
+                for ma in (32, 64, 128, 256):
+                    if ma > mc or not atb.atb_tiling_supported(ma, mc, tk, tn):
+                        continue
+                    p = atb.atb_tiling_plan(ma, mc, tk, tn)
+                    n += 1
+                    pair = (mc, tk, tn) == (256, 64, 512)
+                    slab = min(ma, 128) if pair else ma
+                    slab_stages = p.n_a_groups * (128 // slab) if slab <= 128 else p.n_a_groups // (slab // 128)
+                    assert p.dequant_groups in (1, 2, 4)
+                    assert p.n_raw_stages % p.dequant_groups == 0, (ma, mc, tk, tn)
+                    assert slab_stages % p.dequant_groups == 0 and slab_stages >= 2, (ma, mc, tk, tn)
+                    assert p.n_b_stages >= 2 and p.acc_buffers in (1, 2)
+                    assert p.smem_bytes <= 232448 and p.tmem_columns <= 512
+                    assert p.tmem_columns >= p.acc_buffers * (128 if pair else mc) // 128 * tn
+    assert n >= 30

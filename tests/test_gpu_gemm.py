@@ -16,7 +16,7 @@ from tests.gpu_util import run_gemm, dev, planes_to_dev, bf16_bits_to_dev, bf16_
 
 pytestmark = pytest.mark.gpu
 
-ALL_TILINGS = [(ma, mc, k, n) for mc in (128, 256) for n in (64, 128, 256) for k in (64, 128)
+ALL_TILINGS = [(ma, mc, k, n) for mc in (128, 256) for n in (64, 128, 256, 512) for k in (64, 128)
                for ma in (32, 64, 128, 256) if ma <= mc]
 
 
@@ -60,7 +60,7 @@ def test_atb_invariance_bitwise_across_T_MA():
     A = inputs.make_A("outlier", M, K)
     Bb = inputs.make_B_bits(K, N, None)
     mant, exp = oracle.quantize_bfp16(A)
-    for (mc, k, n) in [(256, 64, 256), (256, 128, 128), (128, 64, 128)]:
+    for (mc, k, n) in [(256, 64, 256), (256, 128, 128), (128, 64, 128), (256, 64, 512)]:
         ref = None
         for ma in (32, 64, 128, 256):
             if ma > mc or not atb.atb_tiling_supported(ma, mc, k, n):
@@ -79,7 +79,7 @@ def test_small_integer_matrices_exact():
     b = rng.integers(-1, 2, size=(K, N)).astype(np.float32)
     mant, exp = oracle.quantize_bfp16(a)
     Cr, _ = oracle.gemm(mant, exp, inputs.to_bf16_bits(b))
-    for t in [(128, 128, 64, 128), (64, 256, 64, 256), (64, 256, 128, 64)]:
+    for t in [(128, 128, 64, 128), (64, 256, 64, 256), (64, 256, 128, 64), (128, 256, 64, 512), (128, 128, 64, 512)]:
         Cg = run_gemm(mant, exp, inputs.to_bf16_bits(b), t)
         assert np.array_equal(inputs.bf16_bits_to_f32(Cg).astype(np.float64), Cr), t
 
@@ -91,7 +91,7 @@ def test_identity_B_returns_dequantised_A_bitwise():
     mant, exp = oracle.quantize_bfp16(A)
     eye = inputs.to_bf16_bits(np.eye(K, dtype=np.float32))
     want = oracle.dequantize(mant, exp)
-    for t in [(64, 128, 64, 128), (128, 256, 128, 256), (32, 256, 64, 64)]:
+    for t in [(64, 128, 64, 128), (128, 256, 128, 256), (32, 256, 64, 64), (64, 256, 64, 512)]:
         if not atb.atb_tiling_supported(*t):
             continue
         Cg = run_gemm(mant, exp, eye, t)
@@ -158,6 +158,7 @@ def test_tiny_and_degenerate_shapes():
         mant, exp = oracle.quantize_bfp16(A)
         _check(mant, exp, Bb, (128, 128, 64, 64))
         _check(mant, exp, Bb, (32, 256, 128, 128))
+        _check(mant, exp, Bb, (256, 256, 64, 512))       # CTA-pair kernel on a single partial tile
 
 
 def test_argument_errors():
@@ -191,7 +192,7 @@ def _sampled_rows(M, T_MC, n_random, seed):
 
 @pytest.mark.parametrize("name,tilings", [
     ("cfg2_4096", [(32, 256, 64, 256), (64, 256, 64, 256), (128, 256, 64, 256), (256, 256, 64, 256)]),
-    ("cfg3_8192", ["selected", (256, 256, 64, 256)]),
+    ("cfg3_8192", ["selected", (256, 256, 64, 256), (128, 256, 64, 512)]),
     ("cfg4_ffn_up", ["selected"]),
     ("cfg4_ffn_down", ["selected"]),
 ])
