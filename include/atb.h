@@ -130,6 +130,13 @@ typedef struct {
     int    share_rows, share_cols;/* array-level sharing factors of Eq. 2 (4 and 8 in the paper)  */
     double eta, eps_cycles, ii;   /* Eq. 13: Eff_micro = eta T_K / (eps + eta II T_K)             */
     double delta_cycles;          /* per-slab switching cost of Eq. 14                            */
+    /* Refinements beyond the paper (0 switches each one off; all 0 in the XDNA2 presets): */
+    int    mma_rows;              /* M extent of one MMA: a larger slab is consumed in pieces of this size, so Eq. 14-15
+                                     count rho_eff = T_MC / min(T_MA, mma_rows) switches (0: rho_eff = rho)          */
+    double load_latency_cycles;   /* atb_select_tiling: free-to-landed latency of a tile load; a B ring whose
+                                     look-ahead is shorter scales the compute bound down                    */
+    double pair_efficiency;       /* atb_select_tiling: measured factor on the compute bound of CTA-pair tilings */
+    double launch_seconds;        /* atb_select_tiling: fixed cost per kernel launch              */
 } atb_hw_params_t;
 
 typedef struct {

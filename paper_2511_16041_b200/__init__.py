@@ -42,7 +42,9 @@ class atb_hw_params_t(ctypes.Structure):
                                                "b_buf_bytes", "c_buf_bytes", "a_scratch_bytes",
                                                "buf_capacity_bytes", "acc_capacity_bytes")] + \
                [("share_rows", ctypes.c_int), ("share_cols", ctypes.c_int)] + \
-               [(n, ctypes.c_double) for n in ("eta", "eps_cycles", "ii", "delta_cycles")]
+               [(n, ctypes.c_double) for n in ("eta", "eps_cycles", "ii", "delta_cycles")] + \
+               [("mma_rows", ctypes.c_int)] + \
+               [(n, ctypes.c_double) for n in ("load_latency_cycles", "pair_efficiency", "launch_seconds")]
 
 
 class atb_tiling_score_t(ctypes.Structure):

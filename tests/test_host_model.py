@@ -33,7 +33,9 @@ def test_score_matches_oracle_formulas():
                 T_MA, T_MC, T_K, T_N = t
                 ai = model.ai_array(T_MC, T_N, K, hw.a_bytes, hw.b_bytes, hw.c_bytes, hw.share_rows, hw.share_cols)
                 em = model.eff_micro(T_K, hw.eta, hw.eps_cycles, hw.ii)
-                ec = model.eff_core(T_MA, T_MC, T_K, T_N, hw.peak_flops_per_cycle, em, hw.delta_cycles)
+                # a slab larger than the MMA's M extent is consumed in pieces: rho_eff of the preset
+                T_MA_eff = min(T_MA, hw.mma_rows) if hw.mma_rows > 0 else T_MA
+                ec = model.eff_core(T_MA_eff, T_MC, T_K, T_N, hw.peak_flops_per_cycle, em, hw.delta_cycles)
                 assert math.isclose(s.ai, ai, rel_tol=1e-12)
                 assert math.isclose(s.eff_micro, em, rel_tol=1e-12)
                 assert math.isclose(s.eff_core, ec, rel_tol=1e-12)
@@ -61,7 +63,12 @@ def test_select_tiling_orders_and_filters():
     # trade-off of Section 5: at fixed (T_MC, T_K, T_N) a larger rho never raises the compute bound,
     # and AI does not depend on T_MA or T_K
     by = {(s.t.T_MA, s.t.T_MC, s.t.T_K, s.t.T_N): s for s in scores}
-    assert by[(32, 256, 64, 256)].compute_bound_flops < by[(256, 256, 64, 256)].compute_bound_flops
+    assert by[(32, 256, 64, 256)].compute_bound_flops < by[(64, 256, 64, 256)].compute_bound_flops \
+        < by[(128, 256, 64, 256)].compute_bound_flops
+    # slabs of 256 and 128 rows are the same thing to a 128-row MMA: equal scores, the smaller buffer first
+    assert by[(128, 256, 64, 256)].predicted_flops == by[(256, 256, 64, 256)].predicted_flops
+    order = [(s.t.T_MA, s.t.T_MC, s.t.T_K, s.t.T_N) for s in scores]
+    assert order.index((128, 256, 64, 256)) < order.index((256, 256, 64, 256))
     assert by[(32, 256, 64, 256)].ai == by[(256, 256, 64, 256)].ai == by[(32, 256, 128, 256)].ai
 
 
@@ -71,6 +78,23 @@ def test_select_tiling_small_problem_prefers_more_tiles():
     big = [s for s in scores if (s.t.T_MC, s.t.T_N) == (256, 256)][0]
     small = [s for s in scores if (s.t.T_MC, s.t.T_N) == (128, 64)][0]
     assert small.compute_bound_flops > big.compute_bound_flops
+    assert (best.T_MC, best.T_N) != (256, 256)
+
+
+def test_b200_refinements_can_be_switched_off():
+    """With the four refinements at 0 the selection is the paper's Eq. 12 times wave quantisation."""
+    hw = atb.atb_hw_params_b200()
+    hw.mma_rows = 0; hw.load_latency_cycles = 0.0; hw.pair_efficiency = 0.0; hw.launch_seconds = 0.0
+    _, scores = atb.atb_select_tiling(8192, 8192, 8192, hw)
+    for s in scores:
+        t = (s.t.T_MA, s.t.T_MC, s.t.T_K, s.t.T_N)
+        if (t[1], t[3]) == (256, 512):
+            continue                                   # pair tilings are scored per CTA
+        ref = atb.atb_score_tiling(hw, 8192, t)
+        tiles = (8192 // t[1]) * (8192 // t[3])
+        useful = tiles / (math.ceil(tiles / 148) * 148)
+        want = min(ref.mem_bound_flops, ref.compute_bound_flops * useful)
+        assert math.isclose(s.predicted_flops, want, rel_tol=1e-12), t
 
 
 def test_select_tiling_errors():
