@@ -89,6 +89,27 @@ atb_status_t atb_gemm(int64_t M, int64_t N, int64_t K, int T_MA, int T_MC, int T
                       const void* B_bf16_dev, int64_t ldb,
                       void* C_bf16_dev, int64_t ldc, void* stream);
 
+/* Split-K variant of atb_gemm for shapes with few output tiles (M x N small, K large): every
+ * T_MC x T_N tile is computed as `splits` partial tiles over disjoint K ranges, written in FP32 to a
+ * caller-provided workspace and summed (FP32) into the BF16 result by a second kernel on the same
+ * stream.  The paper's hardware cannot do this - Section 2.2: an AIE core has no way to bring partial
+ * sums back, so every output tile is fully accumulated in L1 - here partial sums go through L2/HBM.
+ * Same operands and rules as atb_gemm.  Tilings: T_K = 64, T_MC in {128, 256}, T_N in {128, 256},
+ * T_MA in {64, 128}.  splits in [1, min(64, K / T_K)].
+ *   workspace_dev: device memory, 16-byte aligned, at least atb_gemm_splitk_workspace_bytes() bytes;
+ *                  fully overwritten; may be reused by the next call on the same stream.
+ * Errors: as atb_gemm, plus ATB_ERR_BUFFER_TOO_SMALL. */
+size_t atb_gemm_splitk_workspace_bytes(int64_t M, int64_t N, int T_MC, int splits);
+atb_status_t atb_gemm_splitk(int64_t M, int64_t N, int64_t K, int T_MA, int T_MC, int T_K, int T_N,
+                             const int8_t* A_mant_dev, const uint8_t* A_exp_dev,
+                             const void* B_bf16_dev, int64_t ldb,
+                             void* C_bf16_dev, int64_t ldc,
+                             int splits, float* workspace_dev, size_t workspace_bytes, void* stream);
+/* Number of K splits (a power of two, 1 = use atb_gemm) that the host heuristic expects to be
+ * fastest for this shape and tile: fills the SMs, keeps >= 8 K-steps per split, and charges the FP32
+ * partials' traffic.  Host only. */
+int atb_select_splits(int64_t M, int64_t N, int64_t K, int T_MC, int T_K, int T_N);
+
 /* 1 if atb_gemm accepts the tiling (kernel exists, TMEM and shared-memory budgets met), else 0.
  * Host only; touches no device. */
 int atb_tiling_supported(int T_MA, int T_MC, int T_K, int T_N);

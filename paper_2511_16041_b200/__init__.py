@@ -67,7 +67,8 @@ class Tiling(NamedTuple):
 
 EXPORTED_SYMBOLS = [
     "atb_status_string", "atb_last_error_message", "atb_bfp16_mant_bytes", "atb_bfp16_exp_bytes",
-    "atb_quantize_bfp16", "atb_gemm", "atb_tiling_supported", "atb_tiling_plan", "atb_device_status",
+    "atb_quantize_bfp16", "atb_gemm", "atb_gemm_splitk", "atb_gemm_splitk_workspace_bytes", "atb_select_splits",
+    "atb_tiling_supported", "atb_tiling_plan", "atb_device_status",
     "atb_hw_params_b200", "atb_hw_params_xdna2", "atb_score_tiling", "atb_select_tiling",
 ]
 
@@ -93,6 +94,12 @@ def load_library():
     lib.atb_quantize_bfp16.argtypes = [vp, i64, i64, i64, vp, vp, vp]
     lib.atb_gemm.restype = ci
     lib.atb_gemm.argtypes = [i64, i64, i64, ci, ci, ci, ci, vp, vp, vp, i64, vp, i64, vp]
+    lib.atb_gemm_splitk.restype = ci
+    lib.atb_gemm_splitk.argtypes = [i64, i64, i64, ci, ci, ci, ci, vp, vp, vp, i64, vp, i64, ci, vp, ctypes.c_size_t, vp]
+    lib.atb_gemm_splitk_workspace_bytes.restype = ctypes.c_size_t
+    lib.atb_gemm_splitk_workspace_bytes.argtypes = [i64, i64, ci, ci]
+    lib.atb_select_splits.restype = ci
+    lib.atb_select_splits.argtypes = [i64, i64, i64, ci, ci, ci]
     lib.atb_tiling_supported.restype = ci
     lib.atb_tiling_supported.argtypes = [ci, ci, ci, ci]
     lib.atb_tiling_plan.restype = ci
@@ -187,6 +194,33 @@ def atb_gemm(M, N, K, T_MA, T_MC, T_K, T_N, A_mant, A_exp, B, C=None, ldb=None, 
         ldc = C.stride(0) if not isinstance(C, int) else N
     _check(load_library().atb_gemm(M, N, K, T_MA, T_MC, T_K, T_N, _dev_ptr(A_mant), _dev_ptr(A_exp),
                                    _dev_ptr(B), ldb, _dev_ptr(C), ldc, _stream_ptr(stream)))
+    return C
+
+
+def atb_gemm_splitk_workspace_bytes(M: int, N: int, T_MC: int, splits: int) -> int:
+    return int(load_library().atb_gemm_splitk_workspace_bytes(M, N, T_MC, splits))
+
+
+def atb_select_splits(M: int, N: int, K: int, T_MC: int, T_K: int, T_N: int) -> int:
+    return int(load_library().atb_select_splits(M, N, K, T_MC, T_K, T_N))
+
+
+def atb_gemm_splitk(M, N, K, T_MA, T_MC, T_K, T_N, A_mant, A_exp, B, splits, workspace=None, C=None, ldb=None,
+                    ldc=None, stream=None):
+    """Split-K ``C[M][N] = dequant(A) @ B``; ``workspace`` is a float32 CUDA tensor (allocated if None)."""
+    import torch
+    if C is None:
+        C = torch.empty((M, N), dtype=torch.bfloat16, device=B.device)
+    if workspace is None:
+        workspace = torch.empty(atb_gemm_splitk_workspace_bytes(M, N, T_MC, splits) // 4, dtype=torch.float32,
+                                device=B.device)
+    if ldb is None:
+        ldb = B.stride(0)
+    if ldc is None:
+        ldc = C.stride(0)
+    _check(load_library().atb_gemm_splitk(M, N, K, T_MA, T_MC, T_K, T_N, _dev_ptr(A_mant), _dev_ptr(A_exp), _dev_ptr(B),
+                                          ldb, _dev_ptr(C), ldc, splits, _dev_ptr(workspace),
+                                          workspace.numel() * workspace.element_size(), _stream_ptr(stream)))
     return C
 
 

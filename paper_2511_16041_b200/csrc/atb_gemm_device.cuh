@@ -44,6 +44,13 @@ struct GemmParams {
     int m_tiles, n_tiles, k_steps;
     int n_b_stages, n_groups, n_raw_stages, acc_bufs, tmem_cols;
     unsigned int* error_flag;
+    int splits;          // split-K: each output tile is computed as `splits` partial tiles over K ranges
+    int m_pad;           // split-K: rows per split in the FP32 workspace (m_tiles * T_MC)
+};
+
+// One unit of work of a persistent CTA: an output tile and the K-steps [k_begin, k_end) of it.
+struct WorkItem {
+    int mt, nt, k_begin, k_end, split;
 };
 
 struct Ring {
@@ -101,6 +108,24 @@ __device__ __forceinline__ void tile_coords(int tile, int m_tiles, int n_tiles, 
     const int rows = min(16, m_tiles - band * 16);
     mt = band * 16 + i % rows;
     nt = i / rows;
+}
+
+template <bool SPLIT>
+__device__ __forceinline__ WorkItem work_item(int item, const GemmParams& p) {
+    WorkItem w;
+    if (SPLIT) {
+        const int total_tiles = p.m_tiles * p.n_tiles;
+        w.split = item / total_tiles;
+        tile_coords(item - w.split * total_tiles, p.m_tiles, p.n_tiles, w.mt, w.nt);
+        w.k_begin = static_cast<int>(static_cast<int64_t>(w.split) * p.k_steps / p.splits);
+        w.k_end = static_cast<int>(static_cast<int64_t>(w.split + 1) * p.k_steps / p.splits);
+    } else {
+        w.split = 0;
+        tile_coords(item, p.m_tiles, p.n_tiles, w.mt, w.nt);
+        w.k_begin = 0;
+        w.k_end = p.k_steps;
+    }
+    return w;
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -18,6 +18,9 @@
 //   accumulators     (acc_bufs x T_MC/128 row groups in TMEM)  UMMA -> epilogue
 // The UMMA shape is always 128 x T_N x 16.  A slab of T_MA < 128 rows is the unit of loading,
 // dequantising and signalling; 128 / T_MA consecutive slabs fill one 128-row operand group.
+#include <algorithm>
+#include <cmath>
+
 #include "atb_gemm_device.cuh"
 
 namespace {
@@ -50,7 +53,7 @@ struct Cfg {
 };
 
 // ---------------------------------------------------------------------------------------------
-template <int T_MA, int T_MC, int T_K, int T_N>
+template <int T_MA, int T_MC, int T_K, int T_N, bool SPLIT>
 __global__ void __launch_bounds__(kThreads, 1)
 atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_constant__ CUtensorMap tm_exp,
                 const __grid_constant__ CUtensorMap tm_b, const __grid_constant__ CUtensorMap tm_c,
@@ -109,17 +112,17 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
     tcgen05_fence_after_sync();
     const uint32_t tmem_base = misc_gen[0];
 
-    const int total_tiles = p.m_tiles * p.n_tiles;
+    const int total_items = p.m_tiles * p.n_tiles * (SPLIT ? p.splits : 1);
 
     if (warp == 0) {
         // ================================ TMA producer ================================
         if (elect_one()) {
             Ring rb, rr;
             bool ok = true;
-            for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
-                int mt, nt;
-                tile_coords(tile, p.m_tiles, p.n_tiles, mt, nt);
-                for (int k = 0; ok && k < p.k_steps; ++k) {
+            for (int item = blockIdx.x; ok && item < total_items; item += gridDim.x) {
+                const WorkItem w = work_item<SPLIT>(item, p);
+                const int mt = w.mt, nt = w.nt;
+                for (int k = w.k_begin; ok && k < w.k_end; ++k) {
                     if (!(ok = wait_bar_spin(cx, b_empty + 8 * rb.stage, rb.phase ^ 1u, 0x001))) break;
                     const uint32_t fb = b_full + 8 * rb.stage;
                     mbar_arrive_expect_tx(fb, C::B_BYTES);
@@ -147,15 +150,16 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
             Ring rb, rd;
             int it = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++it) {
+            for (int item = blockIdx.x; ok && item < total_items; item += gridDim.x, ++it) {
+                const WorkItem w = work_item<SPLIT>(item, p);
                 const int acc_buf = it % p.acc_bufs;
                 const uint32_t acc_phase = static_cast<uint32_t>(it / p.acc_bufs) & 1u;
-                for (int k = 0; ok && k < p.k_steps; ++k) {
+                for (int k = w.k_begin; ok && k < w.k_end; ++k) {
                     if (!(ok = wait_bar_spin(cx, b_full + 8 * rb.stage, rb.phase, 0x101))) break;
                     const uint32_t bs = b_base + rb.stage * C::B_BYTES;
                     for (int g = 0; g < C::G; ++g) {
                         const int acc = acc_buf * C::G + g;
-                        if (k == 0 && !(ok = wait_bar_spin(cx, acc_empty + 8 * acc, acc_phase ^ 1u, 0x102))) break;
+                        if (k == w.k_begin && !(ok = wait_bar_spin(cx, acc_empty + 8 * acc, acc_phase ^ 1u, 0x102))) break;
                         int group_slot;
                         if (T_MA <= 128) {
                             for (int i = 0; ok && i < C::SPG; ++i)
@@ -176,7 +180,7 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
                                 const uint64_t a_desc = umma_smem_desc_sw128(as + (kk >> 2) * C::KHALF_BYTES + (kk & 3) * 32, 16, 1024);
                                 const uint64_t b_desc = umma_smem_desc_sw128(bs + nc * (C::N_MMA / 64) * C::B_BOX_BYTES + kk * 2048,
                                                                              C::B_BOX_BYTES, 1024);
-                                umma_f16_ss(d_tmem + nc * C::N_MMA, a_desc, b_desc, idesc, (k > 0 || kk > 0) ? 1u : 0u);
+                                umma_f16_ss(d_tmem + nc * C::N_MMA, a_desc, b_desc, idesc, (k > w.k_begin || kk > 0) ? 1u : 0u);
                             }
                         }
                         if (T_MA <= 128) {
@@ -186,7 +190,7 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
                             umma_commit(deq_empty + 8 * rd.stage);
                             rd.advance(n_deq_stages);
                         }
-                        if (k == p.k_steps - 1) umma_commit(acc_full + 8 * acc);
+                        if (k == w.k_end - 1) umma_commit(acc_full + 8 * acc);
                     }
                     if (!ok) break;
                     umma_commit(b_empty + 8 * rb.stage);
@@ -199,9 +203,9 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
         const int q = warp & 3;                       // TMEM lane quadrant this warp may access
         int it = 0;
         bool ok = true;
-        for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++it) {
-            int mt, nt;
-            tile_coords(tile, p.m_tiles, p.n_tiles, mt, nt);
+        for (int item = blockIdx.x; ok && item < total_items; item += gridDim.x, ++it) {
+            const WorkItem w = work_item<SPLIT>(item, p);
+            const int mt = w.mt, nt = w.nt;
             const int acc_buf = it % p.acc_bufs;
             const uint32_t acc_phase = static_cast<uint32_t>(it / p.acc_bufs) & 1u;
             for (int g = 0; g < C::G; ++g) {
@@ -214,6 +218,27 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
                 const uint32_t box = smem_base + stage_off + static_cast<uint32_t>(warp - kFirstEpilogueWarp) * kEpilogueBoxBytes;
                 const uint32_t my_row = box + lane * 128;
                 const uint32_t sw = static_cast<uint32_t>(lane & 7);
+                if (SPLIT) {
+                    // FP32 partial tile -> workspace [split][m_pad][N]: boxes of 32 rows x 32 columns
+#pragma unroll 1
+                    for (int c = 0; c < T_N / 32; ++c) {
+                        if (lane == 0) tma_store_wait_read<0>();
+                        __syncwarp();
+                        uint32_t v[32];
+                        tmem_ld_32x32b_x32(t_addr + c * 32, v);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int j = 0; j < 8; ++j)
+                            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(my_row + ((static_cast<uint32_t>(j) ^ sw) << 4)),
+                                         "r"(v[4 * j]), "r"(v[4 * j + 1]), "r"(v[4 * j + 2]), "r"(v[4 * j + 3]) : "memory");
+                        fence_proxy_async_smem();
+                        __syncwarp();
+                        if (lane == 0 && col0 + c * 32 < p.N) {
+                            tma_store_2d(&tm_c, box, col0 + c * 32, w.split * p.m_pad + row0);
+                            tma_store_commit();
+                        }
+                    }
+                } else {
 #pragma unroll 1
                 for (int c = 0; c < T_N / 64; ++c) {
                     // the previous TMA store of this warp must have finished reading the box
@@ -244,6 +269,7 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
                         tma_store_commit();
                     }
                 }
+                }
                 tcgen05_fence_before_sync();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(acc_empty + 8 * acc);
@@ -258,8 +284,9 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
         for (int i = 0; i < my_group; ++i) { rr.advance(p.n_raw_stages); rd.advance(n_deq_stages); }
         int turn = 0;                                   // slab sequence number modulo the group count
         bool ok = true;
-        for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
-            for (int k = 0; ok && k < p.k_steps; ++k) {
+        for (int item = blockIdx.x; ok && item < total_items; item += gridDim.x) {
+            const WorkItem w = work_item<SPLIT>(item, p);
+            for (int k = w.k_begin; ok && k < w.k_end; ++k) {
                 for (int s = 0; s < C::RHO; ++s) {
                     const bool mine = (turn == my_group);
                     if (++turn == C::DQ_GROUPS) turn = 0;
@@ -304,10 +331,12 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
 // ---------------------------------------------------------------------------------------------
 // Host side
 // ---------------------------------------------------------------------------------------------
-template <int T_MA, int T_MC, int T_K, int T_N>
+// SPLIT = false: Cout is bf16 C[M][ldc].  SPLIT = true: Cout is the FP32 workspace
+// [splits][m_tiles * T_MC][N] that receives one partial tile per (tile, split).
+template <int T_MA, int T_MC, int T_K, int T_N, bool SPLIT = false>
 atb_status_t launch(const atb::GemmPlan& plan, int64_t M, int64_t N, int64_t K, const int8_t* mant,
                     const uint8_t* exp, const void* B, int64_t ldb, void* Cout, int64_t ldc,
-                    int num_sms, unsigned int* error_flag, cudaStream_t stream) {
+                    int num_sms, unsigned int* error_flag, cudaStream_t stream, int splits = 1) {
     CUtensorMap tm_mant, tm_exp, tm_b, tm_c;
     const int64_t M_pad = atb::round_up(M, 32);
     if (!make_map_2d(&tm_mant, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, mant, K, M, K, T_K, T_MA, CU_TENSOR_MAP_SWIZZLE_NONE))
@@ -317,8 +346,13 @@ atb_status_t launch(const atb::GemmPlan& plan, int64_t M, int64_t N, int64_t K, 
         return atb::fail(ATB_ERR_CUDA, "cuTensorMapEncodeTiled failed for the exponent plane");
     if (!make_map_2d(&tm_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, B, N, K, ldb * 2, 64, T_K, CU_TENSOR_MAP_SWIZZLE_128B))
         return atb::fail(ATB_ERR_CUDA, "cuTensorMapEncodeTiled failed for B");
-    if (!make_map_2d(&tm_c, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Cout, N, M, ldc * 2, 64, 32, CU_TENSOR_MAP_SWIZZLE_128B))
+    const int64_t m_pad = atb::ceil_div(M, T_MC) * T_MC;
+    if (SPLIT) {
+        if (!make_map_2d(&tm_c, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, Cout, N, splits * m_pad, N * 4, 32, 32, CU_TENSOR_MAP_SWIZZLE_128B))
+            return atb::fail(ATB_ERR_CUDA, "cuTensorMapEncodeTiled failed for the split-K workspace");
+    } else if (!make_map_2d(&tm_c, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Cout, N, M, ldc * 2, 64, 32, CU_TENSOR_MAP_SWIZZLE_128B)) {
         return atb::fail(ATB_ERR_CUDA, "cuTensorMapEncodeTiled failed for C");
+    }
 
     GemmParams p;
     p.M = M; p.N = N; p.K = K; p.ldc = ldc;
@@ -329,16 +363,44 @@ atb_status_t launch(const atb::GemmPlan& plan, int64_t M, int64_t N, int64_t K, 
     p.n_b_stages = plan.n_b_stages; p.n_groups = plan.n_groups; p.n_raw_stages = plan.n_raw_stages;
     p.acc_bufs = plan.acc_bufs; p.tmem_cols = plan.tmem_cols;
     p.error_flag = error_flag;
+    p.splits = splits;
+    p.m_pad = static_cast<int>(m_pad);
 
-    auto kernel = atb_gemm_kernel<T_MA, T_MC, T_K, T_N>;
+    auto kernel = atb_gemm_kernel<T_MA, T_MC, T_K, T_N, SPLIT>;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(plan.smem_bytes));
     if (e != cudaSuccess) return atb::fail(ATB_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
-    const int64_t tiles = static_cast<int64_t>(p.m_tiles) * p.n_tiles;
-    const int grid = static_cast<int>(tiles < num_sms ? tiles : num_sms);
+    const int64_t items = static_cast<int64_t>(p.m_tiles) * p.n_tiles * splits;
+    const int grid = static_cast<int>(items < num_sms ? items : num_sms);
     kernel<<<grid, kThreads, plan.smem_bytes, stream>>>(tm_mant, tm_exp, tm_b, tm_c, p);
     e = cudaGetLastError();
     if (e != cudaSuccess) return atb::fail(ATB_ERR_CUDA, "gemm launch: %s", cudaGetErrorString(e));
     return ATB_OK;
+}
+
+// Split-K reduction: C[m][n] = bf16(sum over splits of the FP32 partials), 8 columns per thread.
+__global__ void __launch_bounds__(256)
+splitk_reduce_kernel(const float* __restrict__ ws, int splits, int64_t m_pad, int64_t M, int64_t N,
+                     __nv_bfloat16* __restrict__ C, int64_t ldc) {
+    const int64_t vec_per_row = N >> 3;
+    const int64_t total = M * vec_per_row;
+    for (int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; i < total;
+         i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+        const int64_t m = i / vec_per_row, n = (i - m * vec_per_row) << 3;
+        float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+        for (int s = 0; s < splits; ++s) {
+            const float4* src = reinterpret_cast<const float4*>(ws + (s * m_pad + m) * N + n);
+            const float4 a = __ldg(src), b = __ldg(src + 1);
+            acc[0] += a.x; acc[1] += a.y; acc[2] += a.z; acc[3] += a.w;
+            acc[4] += b.x; acc[5] += b.y; acc[6] += b.z; acc[7] += b.w;
+        }
+        uint32_t o[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            __nv_bfloat162 b2 = __floats2bfloat162_rn(acc[2 * j], acc[2 * j + 1]);
+            o[j] = *reinterpret_cast<uint32_t*>(&b2);
+        }
+        *reinterpret_cast<uint4*>(C + m * ldc + n) = make_uint4(o[0], o[1], o[2], o[3]);
+    }
 }
 
 struct DeviceInfo {
@@ -527,4 +589,105 @@ extern "C" atb_status_t atb_device_status(void* stream) {
         return atb::fail(ATB_ERR_DEVICE_TIMEOUT, "a GEMM kernel gave up a bounded wait (code 0x%03x)", flag);
     }
     return ATB_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Split-K
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+bool splitk_tiling_ok(int T_MA, int T_MC, int T_K, int T_N) {
+    return T_K == 64 && (T_MC == 128 || T_MC == 256) && (T_N == 128 || T_N == 256) &&
+           (T_MA == 64 || T_MA == 128) && T_MA <= T_MC;
+}
+
+atb_status_t splitk_validate(int64_t M, int64_t N, int64_t K, int T_MA, int T_MC, int T_K, int T_N, int splits) {
+    if (M < 1 || N < 8 || N % 8 != 0 || K < 64 || K % 64 != 0 || M > (1ll << 30) || N > (1ll << 30) || K > (1ll << 30))
+        return atb::fail(ATB_ERR_BAD_SHAPE, "need M >= 1, N %% 8 == 0, K %% 64 == 0 (got %lld, %lld, %lld)", (long long)M, (long long)N, (long long)K);
+    if (!splitk_tiling_ok(T_MA, T_MC, T_K, T_N))
+        return atb::fail(ATB_ERR_BAD_TILING, "split-K supports T_K = 64, T_MC in {128, 256}, T_N in {128, 256}, T_MA in {64, 128}");
+    if (splits < 1 || splits > 64 || splits > K / T_K)
+        return atb::fail(ATB_ERR_BAD_SHAPE, "splits=%d must be in [1, min(64, K / T_K)]", splits);
+    return ATB_OK;
+}
+
+}  // namespace
+
+extern "C" size_t atb_gemm_splitk_workspace_bytes(int64_t M, int64_t N, int T_MC, int splits) {
+    if (M < 1 || N < 1 || T_MC < 1 || splits < 1) return 0;
+    return static_cast<size_t>(splits) * static_cast<size_t>(atb::ceil_div(M, T_MC) * T_MC) * static_cast<size_t>(N) * sizeof(float);
+}
+
+namespace atb {
+
+// Runs the split-K GEMM with partials in `ws` (device, at least the documented size) and reduces.
+atb_status_t gemm_splitk_with_workspace(int64_t M, int64_t N, int64_t K, int T_MA, int T_MC, int T_K, int T_N,
+                                        const int8_t* mant, const uint8_t* exp, const void* B, int64_t ldb,
+                                        void* C, int64_t ldc, int splits, float* ws, void* stream) {
+    GemmPlan plan;
+    if (!plan_gemm(T_MA, T_MC, T_K, T_N, &plan))
+        return fail(ATB_ERR_BAD_TILING, "tiling (T_MA=%d, T_MC=%d, T_K=%d, T_N=%d) is not supported", T_MA, T_MC, T_K, T_N);
+    DeviceInfo* dev = nullptr;
+    atb_status_t st_dev = device_info(&dev);
+    if (st_dev != ATB_OK) return st_dev;
+    if (dev->cc_major != 10 || dev->cc_minor != 0)
+        return fail(ATB_ERR_UNSUPPORTED_DEVICE, "compute capability %d.%d; this library runs on 10.0 only", dev->cc_major, dev->cc_minor);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    atb_status_t rc = ATB_ERR_BAD_TILING;
+#define ATB_SPLIT_CASE(TMA_, TMC_, TN_)                                                                         \
+    if (T_MA == TMA_ && T_MC == TMC_ && T_N == TN_)                                                             \
+        rc = launch<TMA_, TMC_, 64, TN_, true>(plan, M, N, K, mant, exp, B, ldb, ws, 0, dev->num_sms, dev->error_flag, st, splits);
+    ATB_SPLIT_CASE(64, 128, 128) ATB_SPLIT_CASE(128, 128, 128) ATB_SPLIT_CASE(64, 128, 256) ATB_SPLIT_CASE(128, 128, 256)
+    ATB_SPLIT_CASE(64, 256, 128) ATB_SPLIT_CASE(128, 256, 128) ATB_SPLIT_CASE(64, 256, 256) ATB_SPLIT_CASE(128, 256, 256)
+#undef ATB_SPLIT_CASE
+    if (rc != ATB_OK) return rc;
+    const int64_t vecs = M * (N / 8);
+    const int blocks = static_cast<int>(std::min<int64_t>((vecs + 255) / 256, static_cast<int64_t>(dev->num_sms) * 8));
+    splitk_reduce_kernel<<<blocks, 256, 0, st>>>(ws, splits, ceil_div(M, T_MC) * T_MC, M, N,
+                                                 static_cast<__nv_bfloat16*>(C), ldc);
+    const cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return fail(ATB_ERR_CUDA, "split-K reduce launch: %s", cudaGetErrorString(e));
+    return ATB_OK;
+}
+
+}  // namespace atb
+
+extern "C" atb_status_t atb_gemm_splitk(int64_t M, int64_t N, int64_t K, int T_MA, int T_MC, int T_K, int T_N,
+                                        const int8_t* A_mant_dev, const uint8_t* A_exp_dev,
+                                        const void* B_bf16_dev, int64_t ldb, void* C_bf16_dev, int64_t ldc,
+                                        int splits, float* workspace_dev, size_t workspace_bytes, void* stream) {
+    atb::clear_error();
+    if (!A_mant_dev || !A_exp_dev || !B_bf16_dev || !C_bf16_dev || !workspace_dev)
+        return atb::fail(ATB_ERR_NULL_POINTER, "all device pointers, including the workspace, must be non-NULL");
+    atb_status_t v = splitk_validate(M, N, K, T_MA, T_MC, T_K, T_N, splits);
+    if (v != ATB_OK) return v;
+    if (ldb < N || ldc < N || ldb % 8 != 0 || ldc % 8 != 0)
+        return atb::fail(ATB_ERR_BAD_SHAPE, "ldb=%lld and ldc=%lld must be >= N and multiples of 8", (long long)ldb, (long long)ldc);
+    if (!atb::aligned16(A_mant_dev) || !atb::aligned16(A_exp_dev) || !atb::aligned16(B_bf16_dev) ||
+        !atb::aligned16(C_bf16_dev) || !atb::aligned16(workspace_dev))
+        return atb::fail(ATB_ERR_MISALIGNED, "all device pointers must be 16-byte aligned");
+    if (workspace_bytes < atb_gemm_splitk_workspace_bytes(M, N, T_MC, splits))
+        return atb::fail(ATB_ERR_BUFFER_TOO_SMALL, "workspace of %zu bytes is smaller than the %zu needed", workspace_bytes,
+                         atb_gemm_splitk_workspace_bytes(M, N, T_MC, splits));
+    return atb::gemm_splitk_with_workspace(M, N, K, T_MA, T_MC, T_K, T_N, A_mant_dev, A_exp_dev, B_bf16_dev, ldb,
+                                           C_bf16_dev, ldc, splits, workspace_dev, stream);
+}
+
+extern "C" int atb_select_splits(int64_t M, int64_t N, int64_t K, int T_MC, int T_K, int T_N) {
+    if (M < 1 || N < 1 || K < 1 || T_MC < 1 || T_K < 1 || T_N < 1) return 1;
+    const int64_t tiles = atb::ceil_div(M, T_MC) * atb::ceil_div(N, T_N);
+    const int64_t k_steps = atb::ceil_div(K, T_K);
+    // Fill the 148 SMs once, keep at least 8 K-steps per split, and stop where the FP32 partials
+    // (written and read once each) would cost more than the GEMM itself saves.
+    int best = 1;
+    double best_t = 1e300;
+    for (int s = 1; s <= 32; s *= 2) {
+        if (s > 1 && k_steps / s < 8) break;
+        const double waves = std::ceil(static_cast<double>(tiles * s) / 148.0);
+        const double t_gemm = waves * (static_cast<double>(k_steps) / s) * (2.0 * T_MC * T_N * T_K / 8192.0 / 0.8);   // cycles
+        const double t_part = s > 1 ? (2.0 * s * M * N * 4.0) / (3.0e12 / 1.4e9) : 0.0;                             // cycles at ~3 TB/s
+        const double t = t_gemm + t_part + (s > 1 ? 8000.0 : 0.0);
+        if (t < best_t) { best_t = t; best = s; }
+    }
+    return best;
 }
