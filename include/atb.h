@@ -110,6 +110,35 @@ atb_status_t atb_gemm_splitk(int64_t M, int64_t N, int64_t K, int T_MA, int T_MC
  * partials' traffic.  Host only. */
 int atb_select_splits(int64_t M, int64_t N, int64_t K, int T_MC, int T_K, int T_N);
 
+/* atb_gemm_splitk for callers that must not allocate.  (The paper has no counterpart: this is an
+ * integration convenience of this library, not part of the method.)
+ *
+ * Who needs it: code that sits under somebody else's memory manager - an operator plugged into an
+ * inference server or a framework whose pool has claimed the device memory, where a stray cudaMalloc
+ * can fail, fragment the pool or stall every stream with its implicit synchronisation - and
+ * latency-bound loops that are simply forbidden to call an allocator after start-up.  Such callers
+ * still pass the operands and the result; what they are spared is finding room for the FP32 partial
+ * sums.  Those go to a fixed array of ATB_NOALLOC_SCRATCH_BYTES that is linked into the library: every
+ * GPU that loads the library keeps that much memory reserved until the process ends, used or not.
+ *
+ * Same arguments, tilings and results as atb_gemm_splitk (bit for bit), minus the workspace pair.
+ *   - Limit: atb_gemm_splitk_workspace_bytes(M, N, T_MC, splits) must not exceed
+ *     ATB_NOALLOC_SCRATCH_BYTES, else ATB_ERR_BUFFER_TOO_SMALL and nothing is launched (e.g. 1024 x 1024
+ *     with up to 16 splits, 2048 x 2048 with up to 4).
+ *   - The call itself performs no cudaMalloc / cudaFree and calls no allocating library routine.
+ *   - The first call on each device looks the array's device address up (cudaGetSymbolAddress, with
+ *     that device current) and remembers it; make that first call before starting any stream capture.
+ *   - All calls share the one array and it keeps whatever the last call left there.  Nothing has to be
+ *     cleared: every partial sum the reduction reads is written earlier by the same call.  For the same
+ *     reason two calls whose kernels can run at the same time on one GPU (different streams, or
+ *     different host threads) would trample each other's partial sums: order them on one stream or
+ *     with events. */
+#define ATB_NOALLOC_SCRATCH_BYTES (64u * 1024u * 1024u)
+atb_status_t atb_gemm_splitk_noalloc(int64_t M, int64_t N, int64_t K, int T_MA, int T_MC, int T_K, int T_N,
+                                     const int8_t* A_mant_dev, const uint8_t* A_exp_dev,
+                                     const void* B_bf16_dev, int64_t ldb,
+                                     void* C_bf16_dev, int64_t ldc, int splits, void* stream);
+
 /* 1 if atb_gemm accepts the tiling (kernel exists, TMEM and shared-memory budgets met), else 0.
  * Host only; touches no device. */
 int atb_tiling_supported(int T_MA, int T_MC, int T_K, int T_N);

@@ -68,6 +68,7 @@ class Tiling(NamedTuple):
 EXPORTED_SYMBOLS = [
     "atb_status_string", "atb_last_error_message", "atb_bfp16_mant_bytes", "atb_bfp16_exp_bytes",
     "atb_quantize_bfp16", "atb_gemm", "atb_gemm_splitk", "atb_gemm_splitk_workspace_bytes", "atb_select_splits",
+    "atb_gemm_splitk_noalloc",
     "atb_tiling_supported", "atb_tiling_plan", "atb_device_status",
     "atb_hw_params_b200", "atb_hw_params_xdna2", "atb_score_tiling", "atb_select_tiling",
 ]
@@ -96,6 +97,8 @@ def load_library():
     lib.atb_gemm.argtypes = [i64, i64, i64, ci, ci, ci, ci, vp, vp, vp, i64, vp, i64, vp]
     lib.atb_gemm_splitk.restype = ci
     lib.atb_gemm_splitk.argtypes = [i64, i64, i64, ci, ci, ci, ci, vp, vp, vp, i64, vp, i64, ci, vp, ctypes.c_size_t, vp]
+    lib.atb_gemm_splitk_noalloc.restype = ci
+    lib.atb_gemm_splitk_noalloc.argtypes = [i64, i64, i64, ci, ci, ci, ci, vp, vp, vp, i64, vp, i64, ci, vp]
     lib.atb_gemm_splitk_workspace_bytes.restype = ctypes.c_size_t
     lib.atb_gemm_splitk_workspace_bytes.argtypes = [i64, i64, ci, ci]
     lib.atb_select_splits.restype = ci
@@ -221,6 +224,25 @@ def atb_gemm_splitk(M, N, K, T_MA, T_MC, T_K, T_N, A_mant, A_exp, B, splits, wor
     _check(load_library().atb_gemm_splitk(M, N, K, T_MA, T_MC, T_K, T_N, _dev_ptr(A_mant), _dev_ptr(A_exp), _dev_ptr(B),
                                           ldb, _dev_ptr(C), ldc, splits, _dev_ptr(workspace),
                                           workspace.numel() * workspace.element_size(), _stream_ptr(stream)))
+    return C
+
+
+NOALLOC_SCRATCH_BYTES = 64 * 1024 * 1024
+
+
+def atb_gemm_splitk_noalloc(M, N, K, T_MA, T_MC, T_K, T_N, A_mant, A_exp, B, splits, C, ldb=None, ldc=None, stream=None):
+    """Split-K GEMM whose partial sums live in the library's built-in 64 MiB device array.
+
+    For callers that may not allocate: the binding allocates nothing either, so ``C`` (bf16 CUDA tensor)
+    has to be passed in.  Raises ``AtbError`` (ATB_ERR_BUFFER_TOO_SMALL) when
+    ``atb_gemm_splitk_workspace_bytes(M, N, T_MC, splits)`` exceeds ``NOALLOC_SCRATCH_BYTES``.
+    Calls that may overlap on the GPU must be ordered by the caller: they share the array."""
+    if ldb is None:
+        ldb = B.stride(0)
+    if ldc is None:
+        ldc = C.stride(0)
+    _check(load_library().atb_gemm_splitk_noalloc(M, N, K, T_MA, T_MC, T_K, T_N, _dev_ptr(A_mant), _dev_ptr(A_exp),
+                                                  _dev_ptr(B), ldb, _dev_ptr(C), ldc, splits, _stream_ptr(stream)))
     return C
 
 

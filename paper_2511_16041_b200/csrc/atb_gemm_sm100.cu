@@ -691,3 +691,63 @@ extern "C" int atb_select_splits(int64_t M, int64_t N, int64_t K, int T_MC, int 
     }
     return best;
 }
+
+// ---------------------------------------------------------------------------------------------
+// Split-K without a caller workspace and without any allocation
+// ---------------------------------------------------------------------------------------------
+// The FP32 partial tiles go to this fixed array instead of caller memory.  It is part of the
+// library image: every GPU on which the library's module gets loaded sets the 64 MiB aside until
+// the process exits, whether or not this entry point is ever called.
+static __device__ __align__(256) float g_splitk_scratch[ATB_NOALLOC_SCRATCH_BYTES / sizeof(float)];
+
+namespace {
+
+// In host code `g_splitk_scratch` is only a handle for the runtime, not an address a kernel can
+// use; the device address has to be asked for, per device, with that device current.
+float* g_scratch_ptr[64] = {};
+std::mutex g_scratch_mutex;
+
+atb_status_t scratch_address(float** out) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return atb::fail(ATB_ERR_CUDA, "cudaGetDevice: %s", cudaGetErrorString(e));
+    if (dev < 0 || dev >= 64) return atb::fail(ATB_ERR_UNSUPPORTED_DEVICE, "device ordinal %d out of range", dev);
+    std::lock_guard<std::mutex> lock(g_scratch_mutex);
+    if (!g_scratch_ptr[dev]) {
+        float* ptr = nullptr;
+        e = cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_splitk_scratch);
+        if (e != cudaSuccess || !ptr)
+            return atb::fail(ATB_ERR_CUDA, "cudaGetSymbolAddress(split-K scratch): %s", cudaGetErrorString(e));
+        g_scratch_ptr[dev] = ptr;
+    }
+    *out = g_scratch_ptr[dev];
+    return ATB_OK;
+}
+
+}  // namespace
+
+extern "C" atb_status_t atb_gemm_splitk_noalloc(int64_t M, int64_t N, int64_t K, int T_MA, int T_MC, int T_K, int T_N,
+                                                const int8_t* A_mant_dev, const uint8_t* A_exp_dev,
+                                                const void* B_bf16_dev, int64_t ldb, void* C_bf16_dev, int64_t ldc,
+                                                int splits, void* stream) {
+    atb::clear_error();
+    if (!A_mant_dev || !A_exp_dev || !B_bf16_dev || !C_bf16_dev)
+        return atb::fail(ATB_ERR_NULL_POINTER, "A_mant_dev, A_exp_dev, B_bf16_dev and C_bf16_dev must be non-NULL");
+    atb_status_t v = splitk_validate(M, N, K, T_MA, T_MC, T_K, T_N, splits);
+    if (v != ATB_OK) return v;
+    if (ldb < N || ldc < N || ldb % 8 != 0 || ldc % 8 != 0)
+        return atb::fail(ATB_ERR_BAD_SHAPE, "ldb=%lld and ldc=%lld must be >= N and multiples of 8", (long long)ldb, (long long)ldc);
+    if (!atb::aligned16(A_mant_dev) || !atb::aligned16(A_exp_dev) || !atb::aligned16(B_bf16_dev) || !atb::aligned16(C_bf16_dev))
+        return atb::fail(ATB_ERR_MISALIGNED, "all device pointers must be 16-byte aligned");
+    const size_t need = atb_gemm_splitk_workspace_bytes(M, N, T_MC, splits);
+    if (need > static_cast<size_t>(ATB_NOALLOC_SCRATCH_BYTES))
+        return atb::fail(ATB_ERR_BUFFER_TOO_SMALL,
+                         "splits * roundup(M, T_MC) * N * 4 = %zu bytes of partial sums exceed the built-in scratch of %zu bytes; "
+                         "use fewer splits or atb_gemm_splitk with a workspace of your own",
+                         need, static_cast<size_t>(ATB_NOALLOC_SCRATCH_BYTES));
+    float* scratch = nullptr;
+    v = scratch_address(&scratch);
+    if (v != ATB_OK) return v;
+    return atb::gemm_splitk_with_workspace(M, N, K, T_MA, T_MC, T_K, T_N, A_mant_dev, A_exp_dev, B_bf16_dev, ldb,
+                                           C_bf16_dev, ldc, splits, scratch, stream);
+}
