@@ -31,9 +31,9 @@ sys.path.insert(0, ROOT)
 METRIC = "ATB GEMM TFLOPS (1xB200) at 8192^3 BFP16xBF16"
 DEFAULT_WORKLOAD = "cfg3_8192"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# dram__bytes_read.sum + dram__bytes_write.sum per GEMM launch, from the ncu capture summarised in
-# profiles/ (None until a capture of that workload exists).
-NCU_TRAFFIC_BYTES = {}
+# dram__bytes_read.sum + dram__bytes_write.sum per GEMM launch of the full workload, from the 1-pass ncu
+# capture summarised in profiles/atb_gemm_kernel_dram_traffic_cfg3_8192.md (None where no capture exists).
+NCU_TRAFFIC_BYTES = {"cfg3_8192": 569.5e6 + 116.2e6}
 
 
 def load_peaks():
