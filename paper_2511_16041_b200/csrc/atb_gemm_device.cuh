@@ -134,27 +134,31 @@ __device__ __forceinline__ WorkItem work_item(int item, const GemmParams& p) {
 // GROUP_THREADS / SPR, t % SPR), a slot being two blocks: 16 mantissa bytes (one 16-byte load; the loads of
 // a warp are contiguous), two exponent bytes, and two 16-byte stores into the swizzled row.
 //
-// Per element: the byte u = m + 128 is dropped into the mantissa of the float 2^23 (bit pattern
-// 0x4B0000uu = 2^23 + u); subtracting 2^23 + 128 leaves m exactly, and the product with the
-// block scale 2^(E-133) (taken from a 256-entry table: normal for E >= 7, fp32-subnormal below) is
-// exact for every E.  The result has at most 7 significant bits, so its low 16 bits are zero and
-// the bf16 value is the upper half of the word.
-__device__ __forceinline__ uint64_t pack_f32x2(uint32_t lo, uint32_t hi) {
-    uint64_t r;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+// Per pair of elements (all packed, two values per 32-bit register):
+//   1. prmt drops the bytes u = m + 128 (1..255) into the mantissas of two fp16 values 1024
+//      (0x64uu = 1024 + u); subtracting 1024 (add.f16x2) normalises them: u as fp16, exact.
+//   2. u is positive and non-zero, so fp16 -> bf16 is pure bit arithmetic: drop 3 mantissa bits
+//      (they are zero: u has at most 8 significant bits) and re-bias the exponent by 112 -
+//      (h >> 3) + 0x3800 per half, done for both halves by one mad.hi.u32 (x * 2^29 >> 32).
+//   3. add.bf16x2 subtracts 128 (m, exact: 7 significant bits), mul.bf16x2 scales by the block's
+//      2^(E-133) (from a 256-entry table of packed bf16 pairs: normal for E >= 7, bf16-subnormal
+//      below); the product is exact for every E, subnormal results included.
+// Only the prmt runs on the integer ALU pipe - the pipe the dequantisers saturate first; the other
+// four operations go to the FMA pipe.
+__device__ __forceinline__ uint32_t dequant_pair(uint32_t u, uint32_t selector, uint32_t scale2) {
+    const uint32_t h2 = __byte_perm(u, 0x64646464u, selector);
+    uint32_t t, b, d, r;
+    asm("add.rn.f16x2 %0, %1, %2;" : "=r"(t) : "r"(h2), "r"(0xE400E400u));          // - 1024
+    asm("mad.hi.u32 %0, %1, %2, %3;" : "=r"(b) : "r"(t), "r"(0x20000000u), "r"(0x38003800u));
+    asm("add.rn.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(b), "r"(0xC300C300u));          // - 128
+    asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(d), "r"(scale2));
     return r;
 }
 
-// bf16x2 of (m0, m1) * scale for bytes `sel0`, `sel0 + 1` of the biased word u.
-__device__ __forceinline__ uint32_t dequant_pair(uint32_t u, uint32_t sel0, uint64_t neg_magic2, uint64_t scale2) {
-    const uint32_t x0 = __byte_perm(u, 0x4B000000u, 0x7650u + sel0);
-    const uint32_t x1 = __byte_perm(u, 0x4B000000u, 0x7651u + sel0);
-    uint64_t d, r;
-    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(pack_f32x2(x0, x1)), "l"(neg_magic2));
-    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(d), "l"(scale2));
-    uint32_t f0, f1;
-    asm("mov.b64 {%0, %1}, %2;" : "=r"(f0), "=r"(f1) : "l"(r));
-    return __byte_perm(f0, f1, 0x7632);
+// Table entry for exponent E: 2^(E-133) as bf16, in both halves of the word.
+__device__ __forceinline__ uint32_t scale_table_entry(uint32_t E) {
+    const uint32_t bits = (E >= 7u) ? ((E - 6u) << 7) : (1u << E);
+    return E == 255u ? 0u : bits * 0x10001u;
 }
 
 template <class C>
@@ -178,7 +182,6 @@ __device__ __forceinline__ void dequant_slab(uint32_t raw_mant, uint32_t raw_exp
             e[i] = e2;
         }
     }
-    const uint64_t neg_magic2 = pack_f32x2(0xCB000080u, 0xCB000080u);    // -(2^23 + 128), twice
 #pragma unroll
     for (int i = 0; i < C::DQ_ITERS; ++i) {
         const int r = r0 + i * C::ROWS_PER_ITER;
@@ -186,19 +189,18 @@ __device__ __forceinline__ void dequant_slab(uint32_t raw_mant, uint32_t raw_exp
             uint32_t s0, s1;
             asm volatile("ld.shared.b32 %0, [%1];" : "=r"(s0) : "r"(scale_lut + (e[i] & 0xFFu) * 4));
             asm volatile("ld.shared.b32 %0, [%1];" : "=r"(s1) : "r"(scale_lut + (e[i] >> 8) * 4));
-            const uint64_t sc0 = pack_f32x2(s0, s0), sc1 = pack_f32x2(s1, s1);
             const uint32_t u0 = w[i].x ^ 0x80808080u, u1 = w[i].y ^ 0x80808080u;
             const uint32_t u2 = w[i].z ^ 0x80808080u, u3 = w[i].w ^ 0x80808080u;
             const int rr = row_base + r;
             const uint32_t row_addr = dst_base + (rr >> 7) * C::GROUP_BYTES + (kb >> 3) * C::KHALF_BYTES + (rr & 127) * 128;
             const uint32_t sw = static_cast<uint32_t>(rr & 7);
             asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row_addr + ((((kb & 7)) ^ sw) << 4)),
-                         "r"(dequant_pair(u0, 0, neg_magic2, sc0)), "r"(dequant_pair(u0, 2, neg_magic2, sc0)),
-                         "r"(dequant_pair(u1, 0, neg_magic2, sc0)), "r"(dequant_pair(u1, 2, neg_magic2, sc0))
+                         "r"(dequant_pair(u0, 0x4140u, s0)), "r"(dequant_pair(u0, 0x4342u, s0)),
+                         "r"(dequant_pair(u1, 0x4140u, s0)), "r"(dequant_pair(u1, 0x4342u, s0))
                          : "memory");
             asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row_addr + ((((kb & 7) + 1) ^ sw) << 4)),
-                         "r"(dequant_pair(u2, 0, neg_magic2, sc1)), "r"(dequant_pair(u2, 2, neg_magic2, sc1)),
-                         "r"(dequant_pair(u3, 0, neg_magic2, sc1)), "r"(dequant_pair(u3, 2, neg_magic2, sc1))
+                         "r"(dequant_pair(u2, 0x4140u, s1)), "r"(dequant_pair(u2, 0x4342u, s1)),
+                         "r"(dequant_pair(u3, 0x4140u, s1)), "r"(dequant_pair(u3, 0x4342u, s1))
                          : "memory");
         }
     }

@@ -106,8 +106,7 @@ atb_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_c
     }
     if (threadIdx.x >= kFirstDequantWarp * 32 && threadIdx.x < kFirstDequantWarp * 32 + 256) {
         const uint32_t E = threadIdx.x - kFirstDequantWarp * 32;
-        const uint32_t bits = (E >= 7u) ? ((E - 6u) << 23) : (1u << (E + 16u));
-        asm volatile("st.shared.b32 [%0], %1;" ::"r"(scale_lut + E * 4), "r"(E == 255u ? 0u : bits) : "memory");
+        asm volatile("st.shared.b32 [%0], %1;" ::"r"(scale_lut + E * 4), "r"(scale_table_entry(E)) : "memory");
     }
     tcgen05_fence_before_sync();
     __syncthreads();
