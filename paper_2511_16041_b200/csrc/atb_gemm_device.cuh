@@ -59,6 +59,11 @@ struct Ring {
     __device__ __forceinline__ void advance(int n) {
         if (++stage == n) { stage = 0; phase ^= 1u; }
     }
+    // `step` stages at once; n is a multiple of step and stage stays congruent modulo step
+    __device__ __forceinline__ void advance_by(int step, int n) {
+        stage += step;
+        if (stage >= n) { stage -= n; phase ^= 1u; }
+    }
 };
 
 struct Ctx {

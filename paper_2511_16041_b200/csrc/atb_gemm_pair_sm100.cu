@@ -242,31 +242,27 @@ atb_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_c
         // ================================ dequantisers ================================
         const int t = (threadIdx.x - kFirstDequantWarp * 32) % C::GROUP_THREADS;
         const int my_group = (threadIdx.x - kFirstDequantWarp * 32) / C::GROUP_THREADS;
+        // slabs arrive in ring order: a group takes every DQ_GROUPS-th slab of this CTA's stream
+        int64_t my_slabs = 0;
+        for (int tile = cluster_id; tile < total_tiles; tile += n_clusters) my_slabs += static_cast<int64_t>(p.k_steps) * C::SLABS;
         Ring rr, rd;
-        for (int i = 0; i < my_group; ++i) { rr.advance(p.n_raw_stages); rd.advance(n_deq_stages); }
-        int turn = 0;
-        bool ok = true;
-        for (int tile = cluster_id; ok && tile < total_tiles; tile += n_clusters) {
-            for (int k = 0; ok && k < p.k_steps; ++k) {
-                for (int s = 0; s < C::SLABS; ++s) {
-                    const bool mine = (turn == my_group);
-                    if (++turn == C::DQ_GROUPS) turn = 0;
-                    if (!mine) continue;
-                    if (!(ok = wait_bar_cl(cx, raw_full + 8 * rr.stage, rr.phase, 0x301))) break;
-                    if (!(ok = wait_bar_cl(cx, deq_empty + 8 * rd.stage, rd.phase ^ 1u, 0x302))) break;
-                    const uint32_t raw = raw_base + rr.stage * C::RAW_BYTES;
-                    const uint32_t dst_base = deq_base + (rd.stage / C::SLABS) * C::GROUP_BYTES;
-                    const int row_base = (rd.stage % C::SLABS) * SLAB_ROWS;
-                    dequant_slab<C>(raw, raw + C::RAW_MANT_BYTES, scale_lut, dst_base, row_base, t, SLAB_ROWS);
-                    fence_proxy_async_smem();
-                    __syncwarp();
-                    if (lane == 0) {
-                        mbar_arrive_cluster(mapa_shared(deq_full + 8 * rd.stage, 0));
-                        mbar_arrive(raw_empty + 8 * rr.stage);
-                    }
-                    for (int i = 0; i < C::DQ_GROUPS; ++i) { rr.advance(p.n_raw_stages); rd.advance(n_deq_stages); }
-                }
+        rr.stage = my_group;
+        rd.stage = my_group;
+        for (int64_t n = my_group; n < my_slabs; n += C::DQ_GROUPS) {
+            if (!wait_bar_cl(cx, raw_full + 8 * rr.stage, rr.phase, 0x301)) break;
+            if (!wait_bar_cl(cx, deq_empty + 8 * rd.stage, rd.phase ^ 1u, 0x302)) break;
+            const uint32_t raw = raw_base + rr.stage * C::RAW_BYTES;
+            const uint32_t dst_base = deq_base + (rd.stage / C::SLABS) * C::GROUP_BYTES;
+            const int row_base = (rd.stage % C::SLABS) * SLAB_ROWS;
+            dequant_slab<C>(raw, raw + C::RAW_MANT_BYTES, scale_lut, dst_base, row_base, t, SLAB_ROWS);
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+                mbar_arrive_cluster(mapa_shared(deq_full + 8 * rd.stage, 0));
+                mbar_arrive(raw_empty + 8 * rr.stage);
             }
+            rr.advance_by(C::DQ_GROUPS, p.n_raw_stages);
+            rd.advance_by(C::DQ_GROUPS, n_deq_stages);
         }
     }
 

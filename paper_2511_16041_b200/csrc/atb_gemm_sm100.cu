@@ -104,8 +104,7 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
     }
     if (threadIdx.x >= kFirstDequantWarp * 32 && threadIdx.x < kFirstDequantWarp * 32 + 256) {
         const uint32_t E = threadIdx.x - kFirstDequantWarp * 32;
-        const uint32_t bits = (E >= 7u) ? ((E - 6u) << 23) : (1u << (E + 16u));
-        asm volatile("st.shared.b32 [%0], %1;" ::"r"(scale_lut + E * 4), "r"(E == 255u ? 0u : bits) : "memory");
+        asm volatile("st.shared.b32 [%0], %1;" ::"r"(scale_lut + E * 4), "r"(scale_table_entry(E)) : "memory");
     }
     tcgen05_fence_before_sync();
     __syncthreads();
@@ -280,39 +279,38 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
         // ================================ dequantisers ================================
         const int t = (threadIdx.x - kFirstDequantWarp * 32) % C::GROUP_THREADS;
         const int my_group = (threadIdx.x - kFirstDequantWarp * 32) / C::GROUP_THREADS;
-        Ring rr, rd;
-        for (int i = 0; i < my_group; ++i) { rr.advance(p.n_raw_stages); rd.advance(n_deq_stages); }
-        int turn = 0;                                   // slab sequence number modulo the group count
-        bool ok = true;
-        for (int item = blockIdx.x; ok && item < total_items; item += gridDim.x) {
+        // The dequantisers do not need to know tiles or K-steps: slabs arrive in ring order, so a
+        // group just takes every DQ_GROUPS-th slab of this CTA's stream.
+        int64_t my_slabs = 0;
+        for (int item = blockIdx.x; item < total_items; item += gridDim.x) {
             const WorkItem w = work_item<SPLIT>(item, p);
-            for (int k = w.k_begin; ok && k < w.k_end; ++k) {
-                for (int s = 0; s < C::RHO; ++s) {
-                    const bool mine = (turn == my_group);
-                    if (++turn == C::DQ_GROUPS) turn = 0;
-                    if (!mine) continue;
-                    if (!(ok = wait_bar(cx, raw_full + 8 * rr.stage, rr.phase, 0x301))) break;
-                    if (!(ok = wait_bar(cx, deq_empty + 8 * rd.stage, rd.phase ^ 1u, 0x302))) break;
-                    const uint32_t raw = raw_base + rr.stage * C::RAW_BYTES;
-                    uint32_t dst_base;
-                    int row_base;
-                    if (T_MA <= 128) {
-                        dst_base = deq_base + (rd.stage / C::SPG) * C::GROUP_BYTES;
-                        row_base = (rd.stage % C::SPG) * T_MA;
-                    } else {
-                        dst_base = deq_base + rd.stage * C::GPS * C::GROUP_BYTES;
-                        row_base = 0;
-                    }
-                    dequant_slab<C>(raw, raw + C::RAW_MANT_BYTES, scale_lut, dst_base, row_base, t, T_MA);
-                    fence_proxy_async_smem();
-                    __syncwarp();
-                    if (lane == 0) {
-                        mbar_arrive(deq_full + 8 * rd.stage);
-                        mbar_arrive(raw_empty + 8 * rr.stage);
-                    }
-                    for (int i = 0; i < C::DQ_GROUPS; ++i) { rr.advance(p.n_raw_stages); rd.advance(n_deq_stages); }
-                }
+            my_slabs += static_cast<int64_t>(w.k_end - w.k_begin) * C::RHO;
+        }
+        Ring rr, rd;
+        rr.stage = my_group;
+        rd.stage = my_group;
+        for (int64_t n = my_group; n < my_slabs; n += C::DQ_GROUPS) {
+            if (!wait_bar(cx, raw_full + 8 * rr.stage, rr.phase, 0x301)) break;
+            if (!wait_bar(cx, deq_empty + 8 * rd.stage, rd.phase ^ 1u, 0x302)) break;
+            const uint32_t raw = raw_base + rr.stage * C::RAW_BYTES;
+            uint32_t dst_base;
+            int row_base;
+            if (T_MA <= 128) {
+                dst_base = deq_base + (rd.stage / C::SPG) * C::GROUP_BYTES;
+                row_base = (rd.stage % C::SPG) * T_MA;
+            } else {
+                dst_base = deq_base + rd.stage * C::GPS * C::GROUP_BYTES;
+                row_base = 0;
             }
+            dequant_slab<C>(raw, raw + C::RAW_MANT_BYTES, scale_lut, dst_base, row_base, t, T_MA);
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+                mbar_arrive(deq_full + 8 * rd.stage);
+                mbar_arrive(raw_empty + 8 * rr.stage);
+            }
+            rr.advance_by(C::DQ_GROUPS, p.n_raw_stages);
+            rd.advance_by(C::DQ_GROUPS, n_deq_stages);
         }
     }
 
