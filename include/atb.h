@@ -77,7 +77,8 @@ atb_status_t atb_quantize_bfp16(const float* A_dev, int64_t M, int64_t K, int64_
  *   A_mant_dev, A_exp_dev: the planes described above (16-byte aligned);
  *   B_bf16_dev: bf16 B[K][ldb] row-major, ldb >= N, ldb % 8 == 0, 16-byte aligned;
  *   C_bf16_dev: bf16 C[M][ldc] row-major, ldc >= N, ldc % 8 == 0, 16-byte aligned (written).
- * Shapes: M, N >= 1 (any value; edge tiles are handled), N % 8 == 0, K >= 64 and K % 64 == 0.
+ * Shapes: M >= 1 (any value), N >= 8 with N % 8 == 0, K >= 16 with K % 16 == 0.  Edge tiles in M, N and
+ *         K are handled (TMA zero-fills loads past the edge and clips stores).
  * Tilings: T_MC in {128, 256}; T_N in {64, 128, 256, 512}; T_K in {64, 128};
  *          T_MA in {32, 64, 128, 256} with T_MA <= T_MC; (T_MC / 128) * T_N <= 512 (the FP32
  *          accumulator must fit the 512 TMEM columns); the shared-memory rings must fit 227 KB.
@@ -95,7 +96,7 @@ atb_status_t atb_gemm(int64_t M, int64_t N, int64_t K, int T_MA, int T_MC, int T
  * stream.  The paper's hardware cannot do this - Section 2.2: an AIE core has no way to bring partial
  * sums back, so every output tile is fully accumulated in L1 - here partial sums go through L2/HBM.
  * Same operands and rules as atb_gemm.  Tilings: T_K = 64, T_MC in {128, 256}, T_N in {128, 256},
- * T_MA in {64, 128}.  splits in [1, min(64, K / T_K)].
+ * T_MA in {64, 128}.  splits in [1, min(64, ceil(K / T_K))].
  *   workspace_dev: device memory, 16-byte aligned, at least atb_gemm_splitk_workspace_bytes() bytes;
  *                  fully overwritten; may be reused by the next call on the same stream.
  * Errors: as atb_gemm, plus ATB_ERR_BUFFER_TOO_SMALL. */

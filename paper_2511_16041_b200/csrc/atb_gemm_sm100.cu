@@ -530,8 +530,8 @@ extern "C" atb_status_t atb_gemm(int64_t M, int64_t N, int64_t K, int T_MA, int 
     atb::clear_error();
     if (!A_mant_dev || !A_exp_dev || !B_bf16_dev || !C_bf16_dev)
         return atb::fail(ATB_ERR_NULL_POINTER, "A_mant_dev, A_exp_dev, B_bf16_dev and C_bf16_dev must be non-NULL");
-    if (M < 1 || N < 1 || K < 64 || K % 64 != 0 || N % 8 != 0)
-        return atb::fail(ATB_ERR_BAD_SHAPE, "need M >= 1, N >= 8 with N %% 8 == 0, K >= 64 with K %% 64 == 0 (got %lld, %lld, %lld)",
+    if (M < 1 || N < 1 || K < 16 || K % 16 != 0 || N % 8 != 0)
+        return atb::fail(ATB_ERR_BAD_SHAPE, "need M >= 1, N >= 8 with N %% 8 == 0, K >= 16 with K %% 16 == 0 (got %lld, %lld, %lld)",
                          (long long)M, (long long)N, (long long)K);
     if (M > (1ll << 30) || N > (1ll << 30) || K > (1ll << 30))
         return atb::fail(ATB_ERR_BAD_SHAPE, "dimensions above 2^30 are not supported");
@@ -600,12 +600,12 @@ bool splitk_tiling_ok(int T_MA, int T_MC, int T_K, int T_N) {
 }
 
 atb_status_t splitk_validate(int64_t M, int64_t N, int64_t K, int T_MA, int T_MC, int T_K, int T_N, int splits) {
-    if (M < 1 || N < 8 || N % 8 != 0 || K < 64 || K % 64 != 0 || M > (1ll << 30) || N > (1ll << 30) || K > (1ll << 30))
-        return atb::fail(ATB_ERR_BAD_SHAPE, "need M >= 1, N %% 8 == 0, K %% 64 == 0 (got %lld, %lld, %lld)", (long long)M, (long long)N, (long long)K);
+    if (M < 1 || N < 8 || N % 8 != 0 || K < 16 || K % 16 != 0 || M > (1ll << 30) || N > (1ll << 30) || K > (1ll << 30))
+        return atb::fail(ATB_ERR_BAD_SHAPE, "need M >= 1, N %% 8 == 0, K %% 16 == 0 (got %lld, %lld, %lld)", (long long)M, (long long)N, (long long)K);
     if (!splitk_tiling_ok(T_MA, T_MC, T_K, T_N))
         return atb::fail(ATB_ERR_BAD_TILING, "split-K supports T_K = 64, T_MC in {128, 256}, T_N in {128, 256}, T_MA in {64, 128}");
-    if (splits < 1 || splits > 64 || splits > K / T_K)
-        return atb::fail(ATB_ERR_BAD_SHAPE, "splits=%d must be in [1, min(64, K / T_K)]", splits);
+    if (splits < 1 || splits > 64 || splits > atb::ceil_div(K, T_K))
+        return atb::fail(ATB_ERR_BAD_SHAPE, "splits=%d must be in [1, min(64, ceil(K / T_K))]", splits);
     return ATB_OK;
 }
 

@@ -152,7 +152,7 @@ def test_leading_dimensions_and_untouched_padding():
 
 
 def test_tiny_and_degenerate_shapes():
-    for (M, N, K) in [(1, 8, 64), (7, 24, 64), (129, 72, 192)]:
+    for (M, N, K) in [(1, 8, 64), (7, 24, 64), (129, 72, 192), (5, 16, 16), (130, 264, 80), (300, 40, 464)]:
         A = inputs.make_A("normal", M, K)
         Bb = inputs.make_B_bits(K, N)
         mant, exp = oracle.quantize_bfp16(A)
@@ -175,7 +175,7 @@ def test_argument_errors():
 
     assert call() == 0
     assert call(a=None) == 1
-    assert call(K=100) == 2 and call(N=12) == 2 and call(M=0) == 2 and call(ldb=N - 8) == 2
+    assert call(K=100) == 2 and call(K=72) == 2 and call(N=12) == 2 and call(M=0) == 2 and call(ldb=N - 8) == 2
     assert call(til=(64, 128, 64, 96)) == 3          # unsupported T_N
     assert call(til=(256, 128, 64, 128)) == 3        # T_MA > T_MC
     assert call(til=(128, 256, 128, 256)) == 3       # shared-memory rings do not fit

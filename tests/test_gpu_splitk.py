@@ -23,6 +23,7 @@ def _operands(M, N, K, kind="normal"):
     ((300, 264, 1536), (64, 128, 64, 128), 3),          # ragged M and N, splits not a power of two
     ((1024, 1024, 4096), (128, 256, 64, 256), 8),
     ((129, 136, 448), (128, 128, 64, 256), 7),           # one K-step per split
+    ((200, 136, 400), (64, 128, 64, 128), 7),            # K not a multiple of 64: a ragged last K-step
     ((512, 512, 512), (64, 256, 64, 128), 1),
 ])
 def test_splitk_against_oracle(shape, tiling, splits):
