@@ -232,30 +232,55 @@ def run_ours(args):
 
     tiling_used = []
 
-    def step(ev=None):
+    def step(ev=None, A_d=None, B_d=None, C_d=None, on=None):
         """Whole hot path on device-resident input: quantise -> select tiling -> GEMM."""
-        atb.atb_quantize_bfp16(A_dev, mant, plane, stream=stream)
+        A_d = A_dev if A_d is None else A_d
+        B_d = B_dev if B_d is None else B_d
+        C_d = C_dev if C_d is None else C_d
+        on = stream if on is None else on
+        atb.atb_quantize_bfp16(A_d, mant, plane, stream=on)
         if args.tiling:
             t = tuple(args.tiling)
         else:
             t, _ = atb.atb_select_tiling(M, N, K, max_scores=1)
         if ev is not None:
-            ev[0].record(stream)
-        atb.atb_gemm(M, N, K, *t, mant, plane, B_dev, C_dev, stream=stream)
+            ev[0].record(on)
+        atb.atb_gemm(M, N, K, *t, mant, plane, B_d, C_d, stream=on)
         if ev is not None:
-            ev[1].record(stream)
+            ev[1].record(on)
         if not tiling_used:
             tiling_used.append(tuple(t))
 
-    def step_e2e():
-        """Same, from pinned host buffers and back to the host."""
-        with torch.cuda.stream(stream):
-            A_dev.copy_(A_host, non_blocking=True)
-            B_dev.view(torch.int16).copy_(B_host, non_blocking=True)
-        step()
-        with torch.cuda.stream(stream):
-            C_host.copy_(C_dev.view(torch.int16), non_blocking=True)
-        stream.synchronize()
+    # End-to-end leg: every step copies its A and B from pinned host memory and its C back.  Two sets
+    # of device buffers and three streams let step i+1's upload and step i-1's download overlap step
+    # i's kernels (PCIe is full duplex); every step still pays all three transfers.
+    e2e_sets = []
+
+    def e2e_setup():
+        for _ in range(2):
+            e2e_sets.append(dict(
+                A=torch.empty_like(A_dev), B=torch.empty_like(B_dev), C=torch.empty_like(C_dev),
+                C_host=torch.empty((M, N), dtype=torch.int16).pin_memory(),
+                up=torch.cuda.Event(), done=torch.cuda.Event(), down=torch.cuda.Event()))
+        return torch.cuda.Stream(dev), torch.cuda.Stream(dev)
+
+    def run_e2e(n_steps, s_up, s_down):
+        for i in range(n_steps):
+            b = e2e_sets[i % 2]
+            s_up.wait_event(b["done"])                 # the kernels that read this set two steps ago
+            with torch.cuda.stream(s_up):
+                b["A"].copy_(A_host, non_blocking=True)
+                b["B"].view(torch.int16).copy_(B_host, non_blocking=True)
+                b["up"].record(s_up)
+            stream.wait_event(b["up"])
+            stream.wait_event(b["down"])               # C of this set has been read back
+            step(A_d=b["A"], B_d=b["B"], C_d=b["C"])
+            b["done"].record(stream)
+            s_down.wait_event(b["done"])
+            with torch.cuda.stream(s_down):
+                b["C_host"].copy_(b["C"].view(torch.int16), non_blocking=True)
+                b["down"].record(s_down)
+        s_up.synchronize(); stream.synchronize(); s_down.synchronize()
 
     # ---------------- device-resident timing ----------------
     for _ in range(max(args.warmup, 3)):
@@ -279,18 +304,18 @@ def run_ours(args):
     gemm_ms = sum(a.elapsed_time(b) for a, b in gemm_events) / args.steps
 
     # ---------------- end-to-end timing (host buffers) ----------------
-    e2e_steps = max(2, min(args.steps, 5))
-    step_e2e()
+    e2e_steps = max(4, min(args.steps, 10))
+    s_up, s_down = e2e_setup()
+    run_e2e(2, s_up, s_down)
     barrier()
     t0 = time.perf_counter()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(stream)
-    for _ in range(e2e_steps):
-        step_e2e()
-    e1.record(stream)
-    stream.synchronize()
+    run_e2e(e2e_steps, s_up, s_down)
+    torch.cuda.synchronize()
+    e2e_wall_ms = 1e3 * (time.perf_counter() - t0)
     barrier()
-    e2e_ms = max(e0.elapsed_time(e1), 1e3 * (time.perf_counter() - t0)) / e2e_steps
+    e2e_ms = e2e_wall_ms / e2e_steps
+    e2e_check = e2e_sets[(e2e_steps - 1) % 2]["C_host"]
+    assert bool((e2e_check == C_dev.view(torch.int16).cpu()).all()), "end-to-end result differs from the resident run"
 
     # ---------------- quantiser alone (HBM roofline) ----------------
     q0, q1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -325,7 +350,8 @@ def run_ours(args):
             "clocks": clocks,
             "e2e": {"value": aggregate_tflops(flops, world, e2e_ms), "unit": "TFLOPS",
                     "h2d_bytes_per_step": A_host.numel() * 4 + B_host.numel() * 2,
-                    "d2h_bytes_per_step": C_host.numel() * 2, "ms_per_step": e2e_ms},
+                    "d2h_bytes_per_step": C_host.numel() * 2, "ms_per_step": e2e_ms, "steps": e2e_steps,
+                    "how": "wall clock over pipelined steps: upload, kernels and download of neighbouring steps overlap on three streams"},
             "gpu_launches": 2 * args.steps,
             "roofline": {"bound": "tensor", "kernel": "atb_gemm_kernel", "achieved": achieved,
                          "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"],
