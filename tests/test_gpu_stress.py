@@ -1,0 +1,71 @@
+"""Randomised parity and run-to-run determinism of the GEMM kernels.
+
+A data race between the kernel's roles (TMA producer, dequantisers, UMMA issuer, epilogue) would
+show up as a run-to-run difference or as a tolerance failure on some shape; both are checked here.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2511_16041_b200 as atb
+from paper_2511_16041_b200 import inputs
+from tests.gpu_util import dev, planes_to_dev, bf16_bits_to_dev, bf16_dev_to_bits
+
+pytestmark = pytest.mark.gpu
+
+
+def _all_tilings():
+    return [(ma, mc, k, n) for mc in (128, 256) for n in (64, 128, 256, 512) for k in (64, 128)
+            for ma in (32, 64, 128, 256) if ma <= mc and atb.atb_tiling_supported(ma, mc, k, n)]
+
+
+def test_random_shapes_and_tilings_against_oracle():
+    rng = np.random.default_rng(20251116)
+    tilings = _all_tilings()
+    kinds = ["normal", "laplace", "outlier"]
+    for case in range(40):
+        M = int(rng.integers(1, 1400))
+        N = int(rng.integers(1, 130)) * 8
+        K = int(rng.integers(1, 100)) * 16
+        t = tilings[int(rng.integers(0, len(tilings)))]
+        A = inputs.make_A(kinds[case % 3], M, K, inputs.BASE_SEED + case)
+        Bb = inputs.make_B_bits(K, N, 1.0, inputs.BASE_SEED + case)
+        mant, exp = oracle.quantize_bfp16(A)
+        md, ed = planes_to_dev(mant, exp)
+        Bd = bf16_bits_to_dev(Bb)
+        C = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device=dev())
+        atb.atb_gemm(M, N, K, *t, md, ed, Bd, C)
+        atb.atb_device_status()
+        Cr, S = oracle.gemm(mant, exp, Bb)
+        bad, ratio = oracle.check_tolerance(bf16_dev_to_bits(C), Cr, S)
+        assert bad == 0 and ratio < 0.75, (case, (M, N, K), t, bad, ratio)
+
+
+@pytest.mark.parametrize("tiling", [(128, 256, 64, 256), (64, 256, 64, 256), (32, 128, 64, 128), (128, 256, 64, 512),
+                                     (64, 256, 128, 128)])
+def test_run_to_run_bitwise_determinism(tiling):
+    """Many tiles per CTA and many K-steps: ring phases wrap often; five runs must agree bit for bit."""
+    M, N, K = 4096, 2048, 4096
+    g = torch.Generator(device=dev())
+    g.manual_seed(7)
+    mant = torch.randint(-127, 128, (M, K), dtype=torch.int8, device=dev(), generator=g)
+    plane = torch.randint(120, 135, (atb.atb_bfp16_exp_bytes(M, K),), dtype=torch.uint8, device=dev(), generator=g)
+    B = torch.randn((K, N), device=dev(), generator=g).to(torch.bfloat16)
+    ref = None
+    for run in range(5):
+        C = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device=dev())
+        atb.atb_gemm(M, N, K, *tiling, mant, plane, B, C)
+        atb.atb_device_status()
+        assert bool(torch.isfinite(C.float()).all())
+        if ref is None:
+            ref = C.view(torch.int16).clone()
+        assert torch.equal(C.view(torch.int16), ref), (tiling, run)
+    # and a sampled comparison against the oracle on this large case
+    rows = np.unique(np.random.default_rng(3).integers(0, M, 24)).astype(np.int64)
+    mant_h = mant[torch.from_numpy(rows).to(dev())].cpu().numpy()
+    exp_h = atb.exp_plane_to_logical(plane.cpu().numpy(), M, K)[rows]
+    Cr, S = oracle.gemm(mant_h, exp_h, bf16_dev_to_bits(B))
+    got = bf16_dev_to_bits(ref.view(torch.bfloat16)[torch.from_numpy(rows).to(dev())])
+    bad, ratio = oracle.check_tolerance(got, Cr, S)
+    assert bad == 0 and ratio < 0.75, (tiling, bad, ratio)
