@@ -18,7 +18,8 @@ namespace {
 using namespace sm100;
 
 constexpr int kDequantWarps = 16;
-constexpr int kThreads = (6 + kDequantWarps) * 32;
+constexpr int kThreads = (7 + kDequantWarps) * 32;      // + B producer, UMMA issuer, 4 epilogue warps, A producer
+constexpr int kAProducerWarp = 6 + kDequantWarps;       // the last warp
 // The dequantiser warps work in groups; slabs are dealt to the groups in turn, so that several
 // slabs are in flight and every thread has a few 16-element slots per barrier round trip.
 // Ring depths are multiples of the group count: a ring stage is then always served by the same
@@ -78,7 +79,7 @@ struct Ctx {
 // dequantisers.  kCluster = true uses cluster-scope acquire (arrivals may come from the peer CTA).
 constexpr uint32_t kSuspendNs = 20000;
 template <bool kSpin, bool kCluster>
-__device__ __forceinline__ bool wait_bar_t(const Ctx& cx, uint32_t bar, uint32_t parity, unsigned code) {
+__device__ __forceinline__ bool wait_bar_impl(const Ctx& cx, uint32_t bar, uint32_t parity, unsigned code) {
     auto probe = [&]() { return kCluster ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity); };
     auto probe_suspend = [&]() {
         return kCluster ? mbar_try_wait_cluster_suspend(bar, parity, kSuspendNs) : mbar_try_wait_suspend(bar, parity, kSuspendNs);
@@ -97,6 +98,33 @@ __device__ __forceinline__ bool wait_bar_t(const Ctx& cx, uint32_t bar, uint32_t
             }
         }
     }
+}
+#ifdef ATB_PROFILE
+// Opt-in diagnostic build (-DATB_PROFILE): cycles spent in each kind of wait, one row per CTA, one
+// lane per warp reporting.  Slot = (role << 2 | barrier kind) taken from the wait's code.
+__device__ unsigned long long g_wait_cycles[256][16];
+// Host: sums the counters of this translation unit's kernels over the CTAs into out16, then clears them.
+inline int read_wait_cycles(unsigned long long* out16) {
+    static unsigned long long host[256][16];
+    if (cudaDeviceSynchronize() != cudaSuccess) return 1;
+    if (cudaMemcpyFromSymbol(host, g_wait_cycles, sizeof host) != cudaSuccess) return 1;
+    for (int j = 0; j < 16; ++j) { out16[j] = 0; for (int i = 0; i < 256; ++i) out16[j] += host[i][j]; }
+    for (auto& row : host) for (auto& v : row) v = 0;
+    return cudaMemcpyToSymbol(g_wait_cycles, host, sizeof host) == cudaSuccess ? 0 : 1;
+}
+#endif
+template <bool kSpin, bool kCluster>
+__device__ __forceinline__ bool wait_bar_t(const Ctx& cx, uint32_t bar, uint32_t parity, unsigned code) {
+#ifdef ATB_PROFILE
+    const long long t0 = clock64();
+    const bool ok = wait_bar_impl<kSpin, kCluster>(cx, bar, parity, code);
+    if ((threadIdx.x & 31) == 0 || kSpin)
+        atomicAdd(&g_wait_cycles[blockIdx.x & 255][((code >> 8) << 2 | (code & 3)) & 15],
+                  static_cast<unsigned long long>(clock64() - t0));
+    return ok;
+#else
+    return wait_bar_impl<kSpin, kCluster>(cx, bar, parity, code);
+#endif
 }
 __device__ __forceinline__ bool wait_bar(const Ctx& cx, uint32_t bar, uint32_t parity, unsigned code) {
     return wait_bar_t<false, false>(cx, bar, parity, code);

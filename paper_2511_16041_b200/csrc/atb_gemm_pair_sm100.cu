@@ -14,8 +14,8 @@
 // collect arrivals from both CTAs; stage-free barriers are signalled in both CTAs at once by
 // tcgen05.commit with a CTA mask.  No TMA load uses multicast.
 //
-// Warp roles are those of the single-CTA kernel: 0 TMA producer, 1 UMMA issuer (active in the
-// leader only) + TMEM owner, 2-5 epilogue, 6-21 dequantisers (4 groups of 4 warps).
+// Warp roles are those of the single-CTA kernel: 0 TMA producer of B, 1 UMMA issuer (active in the
+// leader only) + TMEM owner, 2-5 epilogue, 6-21 dequantisers (4 groups of 4 warps), 22 TMA producer of A.
 #include "atb_gemm_device.cuh"
 
 namespace {
@@ -118,14 +118,13 @@ atb_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_c
     const int cluster_id = blockIdx.x >> 1, n_clusters = gridDim.x >> 1;
 
     if (warp == 0) {
-        // ================================ TMA producer ================================
+        // ================================ TMA producer: B half-tiles ===================
         if (elect_one()) {
-            Ring rb, rr;
+            Ring rb;
             bool ok = true;
             for (int tile = cluster_id; ok && tile < total_tiles; tile += n_clusters) {
                 int mt, nt;
                 tile_coords(tile, p.m_tiles, p.n_tiles, mt, nt);
-                const int row0 = mt * 256 + static_cast<int>(rank) * 128;
                 const int colb = nt * 512 + static_cast<int>(rank) * 128;
                 for (int k = 0; ok && k < p.k_steps; ++k) {
                     if (!(ok = wait_bar_cl_spin(cx, b_empty + 8 * rb.stage, rb.phase ^ 1u, 0x001))) break;
@@ -137,6 +136,19 @@ atb_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_c
                         tma_load_2d_pair(b_base + rb.stage * C::B_BYTES + j * C::B_BOX_BYTES, &tm_b,
                                          colb + (j >> 1) * 256 + (j & 1) * 64, k * C::T_K, fb);
                     rb.advance(p.n_b_stages);
+                }
+            }
+        }
+    } else if (warp == kAProducerWarp) {
+        // ================================ TMA producer: raw A slabs ====================
+        if (elect_one()) {
+            Ring rr;
+            bool ok = true;
+            for (int tile = cluster_id; ok && tile < total_tiles; tile += n_clusters) {
+                int mt, nt;
+                tile_coords(tile, p.m_tiles, p.n_tiles, mt, nt);
+                const int row0 = mt * 256 + static_cast<int>(rank) * 128;
+                for (int k = 0; ok && k < p.k_steps; ++k) {
                     for (int s = 0; s < C::SLABS; ++s) {
                         if (!(ok = wait_bar_cl_spin(cx, raw_empty + 8 * rr.stage, rr.phase ^ 1u, 0x002))) break;
                         const uint32_t fr = raw_full + 8 * rr.stage;
@@ -365,3 +377,8 @@ atb_status_t launch_gemm_pair(int T_MA, const GemmPlan& plan, int64_t M, int64_t
 }
 
 }  // namespace atb
+
+#ifdef ATB_PROFILE
+// Diagnostic build only: wait-cycle counters of the CTA-pair kernels (16 values), read and cleared.
+extern "C" int atb_debug_read_wait_cycles_pair(unsigned long long* out16) { return read_wait_cycles(out16); }
+#endif

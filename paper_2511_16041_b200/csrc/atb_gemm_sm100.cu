@@ -5,12 +5,15 @@
 // rho = T_MC / T_MA slabs of A are streamed through it; the FP32 accumulator of the whole
 // T_MC x T_N tile lives in tensor memory and is written out once, after K / T_K steps.
 //
-// Warp roles (704 threads):
-//   warp 0      TMA producer: B tiles and raw BFP16 A slabs (int8 mantissas + uint8 exponents)
+// Warp roles (736 threads):
+//   warp 0      TMA producer of B tiles
 //   warp 1      UMMA issuer (one elected lane) and owner of the TMEM allocation
 //   warps 2-5   epilogue: tcgen05.ld -> round to bf16 -> swizzled shared-memory box -> TMA store
-//   warps 6-21  dequantisers (two groups of 8 warps taking alternate slabs): raw slab -> bf16, K-major, 128-byte-swizzled operand in shared
-//               memory (exact: m * 2^(E-133) has at most 7 significant bits)
+//   warps 6-21  dequantisers, in 2 or 4 groups that take the slabs in turn: raw slab -> bf16,
+//               K-major, 128-byte-swizzled operand in shared memory (exact: m * 2^(E-133) has at
+//               most 7 significant bits)
+//   warp 22     TMA producer of raw BFP16 A slabs (int8 mantissas + uint8 exponents); a warp of its
+//               own, so that a full B ring never holds back the slabs the dequantisers wait for
 // Rings, all guarded by mbarriers with bounded waits:
 //   B tiles          (n_b_stages)    producer -> UMMA          (freed by tcgen05.commit)
 //   raw A slabs      (n_raw_stages)  producer -> dequantisers  (freed by the dequantisers)
@@ -114,13 +117,12 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
     const int total_items = p.m_tiles * p.n_tiles * (SPLIT ? p.splits : 1);
 
     if (warp == 0) {
-        // ================================ TMA producer ================================
+        // ================================ TMA producer: B tiles ========================
         if (elect_one()) {
-            Ring rb, rr;
+            Ring rb;
             bool ok = true;
             for (int item = blockIdx.x; ok && item < total_items; item += gridDim.x) {
                 const WorkItem w = work_item<SPLIT>(item, p);
-                const int mt = w.mt, nt = w.nt;
                 for (int k = w.k_begin; ok && k < w.k_end; ++k) {
                     if (!(ok = wait_bar_spin(cx, b_empty + 8 * rb.stage, rb.phase ^ 1u, 0x001))) break;
                     const uint32_t fb = b_full + 8 * rb.stage;
@@ -128,15 +130,28 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
 #pragma unroll
                     for (int j = 0; j < T_N / 64; ++j)
                         tma_load_2d(b_base + rb.stage * C::B_BYTES + j * C::B_BOX_BYTES, &tm_b,
-                                    nt * T_N + j * 64, k * T_K, fb);
+                                    w.nt * T_N + j * 64, k * T_K, fb);
                     rb.advance(p.n_b_stages);
+                }
+            }
+        }
+    } else if (warp == kAProducerWarp) {
+        // ================================ TMA producer: raw A slabs ====================
+        // A producer of its own: the raw slabs feed the dequantisers, which run ahead of the UMMAs,
+        // so these loads must not queue behind the wait for a free B stage.
+        if (elect_one()) {
+            Ring rr;
+            bool ok = true;
+            for (int item = blockIdx.x; ok && item < total_items; item += gridDim.x) {
+                const WorkItem w = work_item<SPLIT>(item, p);
+                for (int k = w.k_begin; ok && k < w.k_end; ++k) {
                     for (int s = 0; s < C::RHO; ++s) {
                         if (!(ok = wait_bar_spin(cx, raw_empty + 8 * rr.stage, rr.phase ^ 1u, 0x002))) break;
                         const uint32_t fr = raw_full + 8 * rr.stage;
                         const uint32_t dst = raw_base + rr.stage * C::RAW_BYTES;
                         mbar_arrive_expect_tx(fr, C::RAW_BYTES);
-                        tma_load_2d(dst, &tm_mant, k * T_K, mt * T_MC + s * T_MA, fr);
-                        tma_load_2d(dst + C::RAW_MANT_BYTES, &tm_exp, mt * T_MC + s * T_MA, k * (T_K / 64), fr);
+                        tma_load_2d(dst, &tm_mant, k * T_K, w.mt * T_MC + s * T_MA, fr);
+                        tma_load_2d(dst + C::RAW_MANT_BYTES, &tm_exp, w.mt * T_MC + s * T_MA, k * (T_K / 64), fr);
                         rr.advance(p.n_raw_stages);
                     }
                 }
@@ -749,3 +764,8 @@ extern "C" atb_status_t atb_gemm_splitk_noalloc(int64_t M, int64_t N, int64_t K,
     return atb::gemm_splitk_with_workspace(M, N, K, T_MA, T_MC, T_K, T_N, A_mant_dev, A_exp_dev, B_bf16_dev, ldb,
                                            C_bf16_dev, ldc, splits, scratch, stream);
 }
+
+#ifdef ATB_PROFILE
+// Diagnostic build only: wait-cycle counters of the single-CTA kernels (16 values), read and cleared.
+extern "C" int atb_debug_read_wait_cycles(unsigned long long* out16) { return read_wait_cycles(out16); }
+#endif
