@@ -22,8 +22,11 @@ constexpr int kThreads = (7 + kDequantWarps) * 32;      // + B producer, UMMA is
 constexpr int kAProducerWarp = 6 + kDequantWarps;       // the last warp
 // The dequantiser warps work in groups; slabs are dealt to the groups in turn, so that several
 // slabs are in flight and every thread has a few 16-element slots per barrier round trip.
-// Ring depths are multiples of the group count: a ring stage is then always served by the same
-// group, which keeps each mbarrier's phases strictly in order for its waiters.
+// An mbarrier wait only tells two consecutive phases apart, so every barrier must see its phases
+// completed and awaited strictly in order by ONE group.  A ring of n buffers served by d groups
+// therefore has lcm(n, d) barrier pairs: slab c lives in buffer c mod n and is guarded by barrier
+// c mod lcm(n, d), which is always the business of group c mod d.  Ring depths are then free of
+// the group count.
 __host__ __device__ constexpr int dq_groups(int T_MA, int T_K, int T_N) {
 #ifdef ATB_DQ_GROUPS
     return ATB_DQ_GROUPS;
@@ -35,15 +38,136 @@ __host__ __device__ constexpr int dq_groups(int T_MA, int T_K, int T_N) {
 constexpr int kFirstEpilogueWarp = 2;
 constexpr int kFirstDequantWarp = 6;
 constexpr int kMaxStages = 16;
+constexpr int kMaxRingBars = 32;
 constexpr uint32_t kEpilogueBoxBytes = 32 * 128;   // 32 rows x 64 bf16 columns
 constexpr uint32_t kSmemBudget = 232448;          // 227 KB of dynamic shared memory per CTA
 constexpr uint64_t kWaitTimeoutNs = 2000000000ull;  // every mbarrier wait gives up after 2 s
+
+// lcm(n, d) for d a power of two: the number of barrier pairs of a ring of n buffers and d groups
+constexpr int ring_bars(int n, int d) {
+    int g = d;
+    while (n % g) g >>= 1;
+    return n / g * d;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Ring plans: how the 227 KB of shared memory are split between the B ring, the raw-slab ring and
+// the ring of dequantised 128-row groups.  Evaluated at compile time (the kernels take the depths
+// as constants) and at run time (atb_tiling_plan, the tiling selection) from the same functions.
+// ---------------------------------------------------------------------------------------------
+struct RingPlan {
+    bool ok = false;
+    int nb = 2, ng = 2, nr = 1;      // B stages, dequantised 128-row groups, raw slabs
+    int dqg = 1;                     // dequantiser groups
+    int acc_bufs = 1, tmem_cols = 32;
+    uint32_t smem_bytes = 0;
+};
+
+constexpr uint32_t ring_smem_bytes(uint32_t b_bytes, uint32_t group_bytes, uint32_t raw_bytes, int acc_bars,
+                                   int dqg, int b, int g, int n_deq, int r) {
+    const uint32_t bars = 8u * (2 * b + 2 * ring_bars(r, dqg) + 2 * ring_bars(n_deq, dqg) + 2 * acc_bars) + 16u + 1024u;
+    return 1024u + b * b_bytes + g * group_bytes + r * raw_bytes + 1024u + 4u * kEpilogueBoxBytes + bars;
+}
+
+// Single-CTA kernel, tiling (T_MA, T_MC, T_K, T_N).
+constexpr RingPlan plan_single(int T_MA, int T_MC, int T_K, int T_N) {
+    RingPlan pl;
+    if (!(T_MC == 128 || T_MC == 256)) return pl;
+    if (!(T_N == 64 || T_N == 128 || T_N == 256 || T_N == 512)) return pl;
+    if (!(T_K == 64 || T_K == 128)) return pl;
+    if (!(T_MA == 32 || T_MA == 64 || T_MA == 128 || T_MA == 256) || T_MA > T_MC) return pl;
+    const int G = T_MC / 128;
+    if (G * T_N > 512) return pl;
+    const uint32_t b_bytes = T_K * T_N * 2, group_bytes = 128 * T_K * 2, raw_bytes = T_MA * T_K * 9 / 8;
+    const int gps = T_MA > 128 ? T_MA / 128 : 1;          // groups per slab
+    const int spg = T_MA < 128 ? 128 / T_MA : 1;          // slabs per group
+    const int dqg = dq_groups(T_MA, T_K, T_N);
+    pl.dqg = dqg;
+    pl.acc_bufs = (2 * G * T_N <= 512) ? 2 : 1;
+    int cols = 32;
+    while (cols < pl.acc_bufs * G * T_N) cols <<= 1;
+    pl.tmem_cols = cols;
+    // dequantised stages of a plan with g groups; the UMMA issuer takes spg of them at a time
+    const auto total = [=](int b, int g, int r) {
+        return ring_smem_bytes(b_bytes, group_bytes, raw_bytes, 2 * G, dqg, b, g, T_MA <= 128 ? g * spg : g / gps, r);
+    };
+    const auto bars_ok = [=](int g, int r) {
+        return ring_bars(r, dqg) <= kMaxRingBars && ring_bars(T_MA <= 128 ? g * spg : g / gps, dqg) <= kMaxRingBars;
+    };
+    // Any depth is legal (see ring_bars); the default plan gives every dequantiser group the same
+    // number of raw slabs and of dequantised stages, which measured best: one raw slab fewer than
+    // groups costs 10 %, one more gains nothing.
+    const int nr_step = dqg;
+    const int ng_step = T_MA <= 128 ? (dqg >= spg ? dqg / spg : 1) : dqg * gps;
+    int nb = 2, ng = ng_step < 2 ? 2 * ng_step : ng_step, nr = nr_step;
+    pl.nb = nb; pl.ng = ng; pl.nr = nr;
+    if (total(nb, ng, nr) > kSmemBudget) return pl;
+    // Grow the rings towards a target look-ahead, counted in 128-row x T_K operand groups:
+    // B tiles hide the TMA latency for G groups each, raw slabs for T_MA/128 groups each.
+    const double target_b = 8.0 * 64 / T_K, target_r = 6.0 * 64 / T_K, target_g = 4.0;
+    for (;;) {
+        const double cov_b = nb * G / target_b, cov_r = nr * (T_MA / 128.0) / target_r, cov_g = ng / target_g;
+        int pick = -1;
+        double best = 1.0;                               // stop once every ring meets its target
+        if (cov_b < best && nb < kMaxStages && total(nb + 1, ng, nr) <= kSmemBudget) { best = cov_b; pick = 0; }
+        if (cov_r < best && nr + nr_step <= kMaxStages && bars_ok(ng, nr + nr_step) && total(nb, ng, nr + nr_step) <= kSmemBudget) { best = cov_r; pick = 1; }
+        if (cov_g < best && ng + ng_step <= kMaxStages && bars_ok(ng + ng_step, nr) && total(nb, ng + ng_step, nr) <= kSmemBudget) { best = cov_g; pick = 2; }
+        if (pick < 0) break;
+        if (pick == 0) ++nb; else if (pick == 1) nr += nr_step; else ng += ng_step;
+    }
+#if defined(ATB_RINGS_NB) && defined(ATB_RINGS_NG) && defined(ATB_RINGS_NR)
+    // Tuning build: fixed depths wherever they are valid for the tiling and fit.
+    if (ATB_RINGS_NB >= 2 && ATB_RINGS_NG >= gps && ATB_RINGS_NG % gps == 0 && ATB_RINGS_NR >= 1 &&
+        bars_ok(ATB_RINGS_NG, ATB_RINGS_NR) && total(ATB_RINGS_NB, ATB_RINGS_NG, ATB_RINGS_NR) <= kSmemBudget) {
+        nb = ATB_RINGS_NB; ng = ATB_RINGS_NG; nr = ATB_RINGS_NR;
+    }
+#endif
+    pl.nb = nb; pl.ng = ng; pl.nr = nr;
+    pl.smem_bytes = total(nb, ng, nr);
+    pl.ok = true;
+    return pl;
+}
+
+// CTA-pair kernel (T_MC = 256, T_N = 512, T_K = 64); `slab` = min(T_MA, 128) rows.
+constexpr RingPlan plan_pair(int slab) {
+    RingPlan pl;
+    if (!(slab == 32 || slab == 64 || slab == 128)) return pl;
+    const int slabs = 128 / slab;
+    const uint32_t b_bytes = 4 * 64 * 128, group_bytes = 128 * 64 * 2, raw_bytes = slab * 64 * 9 / 8;
+    const int dqg = 4;
+    pl.dqg = dqg;
+    pl.acc_bufs = 1;
+    pl.tmem_cols = 512;
+    const auto total = [=](int b, int g, int r) { return ring_smem_bytes(b_bytes, group_bytes, raw_bytes, 2, dqg, b, g, g * slabs, r); };
+    const auto bars_ok = [=](int g, int r) { return ring_bars(r, dqg) <= kMaxRingBars && ring_bars(g * slabs, dqg) <= kMaxRingBars; };
+    // as in plan_single: whole rounds of the dequantiser groups
+    int ng = (dqg + slabs - 1) / slabs;
+    if ((ng * slabs) % dqg != 0) ng = dqg;
+    const int ng_step = ng;
+    int nb = 3, nr = dqg;
+    pl.nb = nb; pl.ng = ng; pl.nr = nr;
+    if (total(nb, ng, nr) > kSmemBudget) return pl;
+    // Spend what is left on bf16 groups, raw slabs (up to 8 K-steps of look-ahead), then B tiles
+    // (measured: the dequantised-A ring is the one whose depth pays most).
+    while (ng + ng_step <= 4 && bars_ok(ng + ng_step, nr) && total(nb, ng + ng_step, nr) <= kSmemBudget) ng += ng_step;
+    while (nr + dqg <= kMaxStages && nr * slab < 8 * 128 && bars_ok(ng, nr + dqg) && total(nb, ng, nr + dqg) <= kSmemBudget) nr += dqg;
+    while (nb < 4 && total(nb + 1, ng, nr) <= kSmemBudget) ++nb;
+#if defined(ATB_RINGS_NB) && defined(ATB_RINGS_NG) && defined(ATB_RINGS_NR)
+    if (ATB_RINGS_NB >= 2 && ATB_RINGS_NG >= 1 && ATB_RINGS_NR >= 1 && bars_ok(ATB_RINGS_NG, ATB_RINGS_NR) &&
+        total(ATB_RINGS_NB, ATB_RINGS_NG, ATB_RINGS_NR) <= kSmemBudget) {
+        nb = ATB_RINGS_NB; ng = ATB_RINGS_NG; nr = ATB_RINGS_NR;
+    }
+#endif
+    pl.nb = nb; pl.ng = ng; pl.nr = nr;
+    pl.smem_bytes = total(nb, ng, nr);
+    pl.ok = true;
+    return pl;
+}
 
 struct GemmParams {
     int64_t M, N, K, ldc;
     __nv_bfloat16* C;
     int m_tiles, n_tiles, k_steps;
-    int n_b_stages, n_groups, n_raw_stages, acc_bufs, tmem_cols;
     unsigned int* error_flag;
     int splits;          // split-K: each output tile is computed as `splits` partial tiles over K ranges
     int m_pad;           // split-K: rows per split in the FP32 workspace (m_tiles * T_MC)
@@ -60,11 +184,36 @@ struct Ring {
     __device__ __forceinline__ void advance(int n) {
         if (++stage == n) { stage = 0; phase ^= 1u; }
     }
-    // `step` stages at once; n is a multiple of step and stage stays congruent modulo step
-    __device__ __forceinline__ void advance_by(int step, int n) {
-        stage += step;
-        if (stage >= n) { stage -= n; phase ^= 1u; }
+};
+
+// Position of a slab in a ring of N buffers guarded by L = ring_bars(N, groups) barrier pairs.
+// `phase` is the parity of the barrier phase that belongs to this slab.  All sizes are compile-time
+// constants; with L == N the buffer index and the barrier index are one variable.
+template <int N, int L>
+struct Cursor {
+    static_assert(L >= N && L % N == 0, "L is a multiple of N");
+    int bar = 0, buf_ = 0;
+    uint32_t phase = 0;
+    __device__ __forceinline__ void start_at(int slab) {       // slab < L
+        bar = slab;
+        buf_ = slab % N;
     }
+    __device__ __forceinline__ int buf() const { return L == N ? bar : buf_; }
+    template <int STEP>
+    __device__ __forceinline__ void advance() {
+        static_assert(STEP <= L, "step");
+        bar += STEP;
+        if (bar >= L) { bar -= L; phase ^= 1u; }
+        if (L != N) {
+            buf_ += STEP % N;
+            if (buf_ >= N) buf_ -= N;
+        }
+    }
+    // Barrier index and parity of the slab N places back - the last user of this slab's buffer.
+    // For the first N slabs that is a phase "before the first", which a fresh barrier reports
+    // as complete.
+    __device__ __forceinline__ int freed_bar() const { return (L == N || bar < N) ? bar - N + L : bar - N; }
+    __device__ __forceinline__ uint32_t freed_parity() const { return (L == N || bar < N) ? phase ^ 1u : phase; }
 };
 
 struct Ctx {
@@ -194,44 +343,62 @@ __device__ __forceinline__ uint32_t scale_table_entry(uint32_t E) {
     return E == 255u ? 0u : bits * 0x10001u;
 }
 
+// Per-thread constants of the dequantiser: thread t of a group owns slot t (16 mantissas = blocks
+// 2p, 2p+1 of row r0) of every ROWS_PER_ITER-row band of a slab.  All shared-memory offsets of the
+// thread are fixed; a slab only moves the base addresses.
 template <class C>
-__device__ __forceinline__ void dequant_slab(uint32_t raw_mant, uint32_t raw_exp, uint32_t scale_lut,
+struct DequantLane {
+    uint32_t ld_off, exp_off, st_off0, st_off1;
+    __device__ __forceinline__ DequantLane(int t, int slab_rows) {
+        const int p = t % C::SLOTS_PER_ROW, r0 = t / C::SLOTS_PER_ROW, kb = 2 * p;
+        const uint32_t sw = static_cast<uint32_t>(r0 & 7);                  // ROWS_PER_ITER is a multiple of 8
+        ld_off = static_cast<uint32_t>(t) * 16u;
+        exp_off = static_cast<uint32_t>((kb >> 3) * slab_rows * 8 + r0 * 8 + (kb & 7));
+        const uint32_t row = static_cast<uint32_t>((kb >> 3)) * C::KHALF_BYTES + static_cast<uint32_t>(r0) * 128u;
+        st_off0 = row + (((static_cast<uint32_t>(kb) & 7u) ^ sw) << 4);
+        st_off1 = row + ((((static_cast<uint32_t>(kb) & 7u) + 1u) ^ sw) << 4);
+    }
+};
+
+// Dequantises one slab: raw mantissas / exponents in shared memory -> bf16 operand rows starting at
+// row `row_base` (a multiple of 32) of the 128-row groups at dst_base.
+template <class C>
+__device__ __forceinline__ void dequant_slab(const DequantLane<C>& ln, uint32_t raw_mant, uint32_t raw_exp, uint32_t scale_lut,
                                              uint32_t dst_base, int row_base, int t, int T_MA_rows) {
-    const int p = t % C::SLOTS_PER_ROW;                 // blocks 2p, 2p + 1 of the row
+    static_assert(C::ROWS_PER_ITER % 8 == 0 && 128 % C::ROWS_PER_ITER == 0, "band height");
+    const uint32_t ld = raw_mant + ln.ld_off, le = raw_exp + ln.exp_off;
+    const uint32_t st0 = dst_base + static_cast<uint32_t>(row_base) * 128u + ln.st_off0;
+    const uint32_t st1 = dst_base + static_cast<uint32_t>(row_base) * 128u + ln.st_off1;
     const int r0 = t / C::SLOTS_PER_ROW;
-    const int kb = 2 * p;
     uint4 w[C::DQ_ITERS];
     uint32_t e[C::DQ_ITERS];
 #pragma unroll
     for (int i = 0; i < C::DQ_ITERS; ++i) {
-        const int r = r0 + i * C::ROWS_PER_ITER;
-        if (C::SLOTS % C::GROUP_THREADS == 0 || r < T_MA_rows) {
+        if (C::SLOTS % C::GROUP_THREADS == 0 || r0 + i * C::ROWS_PER_ITER < T_MA_rows) {
             asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
                          : "=r"(w[i].x), "=r"(w[i].y), "=r"(w[i].z), "=r"(w[i].w)
-                         : "r"(raw_mant + (r * C::SLOTS_PER_ROW + p) * 16));
+                         : "r"(ld + static_cast<uint32_t>(i * C::GROUP_THREADS * 16)));
             uint16_t e2;
-            asm volatile("ld.shared.u16 %0, [%1];" : "=h"(e2)
-                         : "r"(raw_exp + (kb >> 3) * T_MA_rows * 8 + r * 8 + (kb & 7)));
+            asm volatile("ld.shared.u16 %0, [%1];" : "=h"(e2) : "r"(le + static_cast<uint32_t>(i * C::ROWS_PER_ITER * 8)));
             e[i] = e2;
         }
     }
 #pragma unroll
     for (int i = 0; i < C::DQ_ITERS; ++i) {
-        const int r = r0 + i * C::ROWS_PER_ITER;
-        if (C::SLOTS % C::GROUP_THREADS == 0 || r < T_MA_rows) {
+        if (C::SLOTS % C::GROUP_THREADS == 0 || r0 + i * C::ROWS_PER_ITER < T_MA_rows) {
             uint32_t s0, s1;
             asm volatile("ld.shared.b32 %0, [%1];" : "=r"(s0) : "r"(scale_lut + (e[i] & 0xFFu) * 4));
             asm volatile("ld.shared.b32 %0, [%1];" : "=r"(s1) : "r"(scale_lut + (e[i] >> 8) * 4));
             const uint32_t u0 = w[i].x ^ 0x80808080u, u1 = w[i].y ^ 0x80808080u;
             const uint32_t u2 = w[i].z ^ 0x80808080u, u3 = w[i].w ^ 0x80808080u;
-            const int rr = row_base + r;
-            const uint32_t row_addr = dst_base + (rr >> 7) * C::GROUP_BYTES + (kb >> 3) * C::KHALF_BYTES + (rr & 127) * 128;
-            const uint32_t sw = static_cast<uint32_t>(rr & 7);
-            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row_addr + ((((kb & 7)) ^ sw) << 4)),
+            // band i starts i * ROWS_PER_ITER rows further on: possibly in the next 128-row group
+            constexpr uint32_t kBandRows = C::ROWS_PER_ITER;
+            const uint32_t band = static_cast<uint32_t>((i * kBandRows) >> 7) * C::GROUP_BYTES + static_cast<uint32_t>((i * kBandRows) & 127) * 128u;
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(st0 + band),
                          "r"(dequant_pair(u0, 0x4140u, s0)), "r"(dequant_pair(u0, 0x4342u, s0)),
                          "r"(dequant_pair(u1, 0x4140u, s0)), "r"(dequant_pair(u1, 0x4342u, s0))
                          : "memory");
-            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row_addr + ((((kb & 7) + 1) ^ sw) << 4)),
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(st1 + band),
                          "r"(dequant_pair(u2, 0x4140u, s1)), "r"(dequant_pair(u2, 0x4342u, s1)),
                          "r"(dequant_pair(u3, 0x4140u, s1)), "r"(dequant_pair(u3, 0x4342u, s1))
                          : "memory");

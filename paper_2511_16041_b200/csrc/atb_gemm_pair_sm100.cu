@@ -38,12 +38,17 @@ struct PairCfg {
     static constexpr int GROUP_THREADS = GROUP_WARPS * 32;
     static constexpr int DQ_ITERS = (SLOTS + GROUP_THREADS - 1) / GROUP_THREADS;
     static constexpr int ROWS_PER_ITER = GROUP_THREADS / SLOTS_PER_ROW;
+    // ring depths (compile-time)
+    static constexpr RingPlan PLAN = plan_pair(SLAB_ROWS);
+    static constexpr int NB = PLAN.nb, NG = PLAN.ng, NR = PLAN.nr;
+    static constexpr int ND = NG * SLABS;                      // dequantised slab stages
+    static constexpr int LR = ring_bars(NR, DQ_GROUPS), LD = ring_bars(ND, DQ_GROUPS);
+    static_assert(PLAN.ok && DQ_GROUPS == PLAN.dqg, "plan");
 };
 
 struct PairParams {
     int64_t M, N, K;
     int m_tiles, n_tiles, k_steps;           // tiles of 256 x 512
-    int n_b_stages, n_groups, n_raw_stages;
     unsigned int* error_flag;
 };
 
@@ -66,17 +71,16 @@ atb_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_c
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* const smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
     const uint32_t b_base = smem_base;
-    const uint32_t deq_base = b_base + p.n_b_stages * C::B_BYTES;
-    const uint32_t raw_off = p.n_b_stages * C::B_BYTES + p.n_groups * C::GROUP_BYTES;
+    const uint32_t deq_base = b_base + C::NB * C::B_BYTES;
+    constexpr uint32_t raw_off = C::NB * C::B_BYTES + C::NG * C::GROUP_BYTES;
     const uint32_t raw_base = smem_base + raw_off;
-    const uint32_t stage_off = (raw_off + p.n_raw_stages * C::RAW_BYTES + 1023u) & ~1023u;
-    const uint32_t bar_off = stage_off + 4u * kEpilogueBoxBytes;
+    constexpr uint32_t stage_off = (raw_off + C::NR * C::RAW_BYTES + 1023u) & ~1023u;
+    constexpr uint32_t bar_off = stage_off + 4u * kEpilogueBoxBytes;
     const uint32_t bar_base = smem_base + bar_off;
-    const int n_deq_stages = p.n_groups * C::SLABS;
-    const uint32_t b_full = bar_base, b_empty = b_full + 8 * p.n_b_stages;
-    const uint32_t raw_full = b_empty + 8 * p.n_b_stages, raw_empty = raw_full + 8 * p.n_raw_stages;
-    const uint32_t deq_full = raw_empty + 8 * p.n_raw_stages, deq_empty = deq_full + 8 * n_deq_stages;
-    const uint32_t acc_full = deq_empty + 8 * n_deq_stages, acc_empty = acc_full + 8 * C::N_CHUNKS;
+    const uint32_t b_full = bar_base, b_empty = b_full + 8 * C::NB;
+    const uint32_t raw_full = b_empty + 8 * C::NB, raw_empty = raw_full + 8 * C::LR;
+    const uint32_t deq_full = raw_empty + 8 * C::LR, deq_empty = deq_full + 8 * C::LD;
+    const uint32_t acc_full = deq_empty + 8 * C::LD, acc_empty = acc_full + 8 * C::N_CHUNKS;
     const uint32_t misc = acc_empty + 8 * C::N_CHUNKS;       // [0]: TMEM base, [1]: abort flag
     const uint32_t scale_lut = misc + 16;
     volatile uint32_t* const misc_gen = reinterpret_cast<volatile uint32_t*>(smem_gen + (misc - smem_base));
@@ -89,9 +93,9 @@ atb_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_c
     if (threadIdx.x == 0) {
         // Barriers with arrivals from both CTAs are only used in the leader, but are initialised
         // everywhere so that both CTAs have the same layout.
-        for (int i = 0; i < p.n_b_stages; ++i) { mbar_init(b_full + 8 * i, 1); mbar_init(b_empty + 8 * i, 1); }
-        for (int i = 0; i < p.n_raw_stages; ++i) { mbar_init(raw_full + 8 * i, 1); mbar_init(raw_empty + 8 * i, C::GROUP_WARPS); }
-        for (int i = 0; i < n_deq_stages; ++i) { mbar_init(deq_full + 8 * i, 2 * C::GROUP_WARPS); mbar_init(deq_empty + 8 * i, 1); }
+        for (int i = 0; i < C::NB; ++i) { mbar_init(b_full + 8 * i, 1); mbar_init(b_empty + 8 * i, 1); }
+        for (int i = 0; i < C::LR; ++i) { mbar_init(raw_full + 8 * i, 1); mbar_init(raw_empty + 8 * i, C::GROUP_WARPS); }
+        for (int i = 0; i < C::LD; ++i) { mbar_init(deq_full + 8 * i, 2 * C::GROUP_WARPS); mbar_init(deq_empty + 8 * i, 1); }
         for (int i = 0; i < C::N_CHUNKS; ++i) { mbar_init(acc_full + 8 * i, 1); mbar_init(acc_empty + 8 * i, 8); }
         misc_gen[1] = 0u;
         fence_mbar_init();
@@ -135,14 +139,14 @@ atb_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_c
                     for (int j = 0; j < 4; ++j)
                         tma_load_2d_pair(b_base + rb.stage * C::B_BYTES + j * C::B_BOX_BYTES, &tm_b,
                                          colb + (j >> 1) * 256 + (j & 1) * 64, k * C::T_K, fb);
-                    rb.advance(p.n_b_stages);
+                    rb.advance(C::NB);
                 }
             }
         }
     } else if (warp == kAProducerWarp) {
         // ================================ TMA producer: raw A slabs ====================
         if (elect_one()) {
-            Ring rr;
+            Cursor<C::NR, C::LR> rr;
             bool ok = true;
             for (int tile = cluster_id; ok && tile < total_tiles; tile += n_clusters) {
                 int mt, nt;
@@ -150,13 +154,13 @@ atb_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_c
                 const int row0 = mt * 256 + static_cast<int>(rank) * 128;
                 for (int k = 0; ok && k < p.k_steps; ++k) {
                     for (int s = 0; s < C::SLABS; ++s) {
-                        if (!(ok = wait_bar_cl_spin(cx, raw_empty + 8 * rr.stage, rr.phase ^ 1u, 0x002))) break;
-                        const uint32_t fr = raw_full + 8 * rr.stage;
-                        const uint32_t dst = raw_base + rr.stage * C::RAW_BYTES;
+                        if (!(ok = wait_bar_cl_spin(cx, raw_empty + 8 * rr.freed_bar(), rr.freed_parity(), 0x002))) break;
+                        const uint32_t fr = raw_full + 8 * rr.bar;
+                        const uint32_t dst = raw_base + rr.buf() * C::RAW_BYTES;
                         mbar_arrive_expect_tx(fr, C::RAW_BYTES);
                         tma_load_2d(dst, &tm_mant, k * C::T_K, row0 + s * SLAB_ROWS, fr);
                         tma_load_2d(dst + C::RAW_MANT_BYTES, &tm_exp, row0 + s * SLAB_ROWS, k, fr);
-                        rr.advance(p.n_raw_stages);
+                        rr.template advance<1>();
                     }
                 }
             }
@@ -165,16 +169,17 @@ atb_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_c
         // ================================ UMMA issuer (leader CTA) ====================
         if (leader && elect_one()) {
             constexpr uint32_t idesc = umma_idesc_bf16_f32(256, C::N_MMA, false, true);
-            Ring rb, rd;
+            Ring rb;
+            Cursor<C::ND, C::LD> rd;
             uint32_t acc_phase = 0;
             bool ok = true;
             for (int tile = cluster_id; ok && tile < total_tiles; tile += n_clusters, acc_phase ^= 1u) {
                 for (int k = 0; ok && k < p.k_steps; ++k) {
                     if (!(ok = wait_bar_cl_spin(cx, b_full + 8 * rb.stage, rb.phase, 0x101))) break;
                     for (int i = 0; ok && i < C::SLABS; ++i)
-                        ok = wait_bar_cl_spin(cx, deq_full + 8 * (rd.stage + i), rd.phase, 0x103);
+                        ok = wait_bar_cl_spin(cx, deq_full + 8 * (rd.bar + i), rd.phase, 0x103);
                     if (!ok) break;
-                    const uint32_t as = deq_base + (rd.stage / C::SLABS) * C::GROUP_BYTES;
+                    const uint32_t as = deq_base + (rd.buf() / C::SLABS) * C::GROUP_BYTES;
                     const uint32_t bs = b_base + rb.stage * C::B_BYTES;
 #pragma unroll
                     for (int nc = 0; nc < C::N_CHUNKS; ++nc) {
@@ -191,10 +196,10 @@ atb_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_c
                         if (k == p.k_steps - 1) umma_commit_pair(acc_full + 8 * nc, 3);
                     }
                     if (!ok) break;
-                    for (int i = 0; i < C::SLABS; ++i) umma_commit_pair(deq_empty + 8 * (rd.stage + i), 3);
-                    for (int i = 0; i < C::SLABS; ++i) rd.advance(n_deq_stages);
+                    for (int i = 0; i < C::SLABS; ++i) umma_commit_pair(deq_empty + 8 * (rd.bar + i), 3);
+                    rd.template advance<C::SLABS>();
                     umma_commit_pair(b_empty + 8 * rb.stage, 3);
-                    rb.advance(p.n_b_stages);
+                    rb.advance(C::NB);
                 }
             }
         }
@@ -257,24 +262,26 @@ atb_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_c
         // slabs arrive in ring order: a group takes every DQ_GROUPS-th slab of this CTA's stream
         int64_t my_slabs = 0;
         for (int tile = cluster_id; tile < total_tiles; tile += n_clusters) my_slabs += static_cast<int64_t>(p.k_steps) * C::SLABS;
-        Ring rr, rd;
-        rr.stage = my_group;
-        rd.stage = my_group;
+        const DequantLane<C> ln(t, SLAB_ROWS);
+        Cursor<C::NR, C::LR> rr;
+        Cursor<C::ND, C::LD> rd;
+        rr.start_at(my_group);
+        rd.start_at(my_group);
         for (int64_t n = my_group; n < my_slabs; n += C::DQ_GROUPS) {
-            if (!wait_bar_cl(cx, raw_full + 8 * rr.stage, rr.phase, 0x301)) break;
-            if (!wait_bar_cl(cx, deq_empty + 8 * rd.stage, rd.phase ^ 1u, 0x302)) break;
-            const uint32_t raw = raw_base + rr.stage * C::RAW_BYTES;
-            const uint32_t dst_base = deq_base + (rd.stage / C::SLABS) * C::GROUP_BYTES;
-            const int row_base = (rd.stage % C::SLABS) * SLAB_ROWS;
-            dequant_slab<C>(raw, raw + C::RAW_MANT_BYTES, scale_lut, dst_base, row_base, t, SLAB_ROWS);
+            if (!wait_bar_cl(cx, raw_full + 8 * rr.bar, rr.phase, 0x301)) break;
+            if (!wait_bar_cl(cx, deq_empty + 8 * rd.freed_bar(), rd.freed_parity(), 0x302)) break;
+            const uint32_t raw = raw_base + rr.buf() * C::RAW_BYTES;
+            const uint32_t dst_base = deq_base + (rd.buf() / C::SLABS) * C::GROUP_BYTES;
+            const int row_base = (rd.buf() % C::SLABS) * SLAB_ROWS;
+            dequant_slab<C>(ln, raw, raw + C::RAW_MANT_BYTES, scale_lut, dst_base, row_base, t, SLAB_ROWS);
             fence_proxy_async_smem();
             __syncwarp();
             if (lane == 0) {
-                mbar_arrive_cluster(mapa_shared(deq_full + 8 * rd.stage, 0));
-                mbar_arrive(raw_empty + 8 * rr.stage);
+                mbar_arrive_cluster(mapa_shared(deq_full + 8 * rd.bar, 0));
+                mbar_arrive(raw_empty + 8 * rr.bar);
             }
-            rr.advance_by(C::DQ_GROUPS, p.n_raw_stages);
-            rd.advance_by(C::DQ_GROUPS, n_deq_stages);
+            rr.template advance<C::DQ_GROUPS>();
+            rd.template advance<C::DQ_GROUPS>();
         }
     }
 
@@ -313,7 +320,6 @@ atb_status_t launch_pair_t(const atb::GemmPlan& plan, int64_t M, int64_t N, int6
     p.m_tiles = static_cast<int>(atb::ceil_div(M, 256));
     p.n_tiles = static_cast<int>(atb::ceil_div(N, 512));
     p.k_steps = static_cast<int>(atb::ceil_div(K, C::T_K));
-    p.n_b_stages = plan.n_b_stages; p.n_groups = plan.n_groups; p.n_raw_stages = plan.n_raw_stages;
     p.error_flag = error_flag;
 
     auto kernel = atb_gemm_pair_kernel<SLAB_ROWS>;
@@ -331,37 +337,6 @@ atb_status_t launch_pair_t(const atb::GemmPlan& plan, int64_t M, int64_t N, int6
 }  // namespace
 
 namespace atb {
-
-bool plan_gemm_pair(int T_MA, GemmPlan* plan) {
-    if (!(T_MA == 32 || T_MA == 64 || T_MA == 128 || T_MA == 256)) return false;
-    const int slab = T_MA > 128 ? 128 : T_MA;
-    const int slabs = 128 / slab;
-    const uint32_t b_bytes = 4 * 64 * 128, group_bytes = 128 * 64 * 2, raw_bytes = slab * 64 * 9 / 8;
-    // 4 dequantiser groups: raw ring and slab stages in multiples of 4
-    const int dqg = 4;                                   // PairCfg::DQ_GROUPS
-    int ng = (dqg + slabs - 1) / slabs;
-    if ((ng * slabs) % dqg != 0) ng = dqg;
-    const int ng_step = ng;
-    int nb = 3, nr = dqg;
-    auto total = [&](int b, int g, int r) {
-        const uint32_t bars = 8u * (2 * b + 2 * r + 2 * g * slabs + 4) + 16u + 1024u;
-        return 1024u + b * b_bytes + g * group_bytes + r * raw_bytes + 1024u + 4u * kEpilogueBoxBytes + bars;
-    };
-    if (total(nb, ng, nr) > kSmemBudget) return false;
-    // Spend what is left on raw slabs (up to 8 K-steps of look-ahead), then B tiles, then bf16
-    // groups (measured: the dequantised-A ring is the one whose depth pays most).
-    while (ng + ng_step <= 4 && total(nb, ng + ng_step, nr) <= kSmemBudget) ng += ng_step;
-    while (nr + dqg <= kMaxStages && nr * slab < 8 * 128 && total(nb, ng, nr + dqg) <= kSmemBudget) nr += dqg;
-    while (nb < 4 && total(nb + 1, ng, nr) <= kSmemBudget) ++nb;
-    plan->dq_groups = dqg;
-    plan->n_b_stages = nb;
-    plan->n_groups = ng;
-    plan->n_raw_stages = nr;
-    plan->acc_bufs = 1;
-    plan->tmem_cols = 512;
-    plan->smem_bytes = total(nb, ng, nr);
-    return true;
-}
 
 atb_status_t launch_gemm_pair(int T_MA, const GemmPlan& plan, int64_t M, int64_t N, int64_t K, const int8_t* mant,
                               const uint8_t* exp, const void* B, int64_t ldb, void* C, int64_t ldc, int num_sms,

@@ -53,6 +53,13 @@ struct Cfg {
     static constexpr int GROUP_THREADS = GROUP_WARPS * 32;
     static constexpr int DQ_ITERS = (SLOTS + GROUP_THREADS - 1) / GROUP_THREADS;
     static constexpr int ROWS_PER_ITER = GROUP_THREADS / SLOTS_PER_ROW;
+    // ring depths (compile-time: every ring index below folds to constants)
+    static constexpr RingPlan PLAN = plan_single(T_MA, T_MC, T_K, T_N);
+    static constexpr int NB = PLAN.nb, NG = PLAN.ng, NR = PLAN.nr;
+    static constexpr int ND = (T_MA <= 128) ? NG * SPG : NG / GPS;   // dequantised slab stages
+    static constexpr int LR = ring_bars(NR, DQ_GROUPS), LD = ring_bars(ND, DQ_GROUPS);
+    static constexpr int ACC_BUFS = PLAN.acc_bufs, TMEM_COLS = PLAN.tmem_cols;
+    static_assert(DQ_GROUPS == PLAN.dqg && ND % SPG == 0, "plan");
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -68,20 +75,19 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* const smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
     const uint32_t b_base = smem_base;
-    const uint32_t deq_base = b_base + p.n_b_stages * C::B_BYTES;
-    const uint32_t raw_off = p.n_b_stages * C::B_BYTES + p.n_groups * C::GROUP_BYTES;
+    const uint32_t deq_base = b_base + C::NB * C::B_BYTES;
+    constexpr uint32_t raw_off = C::NB * C::B_BYTES + C::NG * C::GROUP_BYTES;
     const uint32_t raw_base = smem_base + raw_off;
     // epilogue staging: one 32-row x 64-column bf16 box (4 KB, 128-byte swizzle) per epilogue warp
-    const uint32_t stage_off = (raw_off + p.n_raw_stages * C::RAW_BYTES + 1023u) & ~1023u;
-    const uint32_t bar_off = stage_off + 4u * kEpilogueBoxBytes;
+    constexpr uint32_t stage_off = (raw_off + C::NR * C::RAW_BYTES + 1023u) & ~1023u;
+    constexpr uint32_t bar_off = stage_off + 4u * kEpilogueBoxBytes;
     const uint32_t bar_base = smem_base + bar_off;          // 8-byte mbarriers
-    const int n_deq_stages = (T_MA <= 128) ? p.n_groups * C::SPG : p.n_groups / C::GPS;
-    const int n_acc = p.acc_bufs * C::G;
+    constexpr int n_acc = C::ACC_BUFS * C::G;
     // barrier indices
-    const uint32_t b_full = bar_base, b_empty = b_full + 8 * p.n_b_stages;
-    const uint32_t raw_full = b_empty + 8 * p.n_b_stages, raw_empty = raw_full + 8 * p.n_raw_stages;
-    const uint32_t deq_full = raw_empty + 8 * p.n_raw_stages, deq_empty = deq_full + 8 * n_deq_stages;
-    const uint32_t acc_full = deq_empty + 8 * n_deq_stages, acc_empty = acc_full + 8 * n_acc;
+    const uint32_t b_full = bar_base, b_empty = b_full + 8 * C::NB;
+    const uint32_t raw_full = b_empty + 8 * C::NB, raw_empty = raw_full + 8 * C::LR;
+    const uint32_t deq_full = raw_empty + 8 * C::LR, deq_empty = deq_full + 8 * C::LD;
+    const uint32_t acc_full = deq_empty + 8 * C::LD, acc_empty = acc_full + 8 * n_acc;
     const uint32_t misc = acc_empty + 8 * n_acc;             // [0]: TMEM base, [1]: abort flag
     const uint32_t scale_lut = misc + 16;                    // 256 floats: 2^(E-133)
     volatile uint32_t* const misc_gen = reinterpret_cast<volatile uint32_t*>(smem_gen + (misc - smem_base));
@@ -90,9 +96,9 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
     Ctx cx{misc_gen + 1, p.error_flag};
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < p.n_b_stages; ++i) { mbar_init(b_full + 8 * i, 1); mbar_init(b_empty + 8 * i, 1); }
-        for (int i = 0; i < p.n_raw_stages; ++i) { mbar_init(raw_full + 8 * i, 1); mbar_init(raw_empty + 8 * i, C::GROUP_WARPS); }
-        for (int i = 0; i < n_deq_stages; ++i) { mbar_init(deq_full + 8 * i, C::GROUP_WARPS); mbar_init(deq_empty + 8 * i, 1); }
+        for (int i = 0; i < C::NB; ++i) { mbar_init(b_full + 8 * i, 1); mbar_init(b_empty + 8 * i, 1); }
+        for (int i = 0; i < C::LR; ++i) { mbar_init(raw_full + 8 * i, 1); mbar_init(raw_empty + 8 * i, C::GROUP_WARPS); }
+        for (int i = 0; i < C::LD; ++i) { mbar_init(deq_full + 8 * i, C::GROUP_WARPS); mbar_init(deq_empty + 8 * i, 1); }
         for (int i = 0; i < n_acc; ++i) { mbar_init(acc_full + 8 * i, 1); mbar_init(acc_empty + 8 * i, 4); }
         misc_gen[1] = 0u;
         fence_mbar_init();
@@ -102,7 +108,7 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
         prefetch_tensormap(&tm_c);
     }
     if (warp == 1) {
-        tmem_alloc(misc, static_cast<uint32_t>(p.tmem_cols));
+        tmem_alloc(misc, static_cast<uint32_t>(C::TMEM_COLS));
         tmem_relinquish();
     }
     if (threadIdx.x >= kFirstDequantWarp * 32 && threadIdx.x < kFirstDequantWarp * 32 + 256) {
@@ -131,7 +137,7 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
                     for (int j = 0; j < T_N / 64; ++j)
                         tma_load_2d(b_base + rb.stage * C::B_BYTES + j * C::B_BOX_BYTES, &tm_b,
                                     w.nt * T_N + j * 64, k * T_K, fb);
-                    rb.advance(p.n_b_stages);
+                    rb.advance(C::NB);
                 }
             }
         }
@@ -140,19 +146,19 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
         // A producer of its own: the raw slabs feed the dequantisers, which run ahead of the UMMAs,
         // so these loads must not queue behind the wait for a free B stage.
         if (elect_one()) {
-            Ring rr;
+            Cursor<C::NR, C::LR> rr;
             bool ok = true;
             for (int item = blockIdx.x; ok && item < total_items; item += gridDim.x) {
                 const WorkItem w = work_item<SPLIT>(item, p);
                 for (int k = w.k_begin; ok && k < w.k_end; ++k) {
                     for (int s = 0; s < C::RHO; ++s) {
-                        if (!(ok = wait_bar_spin(cx, raw_empty + 8 * rr.stage, rr.phase ^ 1u, 0x002))) break;
-                        const uint32_t fr = raw_full + 8 * rr.stage;
-                        const uint32_t dst = raw_base + rr.stage * C::RAW_BYTES;
+                        if (!(ok = wait_bar_spin(cx, raw_empty + 8 * rr.freed_bar(), rr.freed_parity(), 0x002))) break;
+                        const uint32_t fr = raw_full + 8 * rr.bar;
+                        const uint32_t dst = raw_base + rr.buf() * C::RAW_BYTES;
                         mbar_arrive_expect_tx(fr, C::RAW_BYTES);
                         tma_load_2d(dst, &tm_mant, k * T_K, w.mt * T_MC + s * T_MA, fr);
                         tma_load_2d(dst + C::RAW_MANT_BYTES, &tm_exp, w.mt * T_MC + s * T_MA, k * (T_K / 64), fr);
-                        rr.advance(p.n_raw_stages);
+                        rr.template advance<1>();
                     }
                 }
             }
@@ -161,13 +167,14 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
         // ================================ UMMA issuer =================================
         if (elect_one()) {
             constexpr uint32_t idesc = umma_idesc_bf16_f32(128, C::N_MMA, false, true);
-            Ring rb, rd;
+            Ring rb;
+            Cursor<C::ND, C::LD> rd;
             int it = 0;
             bool ok = true;
             for (int item = blockIdx.x; ok && item < total_items; item += gridDim.x, ++it) {
                 const WorkItem w = work_item<SPLIT>(item, p);
-                const int acc_buf = it % p.acc_bufs;
-                const uint32_t acc_phase = static_cast<uint32_t>(it / p.acc_bufs) & 1u;
+                const int acc_buf = it % C::ACC_BUFS;
+                const uint32_t acc_phase = static_cast<uint32_t>(it / C::ACC_BUFS) & 1u;
                 for (int k = w.k_begin; ok && k < w.k_end; ++k) {
                     if (!(ok = wait_bar_spin(cx, b_full + 8 * rb.stage, rb.phase, 0x101))) break;
                     const uint32_t bs = b_base + rb.stage * C::B_BYTES;
@@ -177,12 +184,12 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
                         int group_slot;
                         if (T_MA <= 128) {
                             for (int i = 0; ok && i < C::SPG; ++i)
-                                ok = wait_bar_spin(cx, deq_full + 8 * (rd.stage + i), rd.phase, 0x103);
+                                ok = wait_bar_spin(cx, deq_full + 8 * (rd.bar + i), rd.phase, 0x103);
                             if (!ok) break;
-                            group_slot = rd.stage / C::SPG;
+                            group_slot = rd.buf() / C::SPG;
                         } else {
-                            if ((g % C::GPS) == 0 && !(ok = wait_bar_spin(cx, deq_full + 8 * rd.stage, rd.phase, 0x103))) break;
-                            group_slot = rd.stage * C::GPS + (g % C::GPS);
+                            if ((g % C::GPS) == 0 && !(ok = wait_bar_spin(cx, deq_full + 8 * rd.bar, rd.phase, 0x103))) break;
+                            group_slot = rd.buf() * C::GPS + (g % C::GPS);
                         }
                         tcgen05_fence_after_sync();
                         const uint32_t as = deq_base + group_slot * C::GROUP_BYTES;
@@ -198,17 +205,17 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
                             }
                         }
                         if (T_MA <= 128) {
-                            for (int i = 0; i < C::SPG; ++i) umma_commit(deq_empty + 8 * (rd.stage + i));
-                            for (int i = 0; i < C::SPG; ++i) rd.advance(n_deq_stages);
+                            for (int i = 0; i < C::SPG; ++i) umma_commit(deq_empty + 8 * (rd.bar + i));
+                            rd.template advance<C::SPG>();
                         } else if ((g % C::GPS) == C::GPS - 1) {
-                            umma_commit(deq_empty + 8 * rd.stage);
-                            rd.advance(n_deq_stages);
+                            umma_commit(deq_empty + 8 * rd.bar);
+                            rd.template advance<1>();
                         }
                         if (k == w.k_end - 1) umma_commit(acc_full + 8 * acc);
                     }
                     if (!ok) break;
                     umma_commit(b_empty + 8 * rb.stage);
-                    rb.advance(p.n_b_stages);
+                    rb.advance(C::NB);
                 }
             }
         }
@@ -220,8 +227,8 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
         for (int item = blockIdx.x; ok && item < total_items; item += gridDim.x, ++it) {
             const WorkItem w = work_item<SPLIT>(item, p);
             const int mt = w.mt, nt = w.nt;
-            const int acc_buf = it % p.acc_bufs;
-            const uint32_t acc_phase = static_cast<uint32_t>(it / p.acc_bufs) & 1u;
+            const int acc_buf = it % C::ACC_BUFS;
+            const uint32_t acc_phase = static_cast<uint32_t>(it / C::ACC_BUFS) & 1u;
             for (int g = 0; g < C::G; ++g) {
                 const int acc = acc_buf * C::G + g;
                 if (!(ok = wait_bar(cx, acc_full + 8 * acc, acc_phase, 0x201))) break;
@@ -301,31 +308,33 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
             const WorkItem w = work_item<SPLIT>(item, p);
             my_slabs += static_cast<int64_t>(w.k_end - w.k_begin) * C::RHO;
         }
-        Ring rr, rd;
-        rr.stage = my_group;
-        rd.stage = my_group;
+        const DequantLane<C> ln(t, T_MA);
+        Cursor<C::NR, C::LR> rr;
+        Cursor<C::ND, C::LD> rd;
+        rr.start_at(my_group);
+        rd.start_at(my_group);
         for (int64_t n = my_group; n < my_slabs; n += C::DQ_GROUPS) {
-            if (!wait_bar(cx, raw_full + 8 * rr.stage, rr.phase, 0x301)) break;
-            if (!wait_bar(cx, deq_empty + 8 * rd.stage, rd.phase ^ 1u, 0x302)) break;
-            const uint32_t raw = raw_base + rr.stage * C::RAW_BYTES;
+            if (!wait_bar(cx, raw_full + 8 * rr.bar, rr.phase, 0x301)) break;
+            if (!wait_bar(cx, deq_empty + 8 * rd.freed_bar(), rd.freed_parity(), 0x302)) break;
+            const uint32_t raw = raw_base + rr.buf() * C::RAW_BYTES;
             uint32_t dst_base;
             int row_base;
             if (T_MA <= 128) {
-                dst_base = deq_base + (rd.stage / C::SPG) * C::GROUP_BYTES;
-                row_base = (rd.stage % C::SPG) * T_MA;
+                dst_base = deq_base + (rd.buf() / C::SPG) * C::GROUP_BYTES;
+                row_base = (rd.buf() % C::SPG) * T_MA;
             } else {
-                dst_base = deq_base + rd.stage * C::GPS * C::GROUP_BYTES;
+                dst_base = deq_base + rd.buf() * C::GPS * C::GROUP_BYTES;
                 row_base = 0;
             }
-            dequant_slab<C>(raw, raw + C::RAW_MANT_BYTES, scale_lut, dst_base, row_base, t, T_MA);
+            dequant_slab<C>(ln, raw, raw + C::RAW_MANT_BYTES, scale_lut, dst_base, row_base, t, T_MA);
             fence_proxy_async_smem();
             __syncwarp();
             if (lane == 0) {
-                mbar_arrive(deq_full + 8 * rd.stage);
-                mbar_arrive(raw_empty + 8 * rr.stage);
+                mbar_arrive(deq_full + 8 * rd.bar);
+                mbar_arrive(raw_empty + 8 * rr.bar);
             }
-            rr.advance_by(C::DQ_GROUPS, p.n_raw_stages);
-            rd.advance_by(C::DQ_GROUPS, n_deq_stages);
+            rr.template advance<C::DQ_GROUPS>();
+            rd.template advance<C::DQ_GROUPS>();
         }
     }
 
@@ -337,7 +346,7 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
     __syncthreads();
     if (warp == 1) {
         tcgen05_fence_after_sync();
-        tmem_dealloc(tmem_base, static_cast<uint32_t>(p.tmem_cols));
+        tmem_dealloc(tmem_base, static_cast<uint32_t>(C::TMEM_COLS));
     }
 }
 
@@ -373,8 +382,6 @@ atb_status_t launch(const atb::GemmPlan& plan, int64_t M, int64_t N, int64_t K, 
     p.m_tiles = static_cast<int>(atb::ceil_div(M, T_MC));
     p.n_tiles = static_cast<int>(atb::ceil_div(N, T_N));
     p.k_steps = static_cast<int>(atb::ceil_div(K, T_K));
-    p.n_b_stages = plan.n_b_stages; p.n_groups = plan.n_groups; p.n_raw_stages = plan.n_raw_stages;
-    p.acc_bufs = plan.acc_bufs; p.tmem_cols = plan.tmem_cols;
     p.error_flag = error_flag;
     p.splits = splits;
     p.m_pad = static_cast<int>(m_pad);
@@ -449,52 +456,21 @@ atb_status_t device_info(DeviceInfo** out) {
 
 namespace atb {
 
+static void fill_plan(const RingPlan& pl, GemmPlan* plan) {
+    plan->dq_groups = pl.dqg;
+    plan->n_b_stages = pl.nb;
+    plan->n_groups = pl.ng;
+    plan->n_raw_stages = pl.nr;
+    plan->acc_bufs = pl.acc_bufs;
+    plan->tmem_cols = pl.tmem_cols;
+    plan->smem_bytes = pl.smem_bytes;
+}
+
 bool plan_gemm(int T_MA, int T_MC, int T_K, int T_N, GemmPlan* plan) {
-    if (is_pair_tiling(T_MC, T_K, T_N)) return T_MA <= T_MC && plan_gemm_pair(T_MA, plan);
-    if (!(T_MC == 128 || T_MC == 256)) return false;
-    if (!(T_N == 64 || T_N == 128 || T_N == 256 || T_N == 512)) return false;
-    if (!(T_K == 64 || T_K == 128)) return false;
-    if (!(T_MA == 32 || T_MA == 64 || T_MA == 128 || T_MA == 256) || T_MA > T_MC) return false;
-    const int G = T_MC / 128;
-    if (G * T_N > 512) return false;
-    const uint32_t b_bytes = T_K * T_N * 2, group_bytes = 128 * T_K * 2, raw_bytes = T_MA * T_K * 9 / 8;
-    const int gps = T_MA > 128 ? T_MA / 128 : 1;          // groups per slab
-    const int spg = T_MA < 128 ? 128 / T_MA : 1;          // slabs per group
-    // The raw-slab ring and the ring of dequantised slab stages come in multiples of the
-    // dequantiser group count (see dq_groups); the bf16 ring itself is counted in 128-row groups.
-    const int dqg = dq_groups(T_MA, T_K, T_N);
-    const int nr_step = dqg;
-    const int ng_step = T_MA <= 128 ? (dqg >= spg ? dqg / spg : 1) : dqg * gps;
-    auto total = [&](int b, int g, int r) {
-        const int n_deq = T_MA <= 128 ? g * spg : g / gps;
-        const uint32_t bars = 8u * (2 * b + 2 * r + 2 * n_deq + 2 * 2 * G) + 16u + 1024u;
-        return 1024u + b * b_bytes + g * group_bytes + r * raw_bytes + 1024u + 4u * kEpilogueBoxBytes + bars;
-    };
-    int nb = 2, ng = ng_step, nr = nr_step;
-    if (ng < 2) ng = 2 * ng_step;
-    if (total(nb, ng, nr) > kSmemBudget) return false;
-    // Grow the rings towards a target look-ahead, counted in 128-row x T_K operand groups:
-    // B tiles hide the TMA latency for G groups each, raw slabs for T_MA/128 groups each.
-    const double target_b = 8.0 * 64 / T_K, target_r = 6.0 * 64 / T_K, target_g = 4.0;
-    for (;;) {
-        const double cov_b = nb * G / target_b, cov_r = nr * (T_MA / 128.0) / target_r, cov_g = ng / target_g;
-        int pick = -1;
-        double best = 1.0;                               // stop once every ring meets its target
-        if (cov_b < best && nb < kMaxStages && total(nb + 1, ng, nr) <= kSmemBudget) { best = cov_b; pick = 0; }
-        if (cov_r < best && nr + nr_step <= kMaxStages && total(nb, ng, nr + nr_step) <= kSmemBudget) { best = cov_r; pick = 1; }
-        if (cov_g < best && ng + ng_step <= kMaxStages && total(nb, ng + ng_step, nr) <= kSmemBudget) { best = cov_g; pick = 2; }
-        if (pick < 0) break;
-        if (pick == 0) ++nb; else if (pick == 1) nr += nr_step; else ng += ng_step;
-    }
-    plan->dq_groups = dqg;
-    plan->n_b_stages = nb;
-    plan->n_groups = ng;
-    plan->n_raw_stages = nr;
-    plan->acc_bufs = (2 * G * T_N <= 512) ? 2 : 1;
-    int cols = 32;
-    while (cols < plan->acc_bufs * G * T_N) cols <<= 1;
-    plan->tmem_cols = cols;
-    plan->smem_bytes = total(nb, ng, nr);
+    if (T_MA <= 0 || T_MC <= 0 || T_MA > T_MC) return false;
+    const RingPlan pl = is_pair_tiling(T_MC, T_K, T_N) ? plan_pair(T_MA > 128 ? 128 : T_MA) : plan_single(T_MA, T_MC, T_K, T_N);
+    if (!pl.ok || !(T_MA == 32 || T_MA == 64 || T_MA == 128 || T_MA == 256)) return false;
+    fill_plan(pl, plan);
     return true;
 }
 

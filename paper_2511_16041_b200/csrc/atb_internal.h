@@ -21,7 +21,7 @@ struct GemmPlan {
     int n_b_stages;      // B-tile ring depth
     int n_groups;        // dequantised-A ring depth, in 128-row groups
     int n_raw_stages;    // raw (BFP16) A-slab ring depth
-    int dq_groups;       // dequantiser warp groups (ring depths are multiples of it)
+    int dq_groups;       // dequantiser warp groups
     int acc_bufs;        // accumulator buffers in TMEM (1 or 2)
     int tmem_cols;       // allocated TMEM columns (power of two)
     uint32_t smem_bytes; // dynamic shared memory of the launch
@@ -30,7 +30,6 @@ struct GemmPlan {
 bool plan_gemm(int T_MA, int T_MC, int T_K, int T_N, GemmPlan* plan);
 // True for the tilings executed by a CTA pair (cluster of 2): T_MC = 256, T_N = 512, T_K = 64.
 inline bool is_pair_tiling(int T_MC, int T_K, int T_N) { return T_MC == 256 && T_N == 512 && T_K == 64; }
-bool plan_gemm_pair(int T_MA, GemmPlan* plan);
 atb_status_t launch_gemm_pair(int T_MA, const GemmPlan& plan, int64_t M, int64_t N, int64_t K, const int8_t* mant,
                               const uint8_t* exp, const void* B, int64_t ldb, void* C, int64_t ldc, int num_sms,
                               unsigned int* error_flag, void* stream);

@@ -74,9 +74,10 @@ def test_argument_validation_needs_no_gpu():
     assert atb.atb_last_error_message() != ""
 
 
-def test_ring_plans_keep_mbarrier_phases_in_order():
-    """Ring depths must be multiples of the dequantiser group count (a stage is then always
-    served by the same group), and everything must fit the 227 KB / 512-column budgets."""
+def test_ring_plans_fit_the_budgets():
+    """Every supported tiling gets rings that fit 227 KB of shared memory and 512 TMEM columns; the
+    barrier layout (lcm of depth and group count, see test_ring_protocol.py) stays small."""
+    import math
     n = 0
     for mc in (128, 256):
         for tn in (64, 128, 256, 512):
@@ -90,8 +91,10 @@ def test_ring_plans_keep_mbarrier_phases_in_order():
                     slab = min(ma, 128) if pair else ma
                     slab_stages = p.n_a_groups * (128 // slab) if slab <= 128 else p.n_a_groups // (slab // 128)
                     assert p.dequant_groups in (1, 2, 4)
-                    assert p.n_raw_stages % p.dequant_groups == 0, (ma, mc, tk, tn)
-                    assert slab_stages % p.dequant_groups == 0 and slab_stages >= 2, (ma, mc, tk, tn)
+                    assert p.n_raw_stages >= p.dequant_groups, (ma, mc, tk, tn)
+                    assert slab_stages >= 2, (ma, mc, tk, tn)
+                    assert math.lcm(p.n_raw_stages, p.dequant_groups) <= 32
+                    assert math.lcm(slab_stages, p.dequant_groups) <= 32
                     assert p.n_b_stages >= 2 and p.acc_buffers in (1, 2)
                     assert p.smem_bytes <= 232448 and p.tmem_columns <= 512
                     assert p.tmem_columns >= p.acc_buffers * (128 if pair else mc) // 128 * tn
