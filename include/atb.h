@@ -188,6 +188,10 @@ typedef struct {
                                      look-ahead is shorter scales the compute bound down                    */
     double pair_efficiency;       /* atb_select_tiling: measured factor on the compute bound of CTA-pair tilings */
     double launch_seconds;        /* atb_select_tiling: fixed cost per kernel launch              */
+    double tile_fixed_cycles;     /* atb_select_tiling: pipeline fill per output tile that no other tile hides    */
+    double drain_cycles_per_column; /* atb_select_tiling: where the accumulator is not double-buffered the UMMAs wait
+                                     while the epilogue drains it: cycles per FP32 accumulator column of a unit  */
+    double pair_tile_cycles;      /* atb_select_tiling: extra per-tile cost of a CTA pair (both units must finish) */
 } atb_hw_params_t;
 
 typedef struct {

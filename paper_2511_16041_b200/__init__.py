@@ -44,7 +44,8 @@ class atb_hw_params_t(ctypes.Structure):
                [("share_rows", ctypes.c_int), ("share_cols", ctypes.c_int)] + \
                [(n, ctypes.c_double) for n in ("eta", "eps_cycles", "ii", "delta_cycles")] + \
                [("mma_rows", ctypes.c_int)] + \
-               [(n, ctypes.c_double) for n in ("load_latency_cycles", "pair_efficiency", "launch_seconds")]
+               [(n, ctypes.c_double) for n in ("load_latency_cycles", "pair_efficiency", "launch_seconds", "tile_fixed_cycles",
+                                               "drain_cycles_per_column", "pair_tile_cycles")]
 
 
 class atb_tiling_score_t(ctypes.Structure):

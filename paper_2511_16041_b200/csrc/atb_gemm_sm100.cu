@@ -119,6 +119,10 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
     __syncthreads();
     tcgen05_fence_after_sync();
     const uint32_t tmem_base = misc_gen[0];
+#ifdef ATB_PROFILE
+    const long long prof_c0 = clock64();
+    const uint64_t prof_t0 = global_timer_ns();
+#endif
 
     const int total_items = p.m_tiles * p.n_tiles * (SPLIT ? p.splits : 1);
 
@@ -326,7 +330,9 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
                 dst_base = deq_base + rd.buf() * C::GPS * C::GROUP_BYTES;
                 row_base = 0;
             }
+#ifndef ATB_PROFILE_SKIP_DEQUANT    // diagnostic: the pipeline without the conversion work (results are wrong)
             dequant_slab<C>(ln, raw, raw + C::RAW_MANT_BYTES, scale_lut, dst_base, row_base, t, T_MA);
+#endif
             fence_proxy_async_smem();
             __syncwarp();
             if (lane == 0) {
@@ -344,6 +350,12 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
     }
     tcgen05_fence_before_sync();
     __syncthreads();
+#ifdef ATB_PROFILE
+    if (threadIdx.x == 0) {     // slots 0 / 4: nanoseconds and SM cycles of this CTA's main loop
+        atomicAdd(&g_wait_cycles[blockIdx.x & 255][0], static_cast<unsigned long long>(global_timer_ns() - prof_t0));
+        atomicAdd(&g_wait_cycles[blockIdx.x & 255][4], static_cast<unsigned long long>(clock64() - prof_c0));
+    }
+#endif
     if (warp == 1) {
         tcgen05_fence_after_sync();
         tmem_dealloc(tmem_base, static_cast<uint32_t>(C::TMEM_COLS));

@@ -82,9 +82,10 @@ def test_select_tiling_small_problem_prefers_more_tiles():
 
 
 def test_b200_refinements_can_be_switched_off():
-    """With the four refinements at 0 the selection is the paper's Eq. 12 times wave quantisation."""
+    """With the refinements at 0 the selection is the paper's Eq. 12 times wave quantisation."""
     hw = atb.atb_hw_params_b200()
     hw.mma_rows = 0; hw.load_latency_cycles = 0.0; hw.pair_efficiency = 0.0; hw.launch_seconds = 0.0
+    hw.tile_fixed_cycles = 0.0; hw.drain_cycles_per_column = 0.0; hw.pair_tile_cycles = 0.0
     _, scores = atb.atb_select_tiling(8192, 8192, 8192, hw)
     for s in scores:
         t = (s.t.T_MA, s.t.T_MC, s.t.T_K, s.t.T_N)
@@ -102,3 +103,26 @@ def test_select_tiling_errors():
     assert lib.atb_select_tiling(0, 8, 64, None, None, None, None) == 2
     with pytest.raises(atb.AtbError):
         atb.atb_score_tiling(atb.atb_hw_params_b200(), 64, (48, 128, 64, 128))
+
+
+def test_per_tile_costs():
+    """The per-tile terms: every tiling's compute bound grows with K (the fixed cost per output tile
+    is spread over more K-steps), the drain term touches only tilings whose accumulator is not
+    double-buffered, and the CTA-pair term only CTA-pair tilings."""
+    def bounds(K, **kw):
+        hw = atb.atb_hw_params_b200()
+        for n, v in kw.items():
+            setattr(hw, n, v)
+        _, scores = atb.atb_select_tiling(8192, 8192, K, hw)
+        return {(s.t.T_MA, s.t.T_MC, s.t.T_K, s.t.T_N): s.compute_bound_flops for s in scores}
+    b1, b4, b16 = bounds(1024), bounds(4096), bounds(16384)
+    assert all(b1[t] < b4[t] < b16[t] for t in b1)
+    no_drain = bounds(1024, drain_cycles_per_column=0.0)
+    for t in b1:
+        single = atb.atb_tiling_plan(*t).acc_buffers == 1
+        assert (no_drain[t] > b1[t]) == single, t
+    no_pair = bounds(1024, pair_tile_cycles=0.0)
+    for t in b1:
+        assert (no_pair[t] > b1[t]) == ((t[1], t[2], t[3]) == (256, 64, 512)), t
+    # shallow K: the CTA-pair tilings (one accumulator of 512 columns to drain per tile) are not chosen
+    assert tuple(atb.atb_select_tiling(8192, 8192, 1024)[0])[3] != 512
