@@ -79,8 +79,9 @@ atb_status_t atb_quantize_bfp16(const float* A_dev, int64_t M, int64_t K, int64_
  *   C_bf16_dev: bf16 C[M][ldc] row-major, ldc >= N, ldc % 8 == 0, 16-byte aligned (written).
  * Shapes: M >= 1 (any value), N >= 8 with N % 8 == 0, K >= 16 with K % 16 == 0.  Edge tiles in M, N and
  *         K are handled (TMA zero-fills loads past the edge and clips stores).
- * Tilings: T_MC in {128, 256}; T_N in {64, 128, 256, 512}; T_K in {64, 128};
- *          T_MA in {32, 64, 128, 256} with T_MA <= T_MC; (T_MC / 128) * T_N <= 512 (the FP32
+ * Tilings: T_MC in {128, 256, 384}; T_N in {64, 128, 256, 512}; T_K in {64, 128};
+ *          T_MA in {32, 64, 128, 256} dividing T_MC (rho = T_MC / T_MA is 1, 2, 3, 4, 6, 8 or 12:
+ *          T_MC = 384 gives the ratios that are not powers of two); (T_MC / 128) * T_N <= 512 (the FP32
  *          accumulator must fit the 512 TMEM columns); the shared-memory rings must fit 227 KB.
  *          atb_tiling_supported() tells in advance.
  * For fixed (T_MC, T_K, T_N) the result is bit-identical for every T_MA.

@@ -72,10 +72,10 @@ constexpr uint32_t ring_smem_bytes(uint32_t b_bytes, uint32_t group_bytes, uint3
 // Single-CTA kernel, tiling (T_MA, T_MC, T_K, T_N).
 constexpr RingPlan plan_single(int T_MA, int T_MC, int T_K, int T_N) {
     RingPlan pl;
-    if (!(T_MC == 128 || T_MC == 256)) return pl;
+    if (!(T_MC == 128 || T_MC == 256 || T_MC == 384)) return pl;
     if (!(T_N == 64 || T_N == 128 || T_N == 256 || T_N == 512)) return pl;
     if (!(T_K == 64 || T_K == 128)) return pl;
-    if (!(T_MA == 32 || T_MA == 64 || T_MA == 128 || T_MA == 256) || T_MA > T_MC) return pl;
+    if (!(T_MA == 32 || T_MA == 64 || T_MA == 128 || T_MA == 256) || T_MA > T_MC || T_MC % T_MA != 0) return pl;
     const int G = T_MC / 128;
     if (G * T_N > 512) return pl;
     const uint32_t b_bytes = T_K * T_N * 2, group_bytes = 128 * T_K * 2, raw_bytes = T_MA * T_K * 9 / 8;

@@ -573,6 +573,13 @@ extern "C" atb_status_t atb_gemm(int64_t M, int64_t N, int64_t K, int T_MA, int 
                 case 256: ATB_DISPATCH_TK(256, 256)
             }
             break;
+        case 384:                       // three 128-row groups: rho = 3, 6, 12
+            switch (T_MA) {
+                case 32:  ATB_DISPATCH_TK(32, 384)
+                case 64:  ATB_DISPATCH_TK(64, 384)
+                case 128: ATB_DISPATCH_TK(128, 384)
+            }
+            break;
     }
     return atb::fail(ATB_ERR_BAD_TILING, "no kernel for tiling (T_MA=%d, T_MC=%d, T_K=%d, T_N=%d)", T_MA, T_MC, T_K, T_N);
 }

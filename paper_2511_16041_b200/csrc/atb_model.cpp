@@ -120,7 +120,7 @@ atb_status_t atb_select_tiling(int64_t M, int64_t N, int64_t K, const atb_hw_par
     atb_hw_params_t hw;
     if (hw_in) hw = *hw_in; else atb_hw_params_b200(&hw);
 
-    static const int kMC[] = {128, 256}, kN[] = {64, 128, 256, 512}, kK[] = {64, 128}, kMA[] = {32, 64, 128, 256};
+    static const int kMC[] = {128, 256, 384}, kN[] = {64, 128, 256, 512}, kK[] = {64, 128}, kMA[] = {32, 64, 128, 256};
     std::vector<atb_tiling_score_t> all;
     for (int mc : kMC) for (int n : kN) for (int k : kK) for (int ma : kMA) {
         atb::GemmPlan plan;
@@ -174,8 +174,8 @@ atb_status_t atb_select_tiling(int64_t M, int64_t N, int64_t K, const atb_hw_par
     }
     std::stable_sort(all.begin(), all.end(), [](const atb_tiling_score_t& x, const atb_tiling_score_t& y) {
         if (x.feasible != y.feasible) return x.feasible > y.feasible;
-        // equal predictions (to 0.1 %): the smaller A buffer first - asymmetric buffering costs nothing there
-        if (std::fabs(x.predicted_flops - y.predicted_flops) > 1e-3 * x.predicted_flops) return x.predicted_flops > y.predicted_flops;
+        // equal predictions: the smaller A buffer first - asymmetric buffering costs nothing there
+        if (x.predicted_flops != y.predicted_flops) return x.predicted_flops > y.predicted_flops;
         return x.t.T_MA < y.t.T_MA;
     });
     if (all.empty() || !all.front().feasible) return atb::fail(ATB_ERR_BAD_SHAPE, "no supported tiling is feasible");

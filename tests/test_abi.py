@@ -42,7 +42,9 @@ def test_tiling_supported_rules():
     ok = atb.atb_tiling_supported
     assert ok(64, 128, 64, 128) and ok(128, 256, 64, 256) and ok(256, 256, 64, 256) and ok(32, 256, 64, 256)
     assert not ok(256, 128, 64, 128)          # T_MA > T_MC
-    assert not ok(64, 192, 64, 128)           # T_MC not 128 / 256
+    assert not ok(64, 192, 64, 128)           # T_MC not 128 / 256 / 384
+    assert ok(64, 384, 64, 128) and ok(128, 384, 64, 128) and ok(32, 384, 128, 64)   # rho = 6, 3, 12
+    assert not ok(256, 384, 64, 128) and not ok(128, 384, 64, 256)   # T_MA must divide T_MC; 3 x 256 columns > TMEM
     assert not ok(64, 128, 32, 128)           # T_K
     assert not ok(64, 128, 64, 96)            # T_N
     assert ok(128, 256, 64, 512) and ok(32, 256, 64, 512) and not ok(128, 256, 128, 512)   # CTA-pair tilings
@@ -79,11 +81,11 @@ def test_ring_plans_fit_the_budgets():
     barrier layout (lcm of depth and group count, see test_ring_protocol.py) stays small."""
     import math
     n = 0
-    for mc in (128, 256):
+    for mc in (128, 256, 384):
         for tn in (64, 128, 256, 512):
             for tk in (64, 128):
                 for ma in (32, 64, 128, 256):
-                    if ma > mc or not atb.atb_tiling_supported(ma, mc, tk, tn):
+                    if ma > mc or mc % ma or not atb.atb_tiling_supported(ma, mc, tk, tn):
                         continue
                     p = atb.atb_tiling_plan(ma, mc, tk, tn)
                     n += 1

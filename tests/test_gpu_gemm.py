@@ -16,8 +16,8 @@ from tests.gpu_util import run_gemm, dev, planes_to_dev, bf16_bits_to_dev, bf16_
 
 pytestmark = pytest.mark.gpu
 
-ALL_TILINGS = [(ma, mc, k, n) for mc in (128, 256) for n in (64, 128, 256, 512) for k in (64, 128)
-               for ma in (32, 64, 128, 256) if ma <= mc]
+ALL_TILINGS = [(ma, mc, k, n) for mc in (128, 256, 384) for n in (64, 128, 256, 512) for k in (64, 128)
+               for ma in (32, 64, 128, 256) if ma <= mc and mc % ma == 0]
 
 
 def supported():
@@ -69,6 +69,24 @@ def test_atb_invariance_bitwise_across_T_MA():
             if ref is None:
                 ref = Cg
             assert np.array_equal(Cg, ref), (ma, mc, k, n)
+
+
+def test_rho_that_is_not_a_power_of_two():
+    """T_MC = 384 (three 128-row groups): rho = 3, 6 and 12 (the paper's Table 2 uses rho = 6).  Several
+    tiles and ragged tails; bitwise equal across T_MA like every other (T_MC, T_K, T_N)."""
+    M, N, K = 1000, 392, 1104
+    A = inputs.make_A("normal", M, K)
+    Bb = inputs.make_B_bits(K, N)
+    mant, exp = oracle.quantize_bfp16(A)
+    for (tk, tn) in [(64, 128), (64, 64), (128, 128)]:
+        ref = None
+        for ma in (128, 64, 32):
+            if not atb.atb_tiling_supported(ma, 384, tk, tn):
+                continue
+            Cg = _check(mant, exp, Bb, (ma, 384, tk, tn))
+            ref = Cg if ref is None else ref
+            assert np.array_equal(Cg, ref), (ma, tk, tn)
+        assert ref is not None
 
 
 def test_small_integer_matrices_exact():

@@ -92,8 +92,8 @@ def test_b200_refinements_can_be_switched_off():
         if (t[1], t[3]) == (256, 512):
             continue                                   # pair tilings are scored per CTA
         ref = atb.atb_score_tiling(hw, 8192, t)
-        tiles = (8192 // t[1]) * (8192 // t[3])
-        useful = tiles / (math.ceil(tiles / 148) * 148)
+        tiles = math.ceil(8192 / t[1]) * math.ceil(8192 / t[3])       # edge tiles compute padding
+        useful = 8192 * 8192 / (math.ceil(tiles / 148) * 148 * t[1] * t[3])
         want = min(ref.mem_bound_flops, ref.compute_bound_flops * useful)
         assert math.isclose(s.predicted_flops, want, rel_tol=1e-12), t
 

@@ -150,11 +150,11 @@ def simulate(n_raw, n_deq, groups, run, n_slabs, seed, lcm_bars=True, group_warp
 
 
 def all_plans():
-    for mc in (128, 256):
+    for mc in (128, 256, 384):
         for tn in (64, 128, 256, 512):
             for tk in (64, 128):
                 for ma in (32, 64, 128, 256):
-                    if ma > mc or not atb.atb_tiling_supported(ma, mc, tk, tn):
+                    if ma > mc or mc % ma or not atb.atb_tiling_supported(ma, mc, tk, tn):
                         continue
                     p = atb.atb_tiling_plan(ma, mc, tk, tn)
                     pair = (mc, tk, tn) == (256, 64, 512)
