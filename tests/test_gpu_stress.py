@@ -69,3 +69,13 @@ def test_run_to_run_bitwise_determinism(tiling):
     got = bf16_dev_to_bits(ref.view(torch.bfloat16)[torch.from_numpy(rows).to(dev())])
     bad, ratio = oracle.check_tolerance(got, Cr, S)
     assert bad == 0 and ratio < 0.75, (tiling, bad, ratio)
+
+
+def test_calibration_measures_and_fits_on_this_gpu(tmp_path):
+    """The calibration tool end to end on two small shapes and a handful of tilings."""
+    from paper_2511_16041_b200 import calibrate
+    tilings = [(128, 256, 64, 256), (64, 256, 64, 256), (128, 128, 64, 256), (128, 256, 64, 128), (128, 256, 64, 512)]
+    records = calibrate.measure([(2048, 2048, 2048), (1024, 4096, 1024)], tilings, reps=3)
+    assert len(records) == 10 and all(r["tflops"] > 10 for r in records)
+    values, ev = calibrate.fit(records, {"a_bytes": (3.0, 3.6), "load_latency_cycles": (1200.0, 2000.0)})
+    assert set(values) == {"a_bytes", "load_latency_cycles"} and 0.5 < ev["pick_quality_mean"] <= 1.0
