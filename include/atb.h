@@ -141,6 +141,23 @@ atb_status_t atb_gemm_splitk_noalloc(int64_t M, int64_t N, int64_t K, int T_MA, 
                                      const void* B_bf16_dev, int64_t ldb,
                                      void* C_bf16_dev, int64_t ldc, int splits, void* stream);
 
+/* atb_gemm with a quantising epilogue: C is written in BFP16 (the C format of the all-BFP16
+ * configurations of Section 6.1, Table 2), in the very layout atb_quantize_bfp16 produces for an
+ * M x N matrix, so that C can be the A operand of the next atb_gemm (its blocks run along N, the K of
+ * that product).  Every block of 8 consecutive columns of a row is quantised from the FP32
+ * accumulators with the rule of atb_quantize_bfp16 (E = exponent of the block's largest magnitude,
+ * m = RNE(x / 2^(E-133)) saturated to +-127): the result equals atb_quantize_bfp16 applied to the FP32
+ * accumulators bit for bit.
+ *   C_mant_dev: int8 [M][N] row-major (contiguous), 16-byte aligned (written);
+ *   C_exp_dev:  exponent plane of atb_bfp16_exp_bytes(M, N) bytes, 16-byte aligned (written; the
+ *               plane's padding rows get exponent 0).
+ * Shapes: M >= 1, N % 16 == 0, K % 16 == 0.  Tilings: T_K = 64, T_MC in {128, 256}, T_N in {128, 256},
+ * T_MA in {64, 128}.  Other arguments, conventions and errors as for atb_gemm. */
+atb_status_t atb_gemm_bfp16_out(int64_t M, int64_t N, int64_t K, int T_MA, int T_MC, int T_K, int T_N,
+                                const int8_t* A_mant_dev, const uint8_t* A_exp_dev,
+                                const void* B_bf16_dev, int64_t ldb,
+                                int8_t* C_mant_dev, uint8_t* C_exp_dev, void* stream);
+
 /* 1 if atb_gemm accepts the tiling (kernel exists, TMEM and shared-memory budgets met), else 0.
  * Host only; touches no device. */
 int atb_tiling_supported(int T_MA, int T_MC, int T_K, int T_N);

@@ -68,7 +68,7 @@ class Tiling(NamedTuple):
 
 EXPORTED_SYMBOLS = [
     "atb_status_string", "atb_last_error_message", "atb_bfp16_mant_bytes", "atb_bfp16_exp_bytes",
-    "atb_quantize_bfp16", "atb_gemm", "atb_gemm_splitk", "atb_gemm_splitk_workspace_bytes", "atb_select_splits",
+    "atb_quantize_bfp16", "atb_gemm", "atb_gemm_bfp16_out", "atb_gemm_splitk", "atb_gemm_splitk_workspace_bytes", "atb_select_splits",
     "atb_gemm_splitk_noalloc",
     "atb_tiling_supported", "atb_tiling_plan", "atb_device_status",
     "atb_hw_params_b200", "atb_hw_params_xdna2", "atb_score_tiling", "atb_select_tiling",
@@ -96,6 +96,8 @@ def load_library():
     lib.atb_quantize_bfp16.argtypes = [vp, i64, i64, i64, vp, vp, vp]
     lib.atb_gemm.restype = ci
     lib.atb_gemm.argtypes = [i64, i64, i64, ci, ci, ci, ci, vp, vp, vp, i64, vp, i64, vp]
+    lib.atb_gemm_bfp16_out.restype = ci
+    lib.atb_gemm_bfp16_out.argtypes = [i64, i64, i64, ci, ci, ci, ci, vp, vp, vp, i64, vp, vp, vp]
     lib.atb_gemm_splitk.restype = ci
     lib.atb_gemm_splitk.argtypes = [i64, i64, i64, ci, ci, ci, ci, vp, vp, vp, i64, vp, i64, ci, vp, ctypes.c_size_t, vp]
     lib.atb_gemm_splitk_noalloc.restype = ci
@@ -226,6 +228,21 @@ def atb_gemm_splitk(M, N, K, T_MA, T_MC, T_K, T_N, A_mant, A_exp, B, splits, wor
                                           ldb, _dev_ptr(C), ldc, splits, _dev_ptr(workspace),
                                           workspace.numel() * workspace.element_size(), _stream_ptr(stream)))
     return C
+
+
+def atb_gemm_bfp16_out(M, N, K, T_MA, T_MC, T_K, T_N, A_mant, A_exp, B, C_mant=None, C_exp=None, ldb=None, stream=None):
+    """``C = dequant(A) @ B`` written as BFP16 planes (quantising epilogue).  Returns ``(C_mant, C_exp)``:
+    an int8 ``[M, N]`` tensor and the exponent plane, both usable as the A operand of the next GEMM."""
+    import torch
+    if C_mant is None:
+        C_mant = torch.empty((M, N), dtype=torch.int8, device=B.device)
+    if C_exp is None:
+        C_exp = torch.empty(atb_bfp16_exp_bytes(M, N), dtype=torch.uint8, device=B.device)
+    if ldb is None:
+        ldb = B.stride(0)
+    _check(load_library().atb_gemm_bfp16_out(M, N, K, T_MA, T_MC, T_K, T_N, _dev_ptr(A_mant), _dev_ptr(A_exp), _dev_ptr(B),
+                                             ldb, _dev_ptr(C_mant), _dev_ptr(C_exp), _stream_ptr(stream)))
+    return C_mant, C_exp
 
 
 NOALLOC_SCRATCH_BYTES = 64 * 1024 * 1024

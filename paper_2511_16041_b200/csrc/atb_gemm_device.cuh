@@ -169,6 +169,8 @@ struct GemmParams {
     __nv_bfloat16* C;
     int m_tiles, n_tiles, k_steps;
     unsigned int* error_flag;
+    uint8_t* C_exp;      // quantising epilogue: exponent plane of C [ceil(N/64)][c_exp_rows][8]
+    int64_t c_exp_rows;  // roundup(M, 32)
     int splits;          // split-K: each output tile is computed as `splits` partial tiles over K ranges
     int m_pad;           // split-K: rows per split in the FP32 workspace (m_tiles * T_MC)
 };

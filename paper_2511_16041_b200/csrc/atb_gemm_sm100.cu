@@ -25,6 +25,7 @@
 #include <cmath>
 
 #include "atb_gemm_device.cuh"
+#include "bfp16_block.cuh"
 
 namespace {
 
@@ -63,7 +64,9 @@ struct Cfg {
 };
 
 // ---------------------------------------------------------------------------------------------
-template <int T_MA, int T_MC, int T_K, int T_N, bool SPLIT>
+// SPLIT: partial tiles over K ranges go to an FP32 workspace.  QOUT: C is written as BFP16 planes
+// (the C format of the paper's all-BFP16 configurations, Section 6.1) by a quantising epilogue.
+template <int T_MA, int T_MC, int T_K, int T_N, bool SPLIT, bool QOUT = false>
 __global__ void __launch_bounds__(kThreads, 1)
 atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_constant__ CUtensorMap tm_exp,
                 const __grid_constant__ CUtensorMap tm_b, const __grid_constant__ CUtensorMap tm_c,
@@ -263,6 +266,56 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
                             tma_store_commit();
                         }
                     }
+                } else if (QOUT) {
+                    // BFP16 C: a thread owns one row; per 64 columns it quantises 8 blocks of 8 FP32
+                    // accumulators (exactly as atb_quantize_bfp16 would), stages the 64 mantissa bytes
+                    // of its row in a 32 x 64-byte box (64-byte swizzle) for one TMA store, and writes
+                    // the 8 exponents - contiguous in the exponent plane, rows adjacent - directly.
+                    const uint32_t my_row64 = box + lane * 64;
+                    const uint32_t sw64 = static_cast<uint32_t>(lane >> 1) & 3u;
+                    const int64_t row = static_cast<int64_t>(row0) + lane;
+#pragma unroll 1
+                    for (int c = 0; c < T_N / 64; ++c) {
+                        if (lane == 0) tma_store_wait_read<0>();
+                        __syncwarp();
+                        uint32_t e_lo = 0, e_hi = 0;
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            uint32_t v[32];
+                            tmem_ld_32x32b_x32(t_addr + c * 64 + h * 32, v);
+                            tmem_ld_wait();
+                            uint32_t m8[8];
+#pragma unroll
+                            for (int b = 0; b < 4; ++b) {
+                                float x[8];
+#pragma unroll
+                                for (int e = 0; e < 8; ++e) x[e] = __uint_as_float(v[b * 8 + e]);
+                                uint32_t pk[2];
+                                const uint32_t E = static_cast<uint32_t>(bfp16::quantize_block8(x, pk));
+                                m8[2 * b] = pk[0];
+                                m8[2 * b + 1] = pk[1];
+                                if (h == 0) e_lo |= E << (8 * b); else e_hi |= E << (8 * b);
+                            }
+#pragma unroll
+                            for (int j = 0; j < 2; ++j)
+                                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(my_row64 + ((static_cast<uint32_t>(h * 2 + j) ^ sw64) << 4)),
+                                             "r"(m8[4 * j]), "r"(m8[4 * j + 1]), "r"(m8[4 * j + 2]), "r"(m8[4 * j + 3]) : "memory");
+                        }
+                        fence_proxy_async_smem();
+                        __syncwarp();
+                        const int64_t col = static_cast<int64_t>(col0) + c * 64;
+                        if (col < p.N) {
+                            if (lane == 0 && row0 < p.M) {
+                                tma_store_2d(&tm_c, box, static_cast<int>(col), row0);
+                                tma_store_commit();
+                            }
+                            if (row < p.c_exp_rows) {       // rows of the plane's padding get exponent 0
+                                const bool real = row < p.M;
+                                uint2 ev = make_uint2(real ? e_lo : 0u, real ? e_hi : 0u);
+                                *reinterpret_cast<uint2*>(p.C_exp + ((col >> 6) * p.c_exp_rows + row) * 8) = ev;
+                            }
+                        }
+                    }
                 } else {
 #pragma unroll 1
                 for (int c = 0; c < T_N / 64; ++c) {
@@ -367,10 +420,11 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
 // ---------------------------------------------------------------------------------------------
 // SPLIT = false: Cout is bf16 C[M][ldc].  SPLIT = true: Cout is the FP32 workspace
 // [splits][m_tiles * T_MC][N] that receives one partial tile per (tile, split).
-template <int T_MA, int T_MC, int T_K, int T_N, bool SPLIT = false>
+template <int T_MA, int T_MC, int T_K, int T_N, bool SPLIT = false, bool QOUT = false>
 atb_status_t launch(const atb::GemmPlan& plan, int64_t M, int64_t N, int64_t K, const int8_t* mant,
                     const uint8_t* exp, const void* B, int64_t ldb, void* Cout, int64_t ldc,
-                    int num_sms, unsigned int* error_flag, cudaStream_t stream, int splits = 1) {
+                    int num_sms, unsigned int* error_flag, cudaStream_t stream, int splits = 1,
+                    uint8_t* C_exp = nullptr) {
     CUtensorMap tm_mant, tm_exp, tm_b, tm_c;
     const int64_t M_pad = atb::round_up(M, 32);
     if (!make_map_2d(&tm_mant, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, mant, K, M, K, T_K, T_MA, CU_TENSOR_MAP_SWIZZLE_NONE))
@@ -384,6 +438,9 @@ atb_status_t launch(const atb::GemmPlan& plan, int64_t M, int64_t N, int64_t K, 
     if (SPLIT) {
         if (!make_map_2d(&tm_c, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, Cout, N, splits * m_pad, N * 4, 32, 32, CU_TENSOR_MAP_SWIZZLE_128B))
             return atb::fail(ATB_ERR_CUDA, "cuTensorMapEncodeTiled failed for the split-K workspace");
+    } else if (QOUT) {
+        if (!make_map_2d(&tm_c, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Cout, N, M, ldc, 64, 32, CU_TENSOR_MAP_SWIZZLE_64B))
+            return atb::fail(ATB_ERR_CUDA, "cuTensorMapEncodeTiled failed for the mantissa plane of C");
     } else if (!make_map_2d(&tm_c, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Cout, N, M, ldc * 2, 64, 32, CU_TENSOR_MAP_SWIZZLE_128B)) {
         return atb::fail(ATB_ERR_CUDA, "cuTensorMapEncodeTiled failed for C");
     }
@@ -397,8 +454,10 @@ atb_status_t launch(const atb::GemmPlan& plan, int64_t M, int64_t N, int64_t K, 
     p.error_flag = error_flag;
     p.splits = splits;
     p.m_pad = static_cast<int>(m_pad);
+    p.C_exp = C_exp;
+    p.c_exp_rows = M_pad;
 
-    auto kernel = atb_gemm_kernel<T_MA, T_MC, T_K, T_N, SPLIT>;
+    auto kernel = atb_gemm_kernel<T_MA, T_MC, T_K, T_N, SPLIT, QOUT>;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(plan.smem_bytes));
     if (e != cudaSuccess) return atb::fail(ATB_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
     const int64_t items = static_cast<int64_t>(p.m_tiles) * p.n_tiles * splits;
@@ -659,6 +718,43 @@ atb_status_t gemm_splitk_with_workspace(int64_t M, int64_t N, int64_t K, int T_M
 }
 
 }  // namespace atb
+
+// ---------------------------------------------------------------------------------------------
+// GEMM with a quantising epilogue: C in BFP16
+// ---------------------------------------------------------------------------------------------
+extern "C" atb_status_t atb_gemm_bfp16_out(int64_t M, int64_t N, int64_t K, int T_MA, int T_MC, int T_K, int T_N,
+                                           const int8_t* A_mant_dev, const uint8_t* A_exp_dev,
+                                           const void* B_bf16_dev, int64_t ldb,
+                                           int8_t* C_mant_dev, uint8_t* C_exp_dev, void* stream) {
+    atb::clear_error();
+    if (!A_mant_dev || !A_exp_dev || !B_bf16_dev || !C_mant_dev || !C_exp_dev)
+        return atb::fail(ATB_ERR_NULL_POINTER, "all device pointers must be non-NULL");
+    if (M < 1 || N < 16 || N % 16 != 0 || K < 16 || K % 16 != 0 || M > (1ll << 30) || N > (1ll << 30) || K > (1ll << 30))
+        return atb::fail(ATB_ERR_BAD_SHAPE, "need M >= 1, N %% 16 == 0, K %% 16 == 0 (got %lld, %lld, %lld)", (long long)M, (long long)N, (long long)K);
+    if (ldb < N || ldb % 8 != 0) return atb::fail(ATB_ERR_BAD_SHAPE, "ldb=%lld must be >= N and a multiple of 8", (long long)ldb);
+    if (!splitk_tiling_ok(T_MA, T_MC, T_K, T_N))
+        return atb::fail(ATB_ERR_BAD_TILING, "the quantising epilogue supports T_K = 64, T_MC in {128, 256}, T_N in {128, 256}, T_MA in {64, 128}");
+    if (!atb::aligned16(A_mant_dev) || !atb::aligned16(A_exp_dev) || !atb::aligned16(B_bf16_dev) || !atb::aligned16(C_mant_dev) ||
+        !atb::aligned16(C_exp_dev))
+        return atb::fail(ATB_ERR_MISALIGNED, "all device pointers must be 16-byte aligned");
+    atb::GemmPlan plan;
+    if (!atb::plan_gemm(T_MA, T_MC, T_K, T_N, &plan))
+        return atb::fail(ATB_ERR_BAD_TILING, "tiling (T_MA=%d, T_MC=%d, T_K=%d, T_N=%d) is not supported", T_MA, T_MC, T_K, T_N);
+    DeviceInfo* dev = nullptr;
+    atb_status_t st_dev = device_info(&dev);
+    if (st_dev != ATB_OK) return st_dev;
+    if (dev->cc_major != 10 || dev->cc_minor != 0)
+        return atb::fail(ATB_ERR_UNSUPPORTED_DEVICE, "compute capability %d.%d; this library runs on 10.0 only", dev->cc_major, dev->cc_minor);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+#define ATB_QOUT_CASE(TMA_, TMC_, TN_)                                                                       \
+    if (T_MA == TMA_ && T_MC == TMC_ && T_N == TN_)                                                          \
+        return launch<TMA_, TMC_, 64, TN_, false, true>(plan, M, N, K, A_mant_dev, A_exp_dev, B_bf16_dev, ldb, \
+                                                        C_mant_dev, N, dev->num_sms, dev->error_flag, st, 1, C_exp_dev);
+    ATB_QOUT_CASE(64, 128, 128) ATB_QOUT_CASE(128, 128, 128) ATB_QOUT_CASE(64, 128, 256) ATB_QOUT_CASE(128, 128, 256)
+    ATB_QOUT_CASE(64, 256, 128) ATB_QOUT_CASE(128, 256, 128) ATB_QOUT_CASE(64, 256, 256) ATB_QOUT_CASE(128, 256, 256)
+#undef ATB_QOUT_CASE
+    return atb::fail(ATB_ERR_BAD_TILING, "no kernel for tiling (T_MA=%d, T_MC=%d, T_K=%d, T_N=%d)", T_MA, T_MC, T_K, T_N);
+}
 
 extern "C" atb_status_t atb_gemm_splitk(int64_t M, int64_t N, int64_t K, int T_MA, int T_MC, int T_K, int T_N,
                                         const int8_t* A_mant_dev, const uint8_t* A_exp_dev,

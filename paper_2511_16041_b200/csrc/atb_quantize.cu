@@ -11,16 +11,13 @@
 #include <cstdint>
 
 #include "atb_internal.h"
+#include "bfp16_block.cuh"
 
 namespace {
 
 constexpr int kTileRows = 32;
 constexpr int kTileBlocks = 32;   // blocks of 8 columns per tile row
 constexpr int kThreads = 256;
-
-__device__ __forceinline__ float pow2f(int e) {   // 2^e for e in [-126, 127]
-    return __uint_as_float(static_cast<uint32_t>(e + 127) << 23);
-}
 
 __global__ void __launch_bounds__(kThreads)
 quantize_bfp16_kernel(const float* __restrict__ A, int64_t M, int64_t K, int64_t lda,
@@ -51,29 +48,8 @@ quantize_bfp16_kernel(const float* __restrict__ A, int64_t M, int64_t K, int64_t
     for (int i = 0; i < 4; ++i) {
         const int64_t m = m0 + warp * 4 + i;
         const float x[8] = {lo[i].x, lo[i].y, lo[i].z, lo[i].w, hi[i].x, hi[i].y, hi[i].z, hi[i].w};
-        // Largest magnitude as an integer compare of the bit patterns; NaNs do not take part.
-        uint32_t amax_bits = 0;
-#pragma unroll
-        for (int t = 0; t < 8; ++t) {
-            uint32_t b = __float_as_uint(x[t]) & 0x7FFFFFFFu;
-            if (b > 0x7F800000u) b = 0;
-            amax_bits = max(amax_bits, b);
-        }
-        int E = static_cast<int>(amax_bits >> 23);
-        E = min(E, 254);
-        // x / 2^(E-133) as two exact power-of-two multiplications (one factor alone would leave
-        // the fp32 range at both ends of E).
-        const int sh = 133 - E;
-        const int sa = sh >> 1, sb = sh - sa;
-        const float fa = pow2f(sa), fb = pow2f(sb);
-        uint32_t packed[2] = {0u, 0u};
-#pragma unroll
-        for (int t = 0; t < 8; ++t) {
-            const float q = (x[t] * fa) * fb;
-            int r = __float2int_rn(q);            // ties to even; NaN -> 0; +-Inf saturate
-            r = max(-127, min(127, r));
-            packed[t >> 2] |= (static_cast<uint32_t>(r) & 0xFFu) << (8 * (t & 3));
-        }
+        uint32_t packed[2];
+        const int E = bfp16::quantize_block8(x, packed);
         if (kb_ok && m < M)
             *reinterpret_cast<uint2*>(mant + m * K + kb * 8) = make_uint2(packed[0], packed[1]);
         s_exp[lane >> 3][warp * 4 + i][lane & 7] = (kb_ok && m < M) ? static_cast<uint8_t>(E) : 0;
