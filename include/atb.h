@@ -167,7 +167,7 @@ int atb_tiling_supported(int T_MA, int T_MC, int T_K, int T_N);
  * slabs of T_MA x T_K, and dequantised BF16 A in 128-row groups of T_K columns. */
 typedef struct {
     int n_b_stages;      /* depth of the B-tile ring                                              */
-    int n_raw_stages;    /* depth of the raw A-slab ring (a multiple of dequant_groups)           */
+    int n_raw_stages;    /* depth of the raw A-slab ring                                          */
     int n_a_groups;      /* depth of the dequantised-A ring, in 128-row groups                    */
     int dequant_groups;  /* groups the 16 dequantiser warps are split into; slabs take turns      */
     int acc_buffers;     /* T_MC x T_N FP32 accumulators resident in TMEM (1 or 2)                */

@@ -73,6 +73,9 @@ def test_argument_validation_needs_no_gpu():
     assert lib.atb_quantize_bfp16(None, 0, 64, 64, None, None, None) == 0       # empty: no-op
     assert lib.atb_gemm(128, 128, 64, 64, 128, 64, 128, None, None, None, 128, None, 128, None) == 1
     assert lib.atb_gemm(128, 128, 72, 64, 128, 64, 128, 16, 16, 16, 128, 16, 128, None) == 2       # K % 16
+    assert lib.atb_gemm_bfp16_out(128, 128, 64, 64, 128, 64, 128, 16, 16, 16, 128, None, 16, None) == 1   # NULL
+    assert lib.atb_gemm_bfp16_out(128, 136, 64, 64, 128, 64, 128, 16, 16, 16, 136, 16, 16, None) == 2     # N % 16
+    assert lib.atb_gemm_bfp16_out(128, 128, 64, 32, 128, 64, 128, 16, 16, 16, 128, 16, 16, None) == 3     # tiling
     assert atb.atb_last_error_message() != ""
 
 
