@@ -110,3 +110,32 @@ def test_argument_errors():
     assert lib.atb_gemm_bfp16_out(256, 256, 256, 32, 128, 64, 128, p, p, p, 256, p, p, None) == 3      # tiling
     assert lib.atb_gemm_bfp16_out(256, 256, 256, 64, 128, 64, 128, p, p, p, 256, None, p, None) == 1   # NULL
     assert lib.atb_gemm_bfp16_out(256, 256, 256, 64, 128, 64, 128, p, p, p, 256, p + 8, p, None) == 4  # alignment
+
+
+def test_full_size_headline_shape_sampled_rows():
+    """8192^3 in the benchmark's launch configuration: sampled rows of the BFP16 planes against the
+    quantiser on the kernel's FP32 accumulators (bit exact) and against the FP64 oracle GEMM."""
+    c = inputs.CONFIGS["cfg3_8192"]
+    M, N, K = c["M"], c["N"], c["K"]
+    A, Bb = inputs.make_config("cfg3_8192")
+    mant_d, plane_d = atb.atb_quantize_bfp16(torch.from_numpy(A).to(dev()))
+    Bd = bf16_bits_to_dev(Bb)
+    tiling = (128, 256, 64, 256)
+    rows = np.unique(np.concatenate([np.arange(0, M, 256), np.arange(255, M, 256),
+                                     np.random.default_rng(5).integers(0, M, 32)])).astype(np.int64)
+    rows_d = torch.from_numpy(rows).to(dev())
+    ws = torch.empty(atb.atb_gemm_splitk_workspace_bytes(M, N, tiling[1], 1) // 4, dtype=torch.float32, device=dev())
+    atb.atb_gemm_splitk(M, N, K, *tiling, mant_d, plane_d, Bd, 1, workspace=ws)
+    acc = ws.view(M, N)[rows_d].cpu().numpy()
+    del ws
+    Cm, Ce = atb.atb_gemm_bfp16_out(M, N, K, *tiling, mant_d, plane_d, Bd)
+    atb.atb_device_status()
+    got_m = Cm[rows_d].cpu().numpy()
+    got_e = atb.exp_plane_to_logical(Ce.cpu().numpy(), M, N)[rows]
+    want_m, want_e = oracle.quantize_bfp16(np.ascontiguousarray(acc))
+    assert np.array_equal(got_e, want_e) and np.array_equal(got_m, want_m)
+    mant_o, exp_o = oracle.quantize_bfp16(A[rows])
+    Cr, S = oracle.gemm(mant_o, exp_o, Bb)
+    half_step = np.repeat(np.ldexp(1.0, got_e.astype(np.int64) - 134), 8, axis=1)
+    q_err = np.where(np.abs(got_m.astype(np.int64)) == 127, 2.0 * half_step, half_step)
+    assert np.all(np.abs(oracle.dequantize(got_m, got_e) - Cr) <= q_err + S * 2.0 ** -12)
