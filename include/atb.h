@@ -158,6 +158,28 @@ atb_status_t atb_gemm_bfp16_out(int64_t M, int64_t N, int64_t K, int T_MA, int T
                                 const void* B_bf16_dev, int64_t ldb,
                                 int8_t* C_mant_dev, uint8_t* C_exp_dev, void* stream);
 
+/* The precision configurations the paper evaluates (Section 6.1, Table 2), with the BFP16 operand on
+ * the B side as the paper has it: the B tile stays in the core for the rho slabs of a K-step and is
+ * converted ONCE per K-step; the slabs of A stream through it (Section 3.1).
+ *   config 1: A in BF16 (streamed as is), B in BFP16, C in BF16;
+ *   config 2: A, B and C in BFP16 (the paper's configurations 2 and 3; accumulation is FP32 here).
+ * Operands (device memory, 16-byte aligned, caller-owned):
+ *   A_dev:       config 1: bf16 A[M][lda] row-major (lda >= K, lda % 8 == 0), A_exp_dev = NULL;
+ *                config 2: int8 mantissas [M][K] with their exponent plane in A_exp_dev (the planes
+ *                of atb_quantize_bfp16; lda is ignored);
+ *   Bt_mant_dev, Bt_exp_dev: the BFP16 planes of B TRANSPOSED, i.e. of the N x K matrix whose row n is
+ *                column n of B, as atb_quantize_bfp16 produces them for that matrix - the blocks of 8
+ *                run along K, as the paper's do;
+ *   C_dev:       config 1: bf16 C[M][ldc] (ldc >= N, ldc % 8 == 0), C_exp_dev = NULL;
+ *                config 2: int8 mantissas [M][N] and the exponent plane in C_exp_dev, as
+ *                atb_gemm_bfp16_out writes them (ldc is ignored).
+ * Shapes: M >= 1, N % 16 == 0, K % 16 == 0.  The tiling is fixed: T_MA = 128, T_MC = 256, T_K = 64,
+ * T_N = 256.  Errors as for atb_gemm; an unknown config is ATB_ERR_BAD_TILING. */
+atb_status_t atb_gemm_config(int config, int64_t M, int64_t N, int64_t K,
+                             const void* A_dev, const uint8_t* A_exp_dev, int64_t lda,
+                             const int8_t* Bt_mant_dev, const uint8_t* Bt_exp_dev,
+                             void* C_dev, uint8_t* C_exp_dev, int64_t ldc, void* stream);
+
 /* 1 if atb_gemm accepts the tiling (kernel exists, TMEM and shared-memory budgets met), else 0.
  * Host only; touches no device. */
 int atb_tiling_supported(int T_MA, int T_MC, int T_K, int T_N);

@@ -8,7 +8,8 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libatb.so")
-SOURCES = ["atb_status.cpp", "atb_model.cpp", "atb_quantize.cu", "atb_gemm_sm100.cu", "atb_gemm_pair_sm100.cu"]
+SOURCES = ["atb_status.cpp", "atb_model.cpp", "atb_quantize.cu", "atb_gemm_sm100.cu", "atb_gemm_pair_sm100.cu",
+           "atb_gemm_cfg_sm100.cu"]
 HEADERS = ["atb_internal.h", "sm100_ptx.cuh", "atb_gemm_device.cuh", "bfp16_block.cuh"]
 
 

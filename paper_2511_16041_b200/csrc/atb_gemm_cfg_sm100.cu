@@ -1,0 +1,389 @@
+// atb_gemm_config: the precision configurations the paper evaluates (Section 6.1, Table 2), sm_100a.
+//
+//   Config 1     A in BF16 (streamed), B in BFP16 (resident), C in BF16
+//   Config 2/3   A, B and C in BFP16 (FP32 accumulation here for both)
+//
+// In both the operand that stays in the core across the rho slabs of a K-step is the BFP16 B tile,
+// exactly as in the paper: it is converted ONCE per K-step and every slab of A is multiplied against
+// the converted copy (Section 3.1; the "converted copy" term of the buffer column of Table 2).
+// B is given as the BFP16 planes of its transpose (N x K, blocks of 8 along K), which is the
+// K-major form the UMMA takes for its N-side operand; the dequantised tile is laid out like the
+// dequantised A slabs of atb_gemm_kernel and read with a K-major descriptor.
+//
+// Fixed tiling: T_MA = 128, T_MC = 256, T_K = 64, T_N = 256 (rho = 2).  Units of 128 rows x 64 K
+// flow through the rings: two A units and two B units per K-step.
+//   warp 0      TMA producer of raw B units (mantissa box + exponent box)
+//   warp 22     TMA producer of A units: raw BFP16 (config 2) or BF16 straight into the operand
+//               ring, K-major with the 128-byte swizzle (config 1: nothing to convert)
+//   warp 1      UMMA issuer: 128 x 256 x 16, both operands K-major
+//   warps 2-5   epilogue (BF16 or quantising BFP16, shared with atb_gemm_kernel)
+//   warps 6-21  dequantisers: 4 groups of 4 warps; config 1: all four on the B stream; config 2:
+//               two on the A stream, two on the B stream
+// Barriers, bounded waits and the ring cursors are those of atb_gemm_kernel.
+#include "atb_gemm_device.cuh"
+
+namespace {
+
+__device__ unsigned int g_cfg_error_flag = 0;
+
+struct CfgDq {                                         // what dequant_slab needs to know
+    static constexpr int SLOTS_PER_ROW = 4, SLOTS = 128 * 4, GROUP_THREADS = 128;
+    static constexpr int DQ_ITERS = 4, ROWS_PER_ITER = 32;
+    static constexpr uint32_t KHALF_BYTES = 128 * 128, GROUP_BYTES = 128 * 128;
+};
+
+template <bool A_Q>
+struct CfgK {
+    static constexpr int T_K = 64, T_N = 256;
+    static constexpr uint32_t UNIT_BYTES = 128 * 128;                 // 128 rows x 64 bf16
+    static constexpr uint32_t RAW_MANT_BYTES = 128 * 64, RAW_BYTES = RAW_MANT_BYTES + 128 * 8;
+    static constexpr int DA = A_Q ? 2 : 0, DB = 4 - DA;               // dequantiser groups per stream
+    static constexpr int NA = 4;                                      // operand units of A in shared memory
+    static constexpr int NAR = A_Q ? 4 : 0;                           // raw A units
+    // A converted B tile (two units) is held for a whole K-step, by both row groups: three tiles
+    // where shared memory allows (config 1), two otherwise.
+    static constexpr int NB = A_Q ? 4 : 6, NBR = 4;                   // operand / raw units of B
+    static constexpr int LB = ring_bars(NB, DB), LBR = ring_bars(NBR, DB);   // barrier pairs of the B rings
+    static constexpr int GROUP_WARPS = 4;
+    static constexpr uint32_t SMEM_BYTES = 1024u + (NA + NB) * UNIT_BYTES + (NAR + NBR) * RAW_BYTES + 1024u +
+                                           4u * kEpilogueBoxBytes + 8u * (2 * NA + 2 * NAR + 2 * LB + 2 * LBR + 4) + 16u + 1024u;
+    static_assert(NB % 2 == 0 && LB % 2 == 0, "B tiles are pairs of units");
+    static_assert(SMEM_BYTES <= kSmemBudget, "shared memory");
+};
+
+struct CfgParams {
+    int64_t M, N, K;
+    int m_tiles, n_tiles, k_steps;
+    uint8_t* C_exp;
+    int64_t c_exp_rows;
+    unsigned int* error_flag;
+};
+
+// One dequantiser group on one BFP16 stream: units arrive in ring order, the group takes every D-th.
+template <int D, int NR, int ND>
+__device__ __forceinline__ void dequant_stream(const Ctx& cx, int my, int64_t units, int t, int lane, uint32_t raw_full,
+                                               uint32_t raw_empty, uint32_t deq_full, uint32_t deq_empty,
+                                               uint32_t raw_base, uint32_t deq_base, uint32_t scale_lut, unsigned code) {
+    constexpr uint32_t kRaw = 128 * 64 + 128 * 8, kMant = 128 * 64;
+    const DequantLane<CfgDq> ln(t, 128);
+    Cursor<NR, ring_bars(NR, D)> rr;
+    Cursor<ND, ring_bars(ND, D)> rd;
+    rr.start_at(my);
+    rd.start_at(my);
+    for (int64_t n = my; n < units; n += D) {
+        if (!wait_bar(cx, raw_full + 8 * rr.bar, rr.phase, code | 1u)) break;
+        if (!wait_bar(cx, deq_empty + 8 * rd.freed_bar(), rd.freed_parity(), code | 2u)) break;
+        const uint32_t raw = raw_base + rr.buf() * kRaw;
+        dequant_slab<CfgDq>(ln, raw, raw + kMant, scale_lut, deq_base + rd.buf() * CfgDq::GROUP_BYTES, 0, t, 128);
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+            mbar_arrive(deq_full + 8 * rd.bar);
+            mbar_arrive(raw_empty + 8 * rr.bar);
+        }
+        rr.template advance<D>();
+        rd.template advance<D>();
+    }
+}
+
+template <bool A_Q, bool C_Q>
+__global__ void __launch_bounds__(kThreads, 1)
+atb_gemm_cfg_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_a_exp,
+                    const __grid_constant__ CUtensorMap tm_b, const __grid_constant__ CUtensorMap tm_b_exp,
+                    const __grid_constant__ CUtensorMap tm_c, const CfgParams p) {
+    using C = CfgK<A_Q>;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* const smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+    const uint32_t a_base = smem_base;                                           // operand units of A
+    const uint32_t b_base = a_base + C::NA * C::UNIT_BYTES;                      // operand units of B
+    const uint32_t a_raw_base = b_base + C::NB * C::UNIT_BYTES;
+    const uint32_t b_raw_base = a_raw_base + C::NAR * C::RAW_BYTES;
+    constexpr uint32_t stage_off = ((C::NA + C::NB) * C::UNIT_BYTES + (C::NAR + C::NBR) * C::RAW_BYTES + 1023u) & ~1023u;
+    const uint32_t bar_base = smem_base + stage_off + 4u * kEpilogueBoxBytes;
+    const uint32_t a_full = bar_base, a_empty = a_full + 8 * C::NA;
+    const uint32_t ar_full = a_empty + 8 * C::NA, ar_empty = ar_full + 8 * C::NAR;
+    const uint32_t b_full = ar_empty + 8 * C::NAR, b_empty = b_full + 8 * C::LB;
+    const uint32_t br_full = b_empty + 8 * C::LB, br_empty = br_full + 8 * C::LBR;
+    const uint32_t acc_full = br_empty + 8 * C::LBR, acc_empty = acc_full + 8 * 2;
+    const uint32_t misc = acc_empty + 8 * 2;                 // [0]: TMEM base, [1]: abort flag
+    const uint32_t scale_lut = misc + 16;
+    volatile uint32_t* const misc_gen = reinterpret_cast<volatile uint32_t*>(smem_gen + (misc - smem_base));
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    Ctx cx{misc_gen + 1, p.error_flag};
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < C::NA; ++i) { mbar_init(a_full + 8 * i, A_Q ? C::GROUP_WARPS : 1); mbar_init(a_empty + 8 * i, 1); }
+        for (int i = 0; i < C::NAR; ++i) { mbar_init(ar_full + 8 * i, 1); mbar_init(ar_empty + 8 * i, C::GROUP_WARPS); }
+        for (int i = 0; i < C::LB; ++i) { mbar_init(b_full + 8 * i, C::GROUP_WARPS); mbar_init(b_empty + 8 * i, 1); }
+        for (int i = 0; i < C::LBR; ++i) { mbar_init(br_full + 8 * i, 1); mbar_init(br_empty + 8 * i, C::GROUP_WARPS); }
+        for (int i = 0; i < 2; ++i) { mbar_init(acc_full + 8 * i, 1); mbar_init(acc_empty + 8 * i, 4); }
+        misc_gen[1] = 0u;
+        fence_mbar_init();
+        prefetch_tensormap(&tm_a);
+        prefetch_tensormap(&tm_b);
+        prefetch_tensormap(&tm_b_exp);
+        prefetch_tensormap(&tm_c);
+    }
+    if (warp == 1) {
+        tmem_alloc(misc, 512u);
+        tmem_relinquish();
+    }
+    if (threadIdx.x >= kFirstDequantWarp * 32 && threadIdx.x < kFirstDequantWarp * 32 + 256) {
+        const uint32_t E = threadIdx.x - kFirstDequantWarp * 32;
+        asm volatile("st.shared.b32 [%0], %1;" ::"r"(scale_lut + E * 4), "r"(scale_table_entry(E)) : "memory");
+    }
+    tcgen05_fence_before_sync();
+    __syncthreads();
+    tcgen05_fence_after_sync();
+    const uint32_t tmem_base = misc_gen[0];
+
+    const int total_tiles = p.m_tiles * p.n_tiles;
+
+    if (warp == 0) {
+        // ================================ TMA producer: raw B units ====================
+        if (elect_one()) {
+            Cursor<C::NBR, ring_bars(C::NBR, C::DB)> rr;
+            bool ok = true;
+            for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+                int mt, nt;
+                tile_coords(tile, p.m_tiles, p.n_tiles, mt, nt);
+                for (int k = 0; ok && k < p.k_steps; ++k) {
+                    for (int u = 0; u < 2; ++u) {
+                        if (!(ok = wait_bar_spin(cx, br_empty + 8 * rr.freed_bar(), rr.freed_parity(), 0x001))) break;
+                        const uint32_t fr = br_full + 8 * rr.bar;
+                        const uint32_t dst = b_raw_base + rr.buf() * C::RAW_BYTES;
+                        mbar_arrive_expect_tx(fr, C::RAW_BYTES);
+                        tma_load_2d(dst, &tm_b, k * C::T_K, nt * C::T_N + u * 128, fr);
+                        tma_load_2d(dst + C::RAW_MANT_BYTES, &tm_b_exp, nt * C::T_N + u * 128, k, fr);
+                        rr.template advance<1>();
+                    }
+                }
+            }
+        }
+    } else if (warp == kAProducerWarp) {
+        // ================================ TMA producer: A units ========================
+        if (elect_one()) {
+            bool ok = true;
+            if (A_Q) {
+                Cursor<(C::NAR > 0 ? C::NAR : 1), ring_bars((C::NAR > 0 ? C::NAR : 1), (C::DA > 0 ? C::DA : 1))> rr;
+                for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+                    int mt, nt;
+                    tile_coords(tile, p.m_tiles, p.n_tiles, mt, nt);
+                    for (int k = 0; ok && k < p.k_steps; ++k) {
+                        for (int u = 0; u < 2; ++u) {
+                            if (!(ok = wait_bar_spin(cx, ar_empty + 8 * rr.freed_bar(), rr.freed_parity(), 0x002))) break;
+                            const uint32_t fr = ar_full + 8 * rr.bar;
+                            const uint32_t dst = a_raw_base + rr.buf() * C::RAW_BYTES;
+                            mbar_arrive_expect_tx(fr, C::RAW_BYTES);
+                            tma_load_2d(dst, &tm_a, k * C::T_K, mt * 256 + u * 128, fr);
+                            tma_load_2d(dst + C::RAW_MANT_BYTES, &tm_a_exp, mt * 256 + u * 128, k, fr);
+                            rr.template advance<1>();
+                        }
+                    }
+                }
+            } else {
+                // BF16 A: the TMA box is the UMMA operand (K-major, 128-byte swizzle)
+                Ring ra;
+                for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+                    int mt, nt;
+                    tile_coords(tile, p.m_tiles, p.n_tiles, mt, nt);
+                    for (int k = 0; ok && k < p.k_steps; ++k) {
+                        for (int u = 0; u < 2; ++u) {
+                            if (!(ok = wait_bar_spin(cx, a_empty + 8 * ra.stage, ra.phase ^ 1u, 0x002))) break;
+                            const uint32_t fa = a_full + 8 * ra.stage;
+                            mbar_arrive_expect_tx(fa, C::UNIT_BYTES);
+                            tma_load_2d(a_base + ra.stage * C::UNIT_BYTES, &tm_a, k * C::T_K, mt * 256 + u * 128, fa);
+                            ra.advance(C::NA);
+                        }
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ================================ UMMA issuer =================================
+        if (elect_one()) {
+            constexpr uint32_t idesc = umma_idesc_bf16_f32(128, 256, false, false);   // both operands K-major
+            Ring ra;
+            Cursor<C::NB, C::LB> rb;                 // first unit of the B tile; the second follows it
+            uint32_t acc_phase = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, acc_phase ^= 1u) {
+                for (int k = 0; ok && k < p.k_steps; ++k) {
+                    // the converted B tile of this K-step: two units, adjacent in shared memory
+                    if (!(ok = wait_bar_spin(cx, b_full + 8 * rb.bar, rb.phase, 0x101))) break;
+                    if (!(ok = wait_bar_spin(cx, b_full + 8 * (rb.bar + 1), rb.phase, 0x101))) break;
+                    const uint32_t bs = b_base + rb.buf() * C::UNIT_BYTES;
+                    for (int g = 0; g < 2; ++g) {
+                        if (k == 0 && !(ok = wait_bar_spin(cx, acc_empty + 8 * g, acc_phase ^ 1u, 0x102))) break;
+                        if (!(ok = wait_bar_spin(cx, a_full + 8 * ra.stage, ra.phase, 0x103))) break;
+                        tcgen05_fence_after_sync();
+                        const uint32_t as = a_base + ra.stage * C::UNIT_BYTES;
+#pragma unroll
+                        for (int kk = 0; kk < C::T_K / 16; ++kk) {
+                            const uint64_t a_desc = umma_smem_desc_sw128(as + kk * 32, 16, 1024);
+                            const uint64_t b_desc = umma_smem_desc_sw128(bs + kk * 32, 16, 1024);
+                            umma_f16_ss(tmem_base + static_cast<uint32_t>(g * 256), a_desc, b_desc, idesc, (k > 0 || kk > 0) ? 1u : 0u);
+                        }
+                        umma_commit(a_empty + 8 * ra.stage);
+                        ra.advance(C::NA);
+                        if (k == p.k_steps - 1) umma_commit(acc_full + 8 * g);
+                    }
+                    if (!ok) break;
+                    umma_commit(b_empty + 8 * rb.bar);
+                    umma_commit(b_empty + 8 * (rb.bar + 1));
+                    rb.template advance<2>();
+                }
+            }
+        }
+    } else if (warp < kFirstDequantWarp) {
+        // ================================ epilogue ====================================
+        const int q = warp & 3;
+        uint32_t acc_phase = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, acc_phase ^= 1u) {
+            int mt, nt;
+            tile_coords(tile, p.m_tiles, p.n_tiles, mt, nt);
+            for (int g = 0; g < 2; ++g) {
+                if (!(ok = wait_bar(cx, acc_full + 8 * g, acc_phase, 0x201))) break;
+                tcgen05_fence_after_sync();
+                const int row0 = mt * 256 + g * 128 + q * 32;
+                const int col0 = nt * C::T_N;
+                const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + static_cast<uint32_t>(g * 256);
+                const uint32_t box = smem_base + stage_off + static_cast<uint32_t>(warp - kFirstEpilogueWarp) * kEpilogueBoxBytes;
+                if (C_Q) epilogue_bfp16<C::T_N>(&tm_c, t_addr, box, lane, row0, col0, p.M, p.N, p.C_exp, p.c_exp_rows);
+                else epilogue_bf16<C::T_N>(&tm_c, t_addr, box, lane, row0, col0, p.M, p.N);
+                tcgen05_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(acc_empty + 8 * g);
+            }
+        }
+        if (lane == 0) tma_store_wait_all<0>();
+    } else {
+        // ================================ dequantisers ================================
+        const int group = (threadIdx.x - kFirstDequantWarp * 32) / 128, t = (threadIdx.x - kFirstDequantWarp * 32) % 128;
+        int64_t units = 0;
+        for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) units += 2 * static_cast<int64_t>(p.k_steps);
+        if (A_Q && group < C::DA) {
+            dequant_stream<(C::DA > 0 ? C::DA : 1), (C::NAR > 0 ? C::NAR : 1), C::NA>(
+                cx, group, units, t, lane, ar_full, ar_empty, a_full, a_empty, a_raw_base, a_base, scale_lut, 0x300);
+        } else {
+            dequant_stream<C::DB, C::NBR, C::NB>(cx, group - C::DA, units, t, lane, br_full, br_empty, b_full, b_empty,
+                                                 b_raw_base, b_base, scale_lut, 0x310);
+        }
+    }
+
+    if (*cx.abort_flag) {
+        for (int i = 0; i < 64; ++i) __nanosleep(20000);
+    }
+    tcgen05_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        tcgen05_fence_after_sync();
+        tmem_dealloc(tmem_base, 512u);
+    }
+}
+
+std::mutex g_cfg_mutex;
+unsigned int* g_cfg_flag_addr[64] = {};
+
+template <bool A_Q, bool C_Q>
+atb_status_t launch_cfg(int64_t M, int64_t N, int64_t K, const void* A, const uint8_t* A_exp, int64_t lda,
+                        const int8_t* Bt_mant, const uint8_t* Bt_exp, void* Cout, uint8_t* C_exp, int64_t ldc,
+                        int num_sms, unsigned int* error_flag, cudaStream_t stream) {
+    using C = CfgK<A_Q>;
+    CUtensorMap tm_a, tm_a_exp, tm_b, tm_b_exp, tm_c;
+    const int64_t M_pad = atb::round_up(M, 32), N_pad = atb::round_up(N, 32);
+    if (A_Q) {
+        if (!make_map_2d(&tm_a, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, A, K, M, K, 64, 128, CU_TENSOR_MAP_SWIZZLE_NONE) ||
+            !make_map_2d(&tm_a_exp, CU_TENSOR_MAP_DATA_TYPE_UINT64, 8, A_exp, M_pad, atb::ceil_div(K, 64), M_pad * 8, 128, 1,
+                         CU_TENSOR_MAP_SWIZZLE_NONE))
+            return atb::fail(ATB_ERR_CUDA, "cuTensorMapEncodeTiled failed for the planes of A");
+    } else {
+        if (!make_map_2d(&tm_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, A, K, M, lda * 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B))
+            return atb::fail(ATB_ERR_CUDA, "cuTensorMapEncodeTiled failed for A");
+        tm_a_exp = tm_a;                                   // unused
+    }
+    if (!make_map_2d(&tm_b, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Bt_mant, K, N, K, 64, 128, CU_TENSOR_MAP_SWIZZLE_NONE) ||
+        !make_map_2d(&tm_b_exp, CU_TENSOR_MAP_DATA_TYPE_UINT64, 8, Bt_exp, N_pad, atb::ceil_div(K, 64), N_pad * 8, 128, 1,
+                     CU_TENSOR_MAP_SWIZZLE_NONE))
+        return atb::fail(ATB_ERR_CUDA, "cuTensorMapEncodeTiled failed for the planes of B");
+    if (C_Q) {
+        if (!make_map_2d(&tm_c, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Cout, N, M, N, 64, 32, CU_TENSOR_MAP_SWIZZLE_64B))
+            return atb::fail(ATB_ERR_CUDA, "cuTensorMapEncodeTiled failed for the mantissa plane of C");
+    } else if (!make_map_2d(&tm_c, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Cout, N, M, ldc * 2, 64, 32, CU_TENSOR_MAP_SWIZZLE_128B)) {
+        return atb::fail(ATB_ERR_CUDA, "cuTensorMapEncodeTiled failed for C");
+    }
+    CfgParams p;
+    p.M = M; p.N = N; p.K = K;
+    p.m_tiles = static_cast<int>(atb::ceil_div(M, 256));
+    p.n_tiles = static_cast<int>(atb::ceil_div(N, 256));
+    p.k_steps = static_cast<int>(atb::ceil_div(K, 64));
+    p.C_exp = C_exp;
+    p.c_exp_rows = M_pad;
+    p.error_flag = error_flag;
+    auto kernel = atb_gemm_cfg_kernel<A_Q, C_Q>;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(C::SMEM_BYTES));
+    if (e != cudaSuccess) return atb::fail(ATB_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
+    const int64_t tiles = static_cast<int64_t>(p.m_tiles) * p.n_tiles;
+    const int grid = static_cast<int>(tiles < num_sms ? tiles : num_sms);
+    kernel<<<grid, kThreads, C::SMEM_BYTES, stream>>>(tm_a, tm_a_exp, tm_b, tm_b_exp, tm_c, p);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return atb::fail(ATB_ERR_CUDA, "gemm (config) launch: %s", cudaGetErrorString(e));
+    return ATB_OK;
+}
+
+}  // namespace
+
+extern "C" atb_status_t atb_gemm_config(int config, int64_t M, int64_t N, int64_t K,
+                                        const void* A_dev, const uint8_t* A_exp_dev, int64_t lda,
+                                        const int8_t* Bt_mant_dev, const uint8_t* Bt_exp_dev,
+                                        void* C_dev, uint8_t* C_exp_dev, int64_t ldc, void* stream) {
+    atb::clear_error();
+    if (config != 1 && config != 2) return atb::fail(ATB_ERR_BAD_TILING, "config=%d: 1 (A BF16, B BFP16, C BF16) or 2 (all BFP16)", config);
+    if (!A_dev || !Bt_mant_dev || !Bt_exp_dev || !C_dev || (config == 2 && (!A_exp_dev || !C_exp_dev)))
+        return atb::fail(ATB_ERR_NULL_POINTER, "operand pointers must be non-NULL");
+    if (M < 1 || N < 16 || N % 16 != 0 || K < 16 || K % 16 != 0 || M > (1ll << 30) || N > (1ll << 30) || K > (1ll << 30))
+        return atb::fail(ATB_ERR_BAD_SHAPE, "need M >= 1, N %% 16 == 0, K %% 16 == 0 (got %lld, %lld, %lld)", (long long)M, (long long)N, (long long)K);
+    if (config == 1 && (lda < K || lda % 8 != 0 || ldc < N || ldc % 8 != 0))
+        return atb::fail(ATB_ERR_BAD_SHAPE, "lda=%lld must be >= K, ldc=%lld >= N, both multiples of 8", (long long)lda, (long long)ldc);
+    if (!atb::aligned16(A_dev) || !atb::aligned16(Bt_mant_dev) || !atb::aligned16(Bt_exp_dev) || !atb::aligned16(C_dev) ||
+        (config == 2 && (!atb::aligned16(A_exp_dev) || !atb::aligned16(C_exp_dev))))
+        return atb::fail(ATB_ERR_MISALIGNED, "all device pointers must be 16-byte aligned");
+    int dev = 0, major = 0, minor = 0, sms = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return atb::fail(ATB_ERR_CUDA, "cudaGetDevice: %s", cudaGetErrorString(e));
+    cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+    cudaDeviceGetAttribute(&minor, cudaDevAttrComputeCapabilityMinor, dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (major != 10 || minor != 0)
+        return atb::fail(ATB_ERR_UNSUPPORTED_DEVICE, "compute capability %d.%d; this library runs on 10.0 only", major, minor);
+    if (dev < 0 || dev >= 64) return atb::fail(ATB_ERR_UNSUPPORTED_DEVICE, "device ordinal %d out of range", dev);
+    unsigned int* flag = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_cfg_mutex);
+        if (!g_cfg_flag_addr[dev]) {
+            e = cudaGetSymbolAddress(reinterpret_cast<void**>(&g_cfg_flag_addr[dev]), g_cfg_error_flag);
+            if (e != cudaSuccess) return atb::fail(ATB_ERR_CUDA, "cudaGetSymbolAddress: %s", cudaGetErrorString(e));
+        }
+        flag = g_cfg_flag_addr[dev];
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (config == 1)
+        return launch_cfg<false, false>(M, N, K, A_dev, nullptr, lda, Bt_mant_dev, Bt_exp_dev, C_dev, nullptr, ldc, sms, flag, st);
+    return launch_cfg<true, true>(M, N, K, A_dev, A_exp_dev, K, Bt_mant_dev, Bt_exp_dev, C_dev, C_exp_dev, N, sms, flag, st);
+}
+
+namespace atb {
+// Reads and clears the timeout flag of the configuration kernels (part of atb_device_status).
+unsigned int take_cfg_error_flag() {
+    unsigned int flag = 0;
+    if (cudaMemcpyFromSymbol(&flag, g_cfg_error_flag, sizeof flag) != cudaSuccess) return 0;
+    if (flag != 0) {
+        const unsigned int zero = 0;
+        cudaMemcpyToSymbol(g_cfg_error_flag, &zero, sizeof zero);
+    }
+    return flag;
+}
+}  // namespace atb

@@ -11,6 +11,7 @@
 #include <mutex>
 
 #include "atb_internal.h"
+#include "bfp16_block.cuh"
 #include "sm100_ptx.cuh"
 
 namespace {
@@ -44,7 +45,7 @@ constexpr uint32_t kSmemBudget = 232448;          // 227 KB of dynamic shared me
 constexpr uint64_t kWaitTimeoutNs = 2000000000ull;  // every mbarrier wait gives up after 2 s
 
 // lcm(n, d) for d a power of two: the number of barrier pairs of a ring of n buffers and d groups
-constexpr int ring_bars(int n, int d) {
+__host__ __device__ constexpr int ring_bars(int n, int d) {
     int g = d;
     while (n % g) g >>= 1;
     return n / g * d;
@@ -404,6 +405,104 @@ __device__ __forceinline__ void dequant_slab(const DequantLane<C>& ln, uint32_t 
                          "r"(dequant_pair(u2, 0x4140u, s1)), "r"(dequant_pair(u2, 0x4342u, s1)),
                          "r"(dequant_pair(u3, 0x4140u, s1)), "r"(dequant_pair(u3, 0x4342u, s1))
                          : "memory");
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Epilogues of one warp: N_COLS accumulator columns of its 32 TMEM lanes (rows row0 .. row0+31,
+// columns col0 ..) -> C.  `box` is the warp's 4 KB of staging in shared memory.  Rows and columns
+// beyond M, N are clipped by the tensor map of the TMA store.
+// ---------------------------------------------------------------------------------------------
+// BF16 C: tcgen05.ld -> round to bf16 (RNE) -> 128-byte-swizzled 32 x 64 box -> TMA store.
+template <int N_COLS>
+__device__ __forceinline__ void epilogue_bf16(const CUtensorMap* tm_c, uint32_t t_addr, uint32_t box, int lane, int row0,
+                                              int col0, int64_t M, int64_t N) {
+    const uint32_t my_row = box + lane * 128;
+    const uint32_t sw = static_cast<uint32_t>(lane & 7);
+#pragma unroll 1
+    for (int c = 0; c < N_COLS / 64; ++c) {
+        // the previous TMA store of this warp must have finished reading the box
+        if (lane == 0) tma_store_wait_read<0>();
+        __syncwarp();
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            uint32_t v[32];
+            tmem_ld_32x32b_x32(t_addr + c * 64 + h * 32, v);
+            tmem_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                uint32_t o[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(v[j * 8 + 2 * e]),
+                                                              __uint_as_float(v[j * 8 + 2 * e + 1]));
+                    o[e] = *reinterpret_cast<uint32_t*>(&b2);
+                }
+                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(my_row + ((static_cast<uint32_t>(h * 4 + j) ^ sw) << 4)),
+                             "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]) : "memory");
+            }
+        }
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0 && row0 < M && col0 + c * 64 < N) {   // rows / columns past the edge are clipped
+            tma_store_2d(tm_c, box, col0 + c * 64, row0);
+            tma_store_commit();
+        }
+    }
+}
+
+// BFP16 C: a thread owns one row; per 64 columns it quantises 8 blocks of 8 FP32 accumulators
+// (exactly as atb_quantize_bfp16 would), stages the 64 mantissa bytes of its row in a 32 x 64-byte
+// box (64-byte swizzle) for one TMA store, and writes the 8 exponents - contiguous in the exponent
+// plane [ceil(N/64)][exp_rows][8], rows adjacent - directly.  Rows of the plane's padding
+// (M <= row < exp_rows) get exponent 0.
+template <int N_COLS>
+__device__ __forceinline__ void epilogue_bfp16(const CUtensorMap* tm_c, uint32_t t_addr, uint32_t box, int lane, int row0,
+                                               int col0, int64_t M, int64_t N, uint8_t* exp_plane, int64_t exp_rows) {
+    const uint32_t my_row64 = box + lane * 64;
+    const uint32_t sw64 = static_cast<uint32_t>(lane >> 1) & 3u;
+    const int64_t row = static_cast<int64_t>(row0) + lane;
+#pragma unroll 1
+    for (int c = 0; c < N_COLS / 64; ++c) {
+        if (lane == 0) tma_store_wait_read<0>();
+        __syncwarp();
+        uint32_t e_lo = 0, e_hi = 0;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            uint32_t v[32];
+            tmem_ld_32x32b_x32(t_addr + c * 64 + h * 32, v);
+            tmem_ld_wait();
+            uint32_t m8[8];
+#pragma unroll
+            for (int b = 0; b < 4; ++b) {
+                float x[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) x[e] = __uint_as_float(v[b * 8 + e]);
+                uint32_t pk[2];
+                const uint32_t E = static_cast<uint32_t>(bfp16::quantize_block8(x, pk));
+                m8[2 * b] = pk[0];
+                m8[2 * b + 1] = pk[1];
+                if (h == 0) e_lo |= E << (8 * b); else e_hi |= E << (8 * b);
+            }
+#pragma unroll
+            for (int j = 0; j < 2; ++j)
+                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(my_row64 + ((static_cast<uint32_t>(h * 2 + j) ^ sw64) << 4)),
+                             "r"(m8[4 * j]), "r"(m8[4 * j + 1]), "r"(m8[4 * j + 2]), "r"(m8[4 * j + 3]) : "memory");
+        }
+        fence_proxy_async_smem();
+        __syncwarp();
+        const int64_t col = static_cast<int64_t>(col0) + c * 64;
+        if (col < N) {
+            if (lane == 0 && row0 < M) {
+                tma_store_2d(tm_c, box, static_cast<int>(col), row0);
+                tma_store_commit();
+            }
+            if (row < exp_rows) {
+                const bool real = row < M;
+                uint2 ev = make_uint2(real ? e_lo : 0u, real ? e_hi : 0u);
+                *reinterpret_cast<uint2*>(exp_plane + ((col >> 6) * exp_rows + row) * 8) = ev;
+            }
         }
     }
 }

@@ -213,42 +213,12 @@ atb_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_c
             tile_coords(tile, p.m_tiles, p.n_tiles, mt, nt);
             const int row0 = mt * 256 + static_cast<int>(rank) * 128 + q * 32;
             const uint32_t box = smem_base + stage_off + static_cast<uint32_t>(warp - kFirstEpilogueWarp) * kEpilogueBoxBytes;
-            const uint32_t my_row = box + lane * 128;
-            const uint32_t sw = static_cast<uint32_t>(lane & 7);
             for (int nc = 0; nc < C::N_CHUNKS; ++nc) {
                 if (!(ok = wait_bar_cl(cx, acc_full + 8 * nc, acc_phase, 0x201))) break;
                 tcgen05_fence_after_sync();
                 const int col0 = nt * 512 + nc * C::N_MMA;
                 const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + static_cast<uint32_t>(nc * C::N_MMA);
-#pragma unroll 1
-                for (int c = 0; c < C::N_MMA / 64; ++c) {
-                    if (lane == 0) tma_store_wait_read<0>();
-                    __syncwarp();
-#pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        uint32_t v[32];
-                        tmem_ld_32x32b_x32(t_addr + c * 64 + h * 32, v);
-                        tmem_ld_wait();
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            uint32_t o[4];
-#pragma unroll
-                            for (int e = 0; e < 4; ++e) {
-                                __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(v[j * 8 + 2 * e]),
-                                                                          __uint_as_float(v[j * 8 + 2 * e + 1]));
-                                o[e] = *reinterpret_cast<uint32_t*>(&b2);
-                            }
-                            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(my_row + ((static_cast<uint32_t>(h * 4 + j) ^ sw) << 4)),
-                                         "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]) : "memory");
-                        }
-                    }
-                    fence_proxy_async_smem();
-                    __syncwarp();
-                    if (lane == 0 && row0 < p.M && col0 + c * 64 < p.N) {
-                        tma_store_2d(&tm_c, box, col0 + c * 64, row0);
-                        tma_store_commit();
-                    }
-                }
+                epilogue_bf16<C::N_MMA>(&tm_c, t_addr, box, lane, row0, col0, p.M, p.N);
                 tcgen05_fence_before_sync();
                 __syncwarp();
                 if (lane == 0) mbar_arrive_cluster(mapa_shared(acc_empty + 8 * nc, 0));

@@ -25,7 +25,6 @@
 #include <cmath>
 
 #include "atb_gemm_device.cuh"
-#include "bfp16_block.cuh"
 
 namespace {
 
@@ -244,10 +243,10 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
                 const int col0 = nt * T_N;
                 const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + static_cast<uint32_t>(acc * T_N);
                 const uint32_t box = smem_base + stage_off + static_cast<uint32_t>(warp - kFirstEpilogueWarp) * kEpilogueBoxBytes;
-                const uint32_t my_row = box + lane * 128;
-                const uint32_t sw = static_cast<uint32_t>(lane & 7);
                 if (SPLIT) {
                     // FP32 partial tile -> workspace [split][m_pad][N]: boxes of 32 rows x 32 columns
+                    const uint32_t my_row = box + lane * 128;
+                    const uint32_t sw = static_cast<uint32_t>(lane & 7);
 #pragma unroll 1
                     for (int c = 0; c < T_N / 32; ++c) {
                         if (lane == 0) tma_store_wait_read<0>();
@@ -267,86 +266,9 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
                         }
                     }
                 } else if (QOUT) {
-                    // BFP16 C: a thread owns one row; per 64 columns it quantises 8 blocks of 8 FP32
-                    // accumulators (exactly as atb_quantize_bfp16 would), stages the 64 mantissa bytes
-                    // of its row in a 32 x 64-byte box (64-byte swizzle) for one TMA store, and writes
-                    // the 8 exponents - contiguous in the exponent plane, rows adjacent - directly.
-                    const uint32_t my_row64 = box + lane * 64;
-                    const uint32_t sw64 = static_cast<uint32_t>(lane >> 1) & 3u;
-                    const int64_t row = static_cast<int64_t>(row0) + lane;
-#pragma unroll 1
-                    for (int c = 0; c < T_N / 64; ++c) {
-                        if (lane == 0) tma_store_wait_read<0>();
-                        __syncwarp();
-                        uint32_t e_lo = 0, e_hi = 0;
-#pragma unroll
-                        for (int h = 0; h < 2; ++h) {
-                            uint32_t v[32];
-                            tmem_ld_32x32b_x32(t_addr + c * 64 + h * 32, v);
-                            tmem_ld_wait();
-                            uint32_t m8[8];
-#pragma unroll
-                            for (int b = 0; b < 4; ++b) {
-                                float x[8];
-#pragma unroll
-                                for (int e = 0; e < 8; ++e) x[e] = __uint_as_float(v[b * 8 + e]);
-                                uint32_t pk[2];
-                                const uint32_t E = static_cast<uint32_t>(bfp16::quantize_block8(x, pk));
-                                m8[2 * b] = pk[0];
-                                m8[2 * b + 1] = pk[1];
-                                if (h == 0) e_lo |= E << (8 * b); else e_hi |= E << (8 * b);
-                            }
-#pragma unroll
-                            for (int j = 0; j < 2; ++j)
-                                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(my_row64 + ((static_cast<uint32_t>(h * 2 + j) ^ sw64) << 4)),
-                                             "r"(m8[4 * j]), "r"(m8[4 * j + 1]), "r"(m8[4 * j + 2]), "r"(m8[4 * j + 3]) : "memory");
-                        }
-                        fence_proxy_async_smem();
-                        __syncwarp();
-                        const int64_t col = static_cast<int64_t>(col0) + c * 64;
-                        if (col < p.N) {
-                            if (lane == 0 && row0 < p.M) {
-                                tma_store_2d(&tm_c, box, static_cast<int>(col), row0);
-                                tma_store_commit();
-                            }
-                            if (row < p.c_exp_rows) {       // rows of the plane's padding get exponent 0
-                                const bool real = row < p.M;
-                                uint2 ev = make_uint2(real ? e_lo : 0u, real ? e_hi : 0u);
-                                *reinterpret_cast<uint2*>(p.C_exp + ((col >> 6) * p.c_exp_rows + row) * 8) = ev;
-                            }
-                        }
-                    }
+                    epilogue_bfp16<T_N>(&tm_c, t_addr, box, lane, row0, col0, p.M, p.N, p.C_exp, p.c_exp_rows);
                 } else {
-#pragma unroll 1
-                for (int c = 0; c < T_N / 64; ++c) {
-                    // the previous TMA store of this warp must have finished reading the box
-                    if (lane == 0) tma_store_wait_read<0>();
-                    __syncwarp();
-#pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        uint32_t v[32];
-                        tmem_ld_32x32b_x32(t_addr + c * 64 + h * 32, v);
-                        tmem_ld_wait();
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            uint32_t o[4];
-#pragma unroll
-                            for (int e = 0; e < 4; ++e) {
-                                __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(v[j * 8 + 2 * e]),
-                                                                          __uint_as_float(v[j * 8 + 2 * e + 1]));
-                                o[e] = *reinterpret_cast<uint32_t*>(&b2);
-                            }
-                            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(my_row + ((static_cast<uint32_t>(h * 4 + j) ^ sw) << 4)),
-                                         "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]) : "memory");
-                        }
-                    }
-                    fence_proxy_async_smem();
-                    __syncwarp();
-                    if (lane == 0 && row0 < p.M && col0 + c * 64 < p.N) {   // rows / columns past the edge are clipped
-                        tma_store_2d(&tm_c, box, col0 + c * 64, row0);
-                        tma_store_commit();
-                    }
-                }
+                    epilogue_bf16<T_N>(&tm_c, t_addr, box, lane, row0, col0, p.M, p.N);
                 }
                 tcgen05_fence_before_sync();
                 __syncwarp();
@@ -655,6 +577,9 @@ extern "C" atb_status_t atb_device_status(void* stream) {
         cudaMemcpyToSymbol(g_gemm_error_flag, &zero, sizeof zero);
         return atb::fail(ATB_ERR_DEVICE_TIMEOUT, "a GEMM kernel gave up a bounded wait (code 0x%03x)", flag);
     }
+    flag = atb::take_cfg_error_flag();
+    if (flag != 0)
+        return atb::fail(ATB_ERR_DEVICE_TIMEOUT, "a precision-configuration GEMM kernel gave up a bounded wait (code 0x%03x)", flag);
     return ATB_OK;
 }
 

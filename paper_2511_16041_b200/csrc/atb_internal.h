@@ -34,4 +34,7 @@ atb_status_t launch_gemm_pair(int T_MA, const GemmPlan& plan, int64_t M, int64_t
                               const uint8_t* exp, const void* B, int64_t ldb, void* C, int64_t ldc, int num_sms,
                               unsigned int* error_flag, void* stream);
 
+// Reads and clears the timeout flag of the precision-configuration kernels (0 = none).
+unsigned int take_cfg_error_flag();
+
 }  // namespace atb

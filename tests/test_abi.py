@@ -76,6 +76,11 @@ def test_argument_validation_needs_no_gpu():
     assert lib.atb_gemm_bfp16_out(128, 128, 64, 64, 128, 64, 128, 16, 16, 16, 128, None, 16, None) == 1   # NULL
     assert lib.atb_gemm_bfp16_out(128, 136, 64, 64, 128, 64, 128, 16, 16, 16, 136, 16, 16, None) == 2     # N % 16
     assert lib.atb_gemm_bfp16_out(128, 128, 64, 32, 128, 64, 128, 16, 16, 16, 128, 16, 16, None) == 3     # tiling
+    assert lib.atb_gemm_config(0, 128, 128, 64, 16, None, 64, 16, 16, 16, None, 128, None) == 3            # config
+    assert lib.atb_gemm_config(1, 128, 128, 64, 16, None, 64, 16, None, 16, None, 128, None) == 1          # NULL plane
+    assert lib.atb_gemm_config(2, 128, 128, 64, 16, 16, 64, 16, 16, 16, None, 128, None) == 1              # config 2 needs C_exp
+    assert lib.atb_gemm_config(1, 128, 136, 64, 16, None, 64, 16, 16, 16, None, 136, None) == 2            # N % 16
+    assert lib.atb_gemm_config(1, 128, 128, 64, 24, None, 64, 16, 16, 16, None, 128, None) == 4            # alignment
     assert atb.atb_last_error_message() != ""
 
 
