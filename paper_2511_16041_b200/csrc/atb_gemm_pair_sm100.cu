@@ -117,6 +117,10 @@ atb_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_c
     cluster_sync_all();                      // the peer's barriers exist before anything arrives on them
     tcgen05_fence_after_sync();
     const uint32_t tmem_base = misc_gen[0];
+#ifdef ATB_PROFILE
+    const long long prof_c0 = clock64();
+    const uint64_t prof_t0 = global_timer_ns();
+#endif
 
     const int total_tiles = p.m_tiles * p.n_tiles;
     const int cluster_id = blockIdx.x >> 1, n_clusters = gridDim.x >> 1;
@@ -233,6 +237,16 @@ atb_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_c
         int64_t my_slabs = 0;
         for (int tile = cluster_id; tile < total_tiles; tile += n_clusters) my_slabs += static_cast<int64_t>(p.k_steps) * C::SLABS;
         const DequantLane<C> ln(t, SLAB_ROWS);
+#ifdef ATB_PROFILE_SKIP_DEQUANT
+        // diagnostic: the operand ring holds fixed pseudo-random bf16 values (zeros would lower the
+        // tensor cores' power and flatter the clock)
+        for (uint32_t i = threadIdx.x - kFirstDequantWarp * 32; i < C::NG * C::GROUP_BYTES / 4; i += kDequantWarps * 32) {
+            uint32_t h = (i + 1u) * 2654435761u; h ^= h >> 15; h *= 2246822519u; h ^= h >> 13;
+            const uint32_t v = (h & 0x807F807Fu) | 0x3F003F00u;          // +-[0.5, 1) in both halves
+            asm volatile("st.shared.b32 [%0], %1;" ::"r"(deq_base + i * 4), "r"(v) : "memory");
+        }
+        fence_proxy_async_smem();
+#endif
         Cursor<C::NR, C::LR> rr;
         Cursor<C::ND, C::LD> rd;
         rr.start_at(my_group);
@@ -243,7 +257,9 @@ atb_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_c
             const uint32_t raw = raw_base + rr.buf() * C::RAW_BYTES;
             const uint32_t dst_base = deq_base + (rd.buf() / C::SLABS) * C::GROUP_BYTES;
             const int row_base = (rd.buf() % C::SLABS) * SLAB_ROWS;
+#ifndef ATB_PROFILE_SKIP_DEQUANT    // diagnostic: the pipeline without the conversion work (results are wrong)
             dequant_slab<C>(ln, raw, raw + C::RAW_MANT_BYTES, scale_lut, dst_base, row_base, t, SLAB_ROWS);
+#endif
             fence_proxy_async_smem();
             __syncwarp();
             if (lane == 0) {
@@ -261,6 +277,12 @@ atb_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_c
     }
     tcgen05_fence_before_sync();
     __syncthreads();
+#ifdef ATB_PROFILE
+    if (threadIdx.x == 0) {     // slots 0 / 4: nanoseconds and SM cycles of this CTA's main loop
+        atomicAdd(&g_wait_cycles[blockIdx.x & 255][0], static_cast<unsigned long long>(global_timer_ns() - prof_t0));
+        atomicAdd(&g_wait_cycles[blockIdx.x & 255][4], static_cast<unsigned long long>(clock64() - prof_c0));
+    }
+#endif
     cluster_sync_all();
     if (warp == 1) {
         tcgen05_fence_after_sync();

@@ -288,6 +288,16 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
             my_slabs += static_cast<int64_t>(w.k_end - w.k_begin) * C::RHO;
         }
         const DequantLane<C> ln(t, T_MA);
+#ifdef ATB_PROFILE_SKIP_DEQUANT
+        // diagnostic: the operand ring holds fixed pseudo-random bf16 values (zeros would lower the
+        // tensor cores' power and flatter the clock)
+        for (uint32_t i = threadIdx.x - kFirstDequantWarp * 32; i < C::NG * C::GROUP_BYTES / 4; i += kDequantWarps * 32) {
+            uint32_t h = (i + 1u) * 2654435761u; h ^= h >> 15; h *= 2246822519u; h ^= h >> 13;
+            const uint32_t v = (h & 0x807F807Fu) | 0x3F003F00u;          // +-[0.5, 1) in both halves
+            asm volatile("st.shared.b32 [%0], %1;" ::"r"(deq_base + i * 4), "r"(v) : "memory");
+        }
+        fence_proxy_async_smem();
+#endif
         Cursor<C::NR, C::LR> rr;
         Cursor<C::ND, C::LD> rd;
         rr.start_at(my_group);
