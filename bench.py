@@ -370,6 +370,93 @@ def run_ours(args):
     return 0
 
 
+def run_entry(args):
+    """--entry bfp16_out | config1 | config2: the further GEMM entry points on the same workload, one GPU,
+    device-resident input.  A step is what the entry needs per batch of A: quantise A where the entry
+    takes BFP16 A, then the GEMM.  B (and the planes of B transposed) are prepared once, like weights.
+    The line has the fields of the main line that apply (no end-to-end leg, no CPU baseline)."""
+    import torch
+    import paper_2511_16041_b200 as atb
+    from paper_2511_16041_b200 import inputs
+
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback of the hot path")
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    atb.load_library()
+    name = args.workload
+    c = inputs.CONFIGS[name]
+    M, N, K = c["M"], c["N"], c["K"]
+    A_dev = torch.from_numpy(inputs.make_A(c["A"], M, K, inputs.BASE_SEED)).to(dev)
+    B_dev = torch.from_numpy(inputs.make_B_bits(K, N, c["b_scale"]).view(np.int16)).to(dev).view(torch.bfloat16)
+    stream = torch.cuda.Stream(dev)
+    mant = torch.empty((M, K), dtype=torch.int8, device=dev)
+    plane = torch.empty(atb.atb_bfp16_exp_bytes(M, K), dtype=torch.uint8, device=dev)
+    tiling = tuple(args.tiling) if args.tiling else (128, 256, 64, 256)
+    if args.entry == "bfp16_out":
+        Cm = torch.empty((M, N), dtype=torch.int8, device=dev)
+        Ce = torch.empty(atb.atb_bfp16_exp_bytes(M, N), dtype=torch.uint8, device=dev)
+        kernel, what = "atb_gemm_kernel (quantising epilogue)", "atb_quantize_bfp16 + atb_gemm_bfp16_out"
+        quantises = True
+        call = lambda: atb.atb_gemm_bfp16_out(M, N, K, *tiling, mant, plane, B_dev, Cm, Ce, stream=stream)
+    else:
+        Bt_m, Bt_e = atb.atb_quantize_bfp16(B_dev.float().t().contiguous())      # planes of B transposed, once
+        tiling = (128, 256, 64, 256)
+        if args.entry == "config1":
+            A16 = A_dev.to(torch.bfloat16)
+            C = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
+            kernel, what, quantises = "atb_gemm_cfg_kernel<A bf16, C bf16>", "atb_gemm_config(1)", False
+            call = lambda: atb.atb_gemm_config(1, M, N, K, A16, None, Bt_m, Bt_e, C, stream=stream)
+        else:
+            Cm = torch.empty((M, N), dtype=torch.int8, device=dev)
+            Ce = torch.empty(atb.atb_bfp16_exp_bytes(M, N), dtype=torch.uint8, device=dev)
+            kernel, what, quantises = "atb_gemm_cfg_kernel<A BFP16, C BFP16>", "atb_quantize_bfp16 + atb_gemm_config(2)", True
+            call = lambda: atb.atb_gemm_config(2, M, N, K, mant, plane, Bt_m, Bt_e, Cm, Ce, stream=stream)
+    torch.cuda.synchronize()
+
+    def step(ev=None):
+        if quantises:
+            atb.atb_quantize_bfp16(A_dev, mant, plane, stream=stream)
+        if ev is not None:
+            ev[0].record(stream)
+        call()
+        if ev is not None:
+            ev[1].record(stream)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    atb.atb_device_status(stream)
+    sampler = ClockSampler(physical_gpu_index(0))
+    events = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    sampler.start()
+    t_begin.record(stream)
+    for i in range(args.steps):
+        step(events[i])
+    t_end.record(stream)
+    stream.synchronize()
+    clocks = sampler.stop()
+    atb.atb_device_status(stream)
+    ms_per_step = t_begin.elapsed_time(t_end) / args.steps
+    gemm_ms = sum(a.elapsed_time(b) for a, b in events) / args.steps
+    peaks, peak_src = load_peaks()
+    flops = 2.0 * M * N * K
+    achieved = flops / (gemm_ms * 1e-3) / 1e12
+    line = {"metric": METRIC + " [entry " + args.entry + "]", "value": flops / (ms_per_step * 1e-3) / 1e12, "unit": "TFLOPS",
+            "n_gpus": 1, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": name, "M": M, "N": N, "K": K, "entry": args.entry, "step": what,
+                       "tiling": dict(zip(("T_MA", "T_MC", "T_K", "T_N"), tiling)),
+                       "l2": "inputs larger than L2", "parallelism": "single GPU"},
+            "clocks": clocks, "e2e": None, "gpu_launches": (2 if quantises else 1) * args.steps,
+            "roofline": {"bound": "tensor", "kernel": kernel, "achieved": achieved, "peak": peaks["bf16_tflops"],
+                         "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"],
+                         "peak_source": f"{peak_src} cuBLAS bf16 burst", "kernel_ms": gemm_ms, "traffic": None}}
+    print(json.dumps(line))
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -380,9 +467,13 @@ def main():
     ap.add_argument("--tiling", type=int, nargs=4, metavar=("T_MA", "T_MC", "T_K", "T_N"), default=None)
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--entry", default="gemm", choices=["gemm", "bfp16_out", "config1", "config2"],
+                    help="gemm: the headline hot path (default); the others time the further entry points")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
+    if args.entry != "gemm":
+        return run_entry(args)
     return run_ours(args)
 
 
