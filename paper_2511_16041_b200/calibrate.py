@@ -139,7 +139,7 @@ def evaluate(hw: atb_hw_params_t, records: Iterable[dict]) -> Dict[str, float]:
 
 def fit(records: Iterable[dict], grid: Optional[Dict[str, Sequence[float]]] = None) -> Tuple[Dict[str, float], Dict[str, float]]:
     """Exhaustive search of ``grid`` (name -> candidate values).  Objective: mean pick quality, then the
-    worst shape's, then the absolute error - the selection is judged by what it picks, the absolute
+    worst shape's, then the absolute error - the selection is rated by what it picks, the absolute
     prediction only breaks ties.  Returns (best values, their evaluation)."""
     records = list(records)
     grid = dict(grid or DEFAULT_GRID)
