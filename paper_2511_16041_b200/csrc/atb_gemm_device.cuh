@@ -51,6 +51,15 @@ __host__ __device__ constexpr int ring_bars(int n, int d) {
     return n / g * d;
 }
 
+// Thin slabs (T_MA < 128) are converted in bundles: the largest power-of-two number of consecutive
+// slabs, at most 128 / T_MA (one operand group), such that the raw ring holds a whole bundle for
+// every dequantiser group.
+__host__ __device__ constexpr int slab_bundle(int spg, int n_raw, int groups) {
+    int b = spg;
+    while (b > 1 && n_raw % (b * groups)) b >>= 1;
+    return b;
+}
+
 // ---------------------------------------------------------------------------------------------
 // Ring plans: how the 227 KB of shared memory are split between the B ring, the raw-slab ring and
 // the ring of dequantised 128-row groups.  Evaluated at compile time (the kernels take the depths
@@ -65,8 +74,8 @@ struct RingPlan {
 };
 
 constexpr uint32_t ring_smem_bytes(uint32_t b_bytes, uint32_t group_bytes, uint32_t raw_bytes, int acc_bars,
-                                   int dqg, int b, int g, int n_deq, int r) {
-    const uint32_t bars = 8u * (2 * b + 2 * ring_bars(r, dqg) + 2 * ring_bars(n_deq, dqg) + 2 * acc_bars) + 16u + 1024u;
+                                   int dqg, int bundle, int b, int g, int n_deq, int r) {
+    const uint32_t bars = 8u * (2 * b + 2 * ring_bars(r, dqg * bundle) + 2 * ring_bars(n_deq, dqg) + 2 * acc_bars) + 16u + 1024u;
     return 1024u + b * b_bytes + g * group_bytes + r * raw_bytes + 1024u + 4u * kEpilogueBoxBytes + bars;
 }
 
@@ -90,17 +99,23 @@ constexpr RingPlan plan_single(int T_MA, int T_MC, int T_K, int T_N) {
     pl.tmem_cols = cols;
     // dequantised stages of a plan with g groups; the UMMA issuer takes spg of them at a time
     const auto total = [=](int b, int g, int r) {
-        return ring_smem_bytes(b_bytes, group_bytes, raw_bytes, 2 * G, dqg, b, g, T_MA <= 128 ? g * spg : g / gps, r);
+        return ring_smem_bytes(b_bytes, group_bytes, raw_bytes, 2 * G, dqg, slab_bundle(spg, r, dqg), b, g,
+                               T_MA <= 128 ? g * (spg / slab_bundle(spg, r, dqg)) : g / gps, r);
     };
     const auto bars_ok = [=](int g, int r) {
-        return ring_bars(r, dqg) <= kMaxRingBars && ring_bars(T_MA <= 128 ? g * spg : g / gps, dqg) <= kMaxRingBars;
+        return ring_bars(r, dqg * slab_bundle(spg, r, dqg)) <= kMaxRingBars &&
+               ring_bars(T_MA <= 128 ? g * (spg / slab_bundle(spg, r, dqg)) : g / gps, dqg) <= kMaxRingBars;
     };
     // Any depth is legal (see ring_bars); the default plan gives every dequantiser group the same
     // number of raw slabs and of dequantised stages, which measured best: one raw slab fewer than
     // groups costs 10 %, one more gains nothing.
-    const int nr_step = dqg;
+    // Raw ring: whole rounds of the dequantiser groups over whole bundles (dqg * spg slabs) where that
+    // fits; a tiling that only fits with fewer slabs gets one slab per group and smaller bundles.
     const int ng_step = T_MA <= 128 ? (dqg >= spg ? dqg / spg : 1) : dqg * gps;
-    int nb = 2, ng = ng_step < 2 ? 2 * ng_step : ng_step, nr = nr_step;
+    int nb = 2, ng = ng_step < 2 ? 2 * ng_step : ng_step;
+    int nr_step = dqg * spg * 64 / T_K;                  // 512 rows of look-ahead at T_K = 64, 256 at T_K = 128
+    if (nr_step < dqg || total(nb, ng, nr_step) > kSmemBudget) nr_step = dqg;
+    int nr = nr_step;
     pl.nb = nb; pl.ng = ng; pl.nr = nr;
     if (total(nb, ng, nr) > kSmemBudget) return pl;
     // Grow the rings towards a target look-ahead, counted in 128-row x T_K operand groups:
@@ -139,8 +154,14 @@ constexpr RingPlan plan_pair(int slab) {
     pl.dqg = dqg;
     pl.acc_bufs = 1;
     pl.tmem_cols = 512;
-    const auto total = [=](int b, int g, int r) { return ring_smem_bytes(b_bytes, group_bytes, raw_bytes, 2, dqg, b, g, g * slabs, r); };
-    const auto bars_ok = [=](int g, int r) { return ring_bars(r, dqg) <= kMaxRingBars && ring_bars(g * slabs, dqg) <= kMaxRingBars; };
+    const auto total = [=](int b, int g, int r) {
+        return ring_smem_bytes(b_bytes, group_bytes, raw_bytes, 2, dqg, slab_bundle(slabs, r, dqg), b, g,
+                               g * (slabs / slab_bundle(slabs, r, dqg)), r);
+    };
+    const auto bars_ok = [=](int g, int r) {
+        return ring_bars(r, dqg * slab_bundle(slabs, r, dqg)) <= kMaxRingBars &&
+               ring_bars(g * (slabs / slab_bundle(slabs, r, dqg)), dqg) <= kMaxRingBars;
+    };
     // as in plan_single: whole rounds of the dequantiser groups
     int ng = (dqg + slabs - 1) / slabs;
     if ((ng * slabs) % dqg != 0) ng = dqg;
@@ -397,6 +418,55 @@ __device__ __forceinline__ void dequant_slab(const DequantLane<C>& ln, uint32_t 
             // band i starts i * ROWS_PER_ITER rows further on: possibly in the next 128-row group
             constexpr uint32_t kBandRows = C::ROWS_PER_ITER;
             const uint32_t band = static_cast<uint32_t>((i * kBandRows) >> 7) * C::GROUP_BYTES + static_cast<uint32_t>((i * kBandRows) & 127) * 128u;
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(st0 + band),
+                         "r"(dequant_pair(u0, 0x4140u, s0)), "r"(dequant_pair(u0, 0x4342u, s0)),
+                         "r"(dequant_pair(u1, 0x4140u, s0)), "r"(dequant_pair(u1, 0x4342u, s0))
+                         : "memory");
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(st1 + band),
+                         "r"(dequant_pair(u2, 0x4140u, s1)), "r"(dequant_pair(u2, 0x4342u, s1)),
+                         "r"(dequant_pair(u3, 0x4140u, s1)), "r"(dequant_pair(u3, 0x4342u, s1))
+                         : "memory");
+        }
+    }
+}
+
+// A bundle of NS consecutive thin slabs (consecutive raw buffers, consecutive row ranges of one
+// 128-row operand group): all loads first, then all conversions and stores, so that a thread has
+// NS * DQ_ITERS slots in flight exactly as with one 128-row slab.
+template <class C, int NS>
+__device__ __forceinline__ void dequant_bundle(const DequantLane<C>& ln, uint32_t raw0, uint32_t raw_stride, uint32_t mant_bytes,
+                                               uint32_t scale_lut, uint32_t dst_base, int row_base0, int t, int slab_rows) {
+    static_assert(C::SLOTS % C::GROUP_THREADS == 0, "whole iterations");
+    const int r0 = t / C::SLOTS_PER_ROW;
+    (void)r0;
+    uint4 w[NS][C::DQ_ITERS];
+    uint32_t e[NS][C::DQ_ITERS];
+#pragma unroll
+    for (int s = 0; s < NS; ++s) {
+        const uint32_t ld = raw0 + s * raw_stride + ln.ld_off, le = raw0 + s * raw_stride + mant_bytes + ln.exp_off;
+#pragma unroll
+        for (int i = 0; i < C::DQ_ITERS; ++i) {
+            asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                         : "=r"(w[s][i].x), "=r"(w[s][i].y), "=r"(w[s][i].z), "=r"(w[s][i].w)
+                         : "r"(ld + static_cast<uint32_t>(i * C::GROUP_THREADS * 16)));
+            uint16_t e2;
+            asm volatile("ld.shared.u16 %0, [%1];" : "=h"(e2) : "r"(le + static_cast<uint32_t>(i * C::ROWS_PER_ITER * 8)));
+            e[s][i] = e2;
+        }
+    }
+#pragma unroll
+    for (int s = 0; s < NS; ++s) {
+        const uint32_t st0 = dst_base + static_cast<uint32_t>(row_base0 + s * slab_rows) * 128u + ln.st_off0;
+        const uint32_t st1 = dst_base + static_cast<uint32_t>(row_base0 + s * slab_rows) * 128u + ln.st_off1;
+#pragma unroll
+        for (int i = 0; i < C::DQ_ITERS; ++i) {
+            uint32_t s0, s1;
+            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(s0) : "r"(scale_lut + (e[s][i] & 0xFFu) * 4));
+            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(s1) : "r"(scale_lut + (e[s][i] >> 8) * 4));
+            const uint32_t u0 = w[s][i].x ^ 0x80808080u, u1 = w[s][i].y ^ 0x80808080u;
+            const uint32_t u2 = w[s][i].z ^ 0x80808080u, u3 = w[s][i].w ^ 0x80808080u;
+            constexpr uint32_t kBandRows = C::ROWS_PER_ITER;
+            const uint32_t band = static_cast<uint32_t>((i * kBandRows) & 127) * 128u;     // thin slabs stay inside one group
             asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(st0 + band),
                          "r"(dequant_pair(u0, 0x4140u, s0)), "r"(dequant_pair(u0, 0x4342u, s0)),
                          "r"(dequant_pair(u1, 0x4140u, s0)), "r"(dequant_pair(u1, 0x4342u, s0))

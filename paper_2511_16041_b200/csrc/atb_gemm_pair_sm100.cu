@@ -41,8 +41,11 @@ struct PairCfg {
     // ring depths (compile-time)
     static constexpr RingPlan PLAN = plan_pair(SLAB_ROWS);
     static constexpr int NB = PLAN.nb, NG = PLAN.ng, NR = PLAN.nr;
-    static constexpr int ND = NG * SLABS;                      // dequantised slab stages
-    static constexpr int LR = ring_bars(NR, DQ_GROUPS), LD = ring_bars(ND, DQ_GROUPS);
+    // thin slabs are converted and signalled in bundles, as in atb_gemm_kernel
+    static constexpr int BUNDLE = slab_bundle(SLABS, NR, DQ_GROUPS), SPB = SLABS / BUNDLE;
+    static constexpr int ND = NG * SPB;                        // dequantised stages
+    static constexpr int LR = ring_bars(NR, DQ_GROUPS * BUNDLE), LD = ring_bars(ND, DQ_GROUPS);
+    static_assert(NR % BUNDLE == 0 && LR % BUNDLE == 0 && DQ_GROUPS * BUNDLE <= LR && LD % SPB == 0, "bundles");
     static_assert(PLAN.ok && DQ_GROUPS == PLAN.dqg, "plan");
 };
 
@@ -180,10 +183,10 @@ atb_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_c
             for (int tile = cluster_id; ok && tile < total_tiles; tile += n_clusters, acc_phase ^= 1u) {
                 for (int k = 0; ok && k < p.k_steps; ++k) {
                     if (!(ok = wait_bar_cl_spin(cx, b_full + 8 * rb.stage, rb.phase, 0x101))) break;
-                    for (int i = 0; ok && i < C::SLABS; ++i)
+                    for (int i = 0; ok && i < C::SPB; ++i)
                         ok = wait_bar_cl_spin(cx, deq_full + 8 * (rd.bar + i), rd.phase, 0x103);
                     if (!ok) break;
-                    const uint32_t as = deq_base + (rd.buf() / C::SLABS) * C::GROUP_BYTES;
+                    const uint32_t as = deq_base + (rd.buf() / C::SPB) * C::GROUP_BYTES;
                     const uint32_t bs = b_base + rb.stage * C::B_BYTES;
 #pragma unroll
                     for (int nc = 0; nc < C::N_CHUNKS; ++nc) {
@@ -200,8 +203,8 @@ atb_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_c
                         if (k == p.k_steps - 1) umma_commit_pair(acc_full + 8 * nc, 3);
                     }
                     if (!ok) break;
-                    for (int i = 0; i < C::SLABS; ++i) umma_commit_pair(deq_empty + 8 * (rd.bar + i), 3);
-                    rd.template advance<C::SLABS>();
+                    for (int i = 0; i < C::SPB; ++i) umma_commit_pair(deq_empty + 8 * (rd.bar + i), 3);
+                    rd.template advance<C::SPB>();
                     umma_commit_pair(b_empty + 8 * rb.stage, 3);
                     rb.advance(C::NB);
                 }
@@ -249,24 +252,37 @@ atb_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_c
 #endif
         Cursor<C::NR, C::LR> rr;
         Cursor<C::ND, C::LD> rd;
-        rr.start_at(my_group);
+        rr.start_at(my_group * C::BUNDLE);
         rd.start_at(my_group);
-        for (int64_t n = my_group; n < my_slabs; n += C::DQ_GROUPS) {
-            if (!wait_bar_cl(cx, raw_full + 8 * rr.bar, rr.phase, 0x301)) break;
-            if (!wait_bar_cl(cx, deq_empty + 8 * rd.freed_bar(), rd.freed_parity(), 0x302)) break;
-            const uint32_t raw = raw_base + rr.buf() * C::RAW_BYTES;
-            const uint32_t dst_base = deq_base + (rd.buf() / C::SLABS) * C::GROUP_BYTES;
-            const int row_base = (rd.buf() % C::SLABS) * SLAB_ROWS;
+        for (int64_t n = static_cast<int64_t>(my_group) * C::BUNDLE; n < my_slabs; n += C::DQ_GROUPS * C::BUNDLE) {
+            bool ok = true;
+#pragma unroll
+            for (int i = 0; i < C::BUNDLE; ++i)        // bars and buffers of a bundle are consecutive
+                ok = ok && wait_bar_cl(cx, raw_full + 8 * (rr.bar + i), rr.phase, 0x301);
+            ok = ok && wait_bar_cl(cx, deq_empty + 8 * rd.freed_bar(), rd.freed_parity(), 0x302);
+            if (!ok) break;
+            const uint32_t dst_base = deq_base + (rd.buf() / C::SPB) * C::GROUP_BYTES;
+            const int row_base0 = (rd.buf() % C::SPB) * C::BUNDLE * SLAB_ROWS;
 #ifndef ATB_PROFILE_SKIP_DEQUANT    // diagnostic: the pipeline without the conversion work (results are wrong)
-            dequant_slab<C>(ln, raw, raw + C::RAW_MANT_BYTES, scale_lut, dst_base, row_base, t, SLAB_ROWS);
+            if constexpr (C::BUNDLE > 1 && C::SLOTS % C::GROUP_THREADS == 0 && C::BUNDLE * C::DQ_ITERS <= 4) {
+                dequant_bundle<C, C::BUNDLE>(ln, raw_base + rr.buf() * C::RAW_BYTES, C::RAW_BYTES, C::RAW_MANT_BYTES, scale_lut,
+                                             dst_base, row_base0, t, SLAB_ROWS);
+            } else {
+#pragma unroll
+                for (int i = 0; i < C::BUNDLE; ++i) {
+                    const uint32_t raw = raw_base + (rr.buf() + i) * C::RAW_BYTES;
+                    dequant_slab<C>(ln, raw, raw + C::RAW_MANT_BYTES, scale_lut, dst_base, row_base0 + i * SLAB_ROWS, t, SLAB_ROWS);
+                }
+            }
 #endif
             fence_proxy_async_smem();
             __syncwarp();
             if (lane == 0) {
                 mbar_arrive_cluster(mapa_shared(deq_full + 8 * rd.bar, 0));
-                mbar_arrive(raw_empty + 8 * rr.bar);
+#pragma unroll
+                for (int i = 0; i < C::BUNDLE; ++i) mbar_arrive(raw_empty + 8 * (rr.bar + i));
             }
-            rr.template advance<C::DQ_GROUPS>();
+            rr.template advance<C::DQ_GROUPS * C::BUNDLE>();
             rd.template advance<C::DQ_GROUPS>();
         }
     }

@@ -56,10 +56,19 @@ struct Cfg {
     // ring depths (compile-time: every ring index below folds to constants)
     static constexpr RingPlan PLAN = plan_single(T_MA, T_MC, T_K, T_N);
     static constexpr int NB = PLAN.nb, NG = PLAN.ng, NR = PLAN.nr;
-    static constexpr int ND = (T_MA <= 128) ? NG * SPG : NG / GPS;   // dequantised slab stages
-    static constexpr int LR = ring_bars(NR, DQ_GROUPS), LD = ring_bars(ND, DQ_GROUPS);
+    // Thin slabs (T_MA < 128) are converted in bundles of SPG: a dequantiser group takes the SPG slabs
+    // of one 128-row operand group per barrier round trip and signals the group once, so the fixed cost
+    // of a round (waits, proxy fence, arrivals, the issuer's wait and commit) is paid per 128 rows
+    // whatever T_MA is (a shallow raw ring may force smaller bundles: slab_bundle).  Bundles, not slabs,
+    // are dealt to the dequantiser groups in turn; a raw-slab barrier must stay with one group, hence
+    // lcm(depth, groups * bundle) of them.
+    static constexpr int BUNDLE = slab_bundle(SPG, NR, DQ_GROUPS);   // slabs per bundle
+    static constexpr int SPB = SPG / BUNDLE;                          // bundles (dequantised stages) per operand group
+    static constexpr int ND = (T_MA <= 128) ? NG * SPB : NG / GPS;   // dequantised stages
+    static constexpr int LR = ring_bars(NR, DQ_GROUPS * BUNDLE), LD = ring_bars(ND, DQ_GROUPS);
+    static_assert(NR % BUNDLE == 0 && LR % BUNDLE == 0 && DQ_GROUPS * BUNDLE <= LR && LD % SPB == 0, "bundles");
     static constexpr int ACC_BUFS = PLAN.acc_bufs, TMEM_COLS = PLAN.tmem_cols;
-    static_assert(DQ_GROUPS == PLAN.dqg && ND % SPG == 0, "plan");
+    static_assert(DQ_GROUPS == PLAN.dqg, "plan");
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -189,10 +198,10 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
                         if (k == w.k_begin && !(ok = wait_bar_spin(cx, acc_empty + 8 * acc, acc_phase ^ 1u, 0x102))) break;
                         int group_slot;
                         if (T_MA <= 128) {
-                            for (int i = 0; ok && i < C::SPG; ++i)
+                            for (int i = 0; ok && i < C::SPB; ++i)
                                 ok = wait_bar_spin(cx, deq_full + 8 * (rd.bar + i), rd.phase, 0x103);
                             if (!ok) break;
-                            group_slot = rd.buf() / C::SPG;
+                            group_slot = rd.buf() / C::SPB;
                         } else {
                             if ((g % C::GPS) == 0 && !(ok = wait_bar_spin(cx, deq_full + 8 * rd.bar, rd.phase, 0x103))) break;
                             group_slot = rd.buf() * C::GPS + (g % C::GPS);
@@ -211,8 +220,8 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
                             }
                         }
                         if (T_MA <= 128) {
-                            for (int i = 0; i < C::SPG; ++i) umma_commit(deq_empty + 8 * (rd.bar + i));
-                            rd.template advance<C::SPG>();
+                            for (int i = 0; i < C::SPB; ++i) umma_commit(deq_empty + 8 * (rd.bar + i));
+                            rd.template advance<C::SPB>();
                         } else if ((g % C::GPS) == C::GPS - 1) {
                             umma_commit(deq_empty + 8 * rd.bar);
                             rd.template advance<1>();
@@ -300,31 +309,38 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
 #endif
         Cursor<C::NR, C::LR> rr;
         Cursor<C::ND, C::LD> rd;
-        rr.start_at(my_group);
+        rr.start_at(my_group * C::BUNDLE);
         rd.start_at(my_group);
-        for (int64_t n = my_group; n < my_slabs; n += C::DQ_GROUPS) {
-            if (!wait_bar(cx, raw_full + 8 * rr.bar, rr.phase, 0x301)) break;
-            if (!wait_bar(cx, deq_empty + 8 * rd.freed_bar(), rd.freed_parity(), 0x302)) break;
-            const uint32_t raw = raw_base + rr.buf() * C::RAW_BYTES;
-            uint32_t dst_base;
-            int row_base;
-            if (T_MA <= 128) {
-                dst_base = deq_base + (rd.buf() / C::SPG) * C::GROUP_BYTES;
-                row_base = (rd.buf() % C::SPG) * T_MA;
-            } else {
-                dst_base = deq_base + rd.buf() * C::GPS * C::GROUP_BYTES;
-                row_base = 0;
-            }
+        for (int64_t n = static_cast<int64_t>(my_group) * C::BUNDLE; n < my_slabs; n += C::DQ_GROUPS * C::BUNDLE) {
+            bool ok = true;
+#pragma unroll
+            for (int i = 0; i < C::BUNDLE; ++i)        // bars and buffers of a bundle are consecutive
+                ok = ok && wait_bar(cx, raw_full + 8 * (rr.bar + i), rr.phase, 0x301);
+            ok = ok && wait_bar(cx, deq_empty + 8 * rd.freed_bar(), rd.freed_parity(), 0x302);
+            if (!ok) break;
 #ifndef ATB_PROFILE_SKIP_DEQUANT    // diagnostic: the pipeline without the conversion work (results are wrong)
-            dequant_slab<C>(ln, raw, raw + C::RAW_MANT_BYTES, scale_lut, dst_base, row_base, t, T_MA);
+            // all slots of the bundle in flight at once where that is at most four per thread (registers)
+            if constexpr (C::BUNDLE > 1 && C::SLOTS % C::GROUP_THREADS == 0 && C::BUNDLE * C::DQ_ITERS <= 4) {
+                dequant_bundle<C, C::BUNDLE>(ln, raw_base + rr.buf() * C::RAW_BYTES, C::RAW_BYTES, C::RAW_MANT_BYTES, scale_lut,
+                                             deq_base + (rd.buf() / C::SPB) * C::GROUP_BYTES, (rd.buf() % C::SPB) * C::BUNDLE * T_MA, t, T_MA);
+            } else {
+#pragma unroll
+                for (int i = 0; i < C::BUNDLE; ++i) {
+                    const uint32_t raw = raw_base + (rr.buf() + i) * C::RAW_BYTES;
+                    const uint32_t dst_base = deq_base + (T_MA <= 128 ? rd.buf() / C::SPB : rd.buf() * C::GPS) * C::GROUP_BYTES;
+                    dequant_slab<C>(ln, raw, raw + C::RAW_MANT_BYTES, scale_lut, dst_base,
+                                    T_MA <= 128 ? ((rd.buf() % C::SPB) * C::BUNDLE + i) * T_MA : 0, t, T_MA);
+                }
+            }
 #endif
             fence_proxy_async_smem();
             __syncwarp();
             if (lane == 0) {
                 mbar_arrive(deq_full + 8 * rd.bar);
-                mbar_arrive(raw_empty + 8 * rr.bar);
+#pragma unroll
+                for (int i = 0; i < C::BUNDLE; ++i) mbar_arrive(raw_empty + 8 * (rr.bar + i));
             }
-            rr.template advance<C::DQ_GROUPS>();
+            rr.template advance<C::DQ_GROUPS * C::BUNDLE>();
             rd.template advance<C::DQ_GROUPS>();
         }
     }

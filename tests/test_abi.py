@@ -99,12 +99,16 @@ def test_ring_plans_fit_the_budgets():
                     n += 1
                     pair = (mc, tk, tn) == (256, 64, 512)
                     slab = min(ma, 128) if pair else ma
-                    slab_stages = p.n_a_groups * (128 // slab) if slab <= 128 else p.n_a_groups // (slab // 128)
+                    spg = max(128 // slab, 1)
+                    bundle = spg                       # slabs converted per barrier round trip
+                    while bundle > 1 and p.n_raw_stages % (bundle * p.dequant_groups):
+                        bundle //= 2
+                    stages = p.n_a_groups * (spg // bundle) if slab <= 128 else p.n_a_groups // (slab // 128)
                     assert p.dequant_groups in (1, 2, 4)
-                    assert p.n_raw_stages >= p.dequant_groups, (ma, mc, tk, tn)
-                    assert slab_stages >= 2, (ma, mc, tk, tn)
-                    assert math.lcm(p.n_raw_stages, p.dequant_groups) <= 32
-                    assert math.lcm(slab_stages, p.dequant_groups) <= 32
+                    assert p.n_raw_stages >= p.dequant_groups and p.n_raw_stages % bundle == 0, (ma, mc, tk, tn)
+                    assert stages >= 2, (ma, mc, tk, tn)
+                    assert math.lcm(p.n_raw_stages, p.dequant_groups * bundle) <= 32
+                    assert math.lcm(stages, p.dequant_groups) <= 32
                     assert p.n_b_stages >= 2 and p.acc_buffers in (1, 2)
                     assert p.smem_bytes <= 232448 and p.tmem_columns <= 512
                     assert p.tmem_columns >= p.acc_buffers * (128 if pair else mc) // 128 * tn

@@ -53,11 +53,14 @@ def lcm(a, b):
     return a * b // math.gcd(a, b)
 
 
-def simulate(n_raw, n_deq, groups, run, n_slabs, seed, lcm_bars=True, group_warps=2, land_prob=0.5, newest_first=False):
-    """Runs the protocol; returns the list of slab ids the issuer consumed.  `run` = slabs the issuer
-    takes per UMMA group (128 / T_MA for thin slabs)."""
+def simulate(n_raw, n_deq, groups, run, n_slabs, seed, lcm_bars=True, group_warps=2, land_prob=0.5, newest_first=False,
+             bundle=1):
+    """Runs the protocol; returns the list of slab ids the issuer consumed.  `bundle` = raw slabs a
+    dequantiser group converts per barrier round trip into ONE dequantised stage (thin slabs are
+    bundled up to a 128-row operand group); `run` = dequantised stages the issuer takes per UMMA group.
+    n_deq counts dequantised stages."""
     rng = random.Random(seed)
-    raw_bars = lcm(n_raw, groups) if lcm_bars else n_raw
+    raw_bars = lcm(n_raw, groups * bundle) if lcm_bars else n_raw
     deq_bars = lcm(n_deq, groups) if lcm_bars else n_deq
     raw_full = [Barrier(1) for _ in range(raw_bars)]
     raw_empty = [Barrier(group_warps) for _ in range(raw_bars)]
@@ -83,37 +86,40 @@ def simulate(n_raw, n_deq, groups, run, n_slabs, seed, lcm_bars=True, group_warp
             yield
 
     def dequantiser(g, w):
-        rr, rd = Cursor(g % n_raw, g), Cursor(g % n_deq, g)
+        rr, rd = Cursor((g * bundle) % n_raw, g * bundle), Cursor(g % n_deq, g)
         first_reuse = g
         while first_reuse < n_deq:
             first_reuse += groups
         freed = Cursor(0, first_reuse - n_deq)
-        for c in range(g, n_slabs, groups):
-            while not raw_full[rr.bar].test(rr.phase):
-                yield
-            if c >= first_reuse:
+        for st in range(g, n_slabs // bundle, groups):          # st = index of the bundle / dequantised stage
+            for i in range(bundle):
+                while not raw_full[rr.bar + i].test(rr.phase):
+                    yield
+            if st >= first_reuse:
                 while not deq_empty[freed.bar].test(freed.phase):
                     yield
                 freed.advance(groups, n_deq, deq_bars)
-            if raw_buf[rr.buf] != c:
-                errors.append(("raw", c, raw_buf[rr.buf]))
+            got = [raw_buf[(rr.buf + i) % n_raw] for i in range(bundle)]
+            if got != list(range(st * bundle, (st + 1) * bundle)):
+                errors.append(("raw", st, got))
             yield                                   # the warps of a group run at their own pace
-            deq_buf[rd.buf] = raw_buf[rr.buf]
+            deq_buf[rd.buf] = got
             yield
             deq_full[rd.bar].arrive()
-            raw_empty[rr.bar].arrive()
-            rr.advance(groups, n_raw, raw_bars)
+            for i in range(bundle):
+                raw_empty[rr.bar + i].arrive()
+            rr.advance(groups * bundle, n_raw, raw_bars)
             rd.advance(groups, n_deq, deq_bars)
             yield
 
     def issuer():
         rd = Cursor()
-        for c in range(0, n_slabs, run):
+        for c in range(0, n_slabs // bundle, run):
             for i in range(run):
                 while not deq_full[rd.bar + i].test(rd.phase):
                     yield
             for i in range(run):
-                consumed.append(deq_buf[(rd.buf + i) % n_deq])
+                consumed.extend(deq_buf[(rd.buf + i) % n_deq])
             yield                                   # the UMMAs execute
             for i in range(run):
                 deq_empty[rd.bar + i].arrive()      # tcgen05.commit
@@ -149,7 +155,15 @@ def simulate(n_raw, n_deq, groups, run, n_slabs, seed, lcm_bars=True, group_warp
     return consumed, errors
 
 
+def slab_bundle(spg, n_raw, groups):
+    b = spg
+    while b > 1 and n_raw % (b * groups):
+        b //= 2
+    return b
+
+
 def all_plans():
+    """(tiling, raw depth, dequantised stages, groups, stages per UMMA group, bundle) of every supported tiling."""
     for mc in (128, 256, 384):
         for tn in (64, 128, 256, 512):
             for tk in (64, 128):
@@ -159,24 +173,28 @@ def all_plans():
                     p = atb.atb_tiling_plan(ma, mc, tk, tn)
                     pair = (mc, tk, tn) == (256, 64, 512)
                     slab = min(ma, 128) if pair else ma
-                    n_deq = p.n_a_groups * (128 // slab) if slab <= 128 else p.n_a_groups // (slab // 128)
-                    run = 128 // slab if slab <= 128 else 1
-                    yield (ma, mc, tk, tn), p.n_raw_stages, n_deq, p.dequant_groups, run
+                    if slab <= 128:
+                        spg = 128 // slab
+                        bundle = slab_bundle(spg, p.n_raw_stages, p.dequant_groups)
+                        spb = spg // bundle
+                        yield (ma, mc, tk, tn), p.n_raw_stages, p.n_a_groups * spb, p.dequant_groups, spb, bundle
+                    else:
+                        yield (ma, mc, tk, tn), p.n_raw_stages, p.n_a_groups // (slab // 128), p.dequant_groups, 1, 1
 
 
 def test_library_ring_plans_deliver_every_slab_in_order():
     seen = set()
-    for tiling, n_raw, n_deq, groups, run in all_plans():
-        key = (n_raw, n_deq, groups, run)
+    for tiling, n_raw, n_deq, groups, run, bundle in all_plans():
+        key = (n_raw, n_deq, groups, run, bundle)
         if key in seen:
             continue
         seen.add(key)
-        n_slabs = 12 * lcm(lcm(n_raw, n_deq), groups * run)
+        n_slabs = 12 * lcm(lcm(n_raw, n_deq * bundle), groups * run * bundle)
         for seed, kw in enumerate([{}, {"land_prob": 0.05}, {"land_prob": 0.03, "newest_first": True}]):
-            consumed, errors = simulate(n_raw, n_deq, groups, run, n_slabs, seed, **kw)
+            consumed, errors = simulate(n_raw, n_deq, groups, run, n_slabs, seed, bundle=bundle, **kw)
             assert not errors, (tiling, key, errors[:3])
             assert consumed == list(range(n_slabs)), (tiling, key)
-    assert len(seen) >= 4
+    assert len(seen) >= 4 and any(k[4] > 1 for k in seen)
 
 
 @pytest.mark.parametrize("groups", [1, 2, 4])
@@ -191,6 +209,19 @@ def test_any_depth_is_safe_with_lcm_barriers(groups):
                 consumed, errors = simulate(n_raw, n_deq, groups, run, n_slabs, seed=n_raw * 100 + n_deq, **slow)
                 assert not errors, (n_raw, n_deq, groups, run, errors[:3])
                 assert consumed == list(range(n_slabs))
+
+
+def test_bundles_of_thin_slabs_are_safe_for_any_depth():
+    for groups in (2, 4):
+        for bundle in (2, 4):
+            for k in range(1, 4):
+                n_raw = k * bundle * groups // 2 if (k * bundle * groups // 2) % bundle == 0 else k * bundle * groups
+                for n_deq in (2, 3, 4, 6):
+                    n_slabs = 6 * lcm(lcm(n_raw, n_deq * bundle), groups * bundle)
+                    consumed, errors = simulate(n_raw, n_deq, groups, 1, n_slabs, seed=n_raw + n_deq, bundle=bundle,
+                                                land_prob=0.05 if n_deq & 1 else 0.5)
+                    assert not errors, (n_raw, n_deq, groups, bundle, errors[:3])
+                    assert consumed == list(range(n_slabs))
 
 
 def test_model_detects_phase_aliasing_with_one_barrier_per_buffer():
