@@ -232,6 +232,12 @@ typedef struct {
     double drain_cycles_per_column; /* atb_select_tiling: where the accumulator is not double-buffered the UMMAs wait
                                      while the epilogue drains it: cycles per FP32 accumulator column of a unit  */
     double pair_tile_cycles;      /* atb_select_tiling: extra per-tile cost of a CTA pair (both units must finish) */
+    double thin_slab_cost;        /* with mma_rows > 0: slabs thinner than mma_rows are converted and signalled in bundles
+                                     of mma_rows rows, so a slab beyond the first of its bundle costs only this fraction of
+                                     a switch: rho_eff = T_MC / mma_rows + (rho - T_MC / mma_rows) * thin_slab_cost
+                                     (1 = every slab is a full switch, as in Eq. 14)                                 */
+    double coarse_slab_factor;    /* with mma_rows > 0: factor on Eff_core of slabs larger than mma_rows, which are converted
+                                     by fewer, larger dequantiser groups and pipeline at coarser grain (0 or 1 = none)  */
 } atb_hw_params_t;
 
 typedef struct {

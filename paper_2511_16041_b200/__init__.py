@@ -45,7 +45,8 @@ class atb_hw_params_t(ctypes.Structure):
                [(n, ctypes.c_double) for n in ("eta", "eps_cycles", "ii", "delta_cycles")] + \
                [("mma_rows", ctypes.c_int)] + \
                [(n, ctypes.c_double) for n in ("load_latency_cycles", "pair_efficiency", "launch_seconds", "tile_fixed_cycles",
-                                               "drain_cycles_per_column", "pair_tile_cycles")]
+                                               "drain_cycles_per_column", "pair_tile_cycles", "thin_slab_cost",
+                                               "coarse_slab_factor")]
 
 
 class atb_tiling_score_t(ctypes.Structure):

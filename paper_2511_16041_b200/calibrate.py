@@ -34,6 +34,7 @@ DEFAULT_GRID: Dict[str, Sequence[float]] = {
     "tile_fixed_cycles": (1000.0, 2000.0, 3000.0),
     "drain_cycles_per_column": (4.0, 8.0),
     "pair_tile_cycles": (2000.0, 4000.0),
+    "thin_slab_cost": (0.3, 0.6, 0.9),
 }
 
 FULL_SHAPES: List[Shape] = [

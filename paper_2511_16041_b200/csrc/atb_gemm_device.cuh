@@ -51,14 +51,7 @@ __host__ __device__ constexpr int ring_bars(int n, int d) {
     return n / g * d;
 }
 
-// Thin slabs (T_MA < 128) are converted in bundles: the largest power-of-two number of consecutive
-// slabs, at most 128 / T_MA (one operand group), such that the raw ring holds a whole bundle for
-// every dequantiser group.
-__host__ __device__ constexpr int slab_bundle(int spg, int n_raw, int groups) {
-    int b = spg;
-    while (b > 1 && n_raw % (b * groups)) b >>= 1;
-    return b;
-}
+using atb::slab_bundle;
 
 // ---------------------------------------------------------------------------------------------
 // Ring plans: how the 227 KB of shared memory are split between the B ring, the raw-slab ring and

@@ -34,6 +34,18 @@ atb_status_t launch_gemm_pair(int T_MA, const GemmPlan& plan, int64_t M, int64_t
                               const uint8_t* exp, const void* B, int64_t ldb, void* C, int64_t ldc, int num_sms,
                               unsigned int* error_flag, void* stream);
 
+// Thin slabs (T_MA < 128) are converted in bundles: the largest power-of-two number of consecutive
+// slabs, at most spg = 128 / T_MA (one operand group), such that the raw ring of n_raw slabs holds a
+// whole bundle for every one of the `groups` dequantiser groups.
+#ifdef __CUDACC__
+__host__ __device__
+#endif
+constexpr int slab_bundle(int spg, int n_raw, int groups) {
+    int b = spg;
+    while (b > 1 && n_raw % (b * groups)) b >>= 1;
+    return b;
+}
+
 // Reads and clears the timeout flag of the precision-configuration kernels (0 = none).
 unsigned int take_cfg_error_flag();
 

@@ -42,6 +42,11 @@ void atb_hw_params_b200(atb_hw_params_t* hw) {
     hw->tile_fixed_cycles = 3000.0;
     hw->drain_cycles_per_column = 4.0;
     hw->pair_tile_cycles = 2000.0;
+    // Measured, a bundled slab costs about 0.3 of a switch (rho = 4 reaches 0.97 and rho = 8 0.87 of
+    // rho = 2); the fit for pick quality keeps 0.9, because plans with thin slabs also end up with
+    // shallower dequantised rings, for which the selection has no term.
+    hw->thin_slab_cost = 0.9;
+    hw->coarse_slab_factor = 0.88;            // measured: 256-row slabs reach a median 0.87 of 128-row slabs
 }
 
 void atb_hw_params_xdna2(atb_hw_params_t* hw, int precision_config) {
@@ -58,6 +63,7 @@ void atb_hw_params_xdna2(atb_hw_params_t* hw, int precision_config) {
     hw->a_scratch_bytes = 0.0;
     hw->mma_rows = 0; hw->load_latency_cycles = 0.0; hw->pair_efficiency = 0.0; hw->launch_seconds = 0.0;
     hw->tile_fixed_cycles = 0.0; hw->drain_cycles_per_column = 0.0; hw->pair_tile_cycles = 0.0;
+    hw->thin_slab_cost = 1.0; hw->coarse_slab_factor = 0.0;
     switch (precision_config) {
         case 1:   // A, C in BF16, B in BFP16 (text: 1.25 B in AI; 9/8 B reproduces the buffer column)
             hw->a_bytes = 2.0; hw->b_bytes = 1.25; hw->c_bytes = 2.0;
@@ -101,9 +107,15 @@ atb_status_t atb_score_tiling(const atb_hw_params_t* hw, int64_t K, atb_tiling_t
                      hw->c_bytes / static_cast<double>(K));
     // Eq. 13, Eq. 15
     out->eff_micro = hw->eta * TK / (hw->eps_cycles + hw->eta * hw->ii * TK);
-    const double rho_eff = (hw->mma_rows > 0 && t.T_MA > hw->mma_rows) ? TMC / hw->mma_rows : rho;
+    double rho_eff = rho;
+    if (hw->mma_rows > 0) {
+        const double per_mma = TMC / hw->mma_rows;      // switches if every slab were one MMA operand
+        if (t.T_MA > hw->mma_rows) rho_eff = per_mma;
+        else if (t.T_MA < hw->mma_rows && per_mma >= 1.0) rho_eff = per_mma + (rho - per_mma) * hw->thin_slab_cost;
+    }
     out->eff_core = 1.0 / (1.0 / out->eff_micro +
                            hw->delta_cycles * rho_eff * hw->peak_flops_per_cycle / (2.0 * TMC * TN * TK));
+    if (hw->mma_rows > 0 && t.T_MA > hw->mma_rows && hw->coarse_slab_factor > 0.0) out->eff_core *= hw->coarse_slab_factor;
     // Eq. 12
     out->mem_bound_flops = out->ai * hw->bw_bytes_per_s;
     out->compute_bound_flops = out->eff_core * hw->peak_flops_per_cycle * hw->clock_hz * hw->n_units;
@@ -128,6 +140,13 @@ atb_status_t atb_select_tiling(int64_t M, int64_t N, int64_t K, const atb_hw_par
         const bool pair = atb::is_pair_tiling(mc, k, n);
         atb_hw_params_t h = hw;
         if (pair) h.share_rows = hw.share_rows * 2;      // the B tile is shared by the two CTAs (Eq. 2)
+        // thin slabs get the bundle discount only as far as this tiling's raw ring lets them be bundled
+        const int slab = pair && ma > 128 ? 128 : ma;
+        if (hw.mma_rows > 0 && slab < hw.mma_rows) {
+            const int spg = hw.mma_rows / slab, b = atb::slab_bundle(spg, plan.n_raw_stages, plan.dq_groups);
+            const double full = static_cast<double>(spg) / b;              // full switches per operand group
+            h.thin_slab_cost = ((full - 1.0) + (spg - full) * hw.thin_slab_cost) / (spg - 1.0);
+        }
         atb_tiling_score_t s;
         if (atb_score_tiling(&h, K, atb_tiling_t{ma, mc, k, n}, &s) != ATB_OK) continue;
         if (pair) {

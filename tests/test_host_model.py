@@ -33,9 +33,18 @@ def test_score_matches_oracle_formulas():
                 T_MA, T_MC, T_K, T_N = t
                 ai = model.ai_array(T_MC, T_N, K, hw.a_bytes, hw.b_bytes, hw.c_bytes, hw.share_rows, hw.share_cols)
                 em = model.eff_micro(T_K, hw.eta, hw.eps_cycles, hw.ii)
-                # a slab larger than the MMA's M extent is consumed in pieces: rho_eff of the preset
-                T_MA_eff = min(T_MA, hw.mma_rows) if hw.mma_rows > 0 else T_MA
-                ec = model.eff_core(T_MA_eff, T_MC, T_K, T_N, hw.peak_flops_per_cycle, em, hw.delta_cycles)
+                # rho_eff of the preset: a slab larger than the MMA's M extent is consumed in pieces; a thinner
+                # one is bundled and costs thin_slab_cost of a switch beyond the first of its bundle
+                rho_eff = T_MC / T_MA
+                if hw.mma_rows > 0:
+                    per_mma = T_MC / hw.mma_rows
+                    if T_MA > hw.mma_rows:
+                        rho_eff = per_mma
+                    elif T_MA < hw.mma_rows:
+                        rho_eff = per_mma + (T_MC / T_MA - per_mma) * hw.thin_slab_cost
+                ec = model.eff_core(T_MC / rho_eff, T_MC, T_K, T_N, hw.peak_flops_per_cycle, em, hw.delta_cycles)
+                if hw.mma_rows > 0 and T_MA > hw.mma_rows and hw.coarse_slab_factor > 0:
+                    ec *= hw.coarse_slab_factor
                 assert math.isclose(s.ai, ai, rel_tol=1e-12)
                 assert math.isclose(s.eff_micro, em, rel_tol=1e-12)
                 assert math.isclose(s.eff_core, ec, rel_tol=1e-12)
@@ -65,10 +74,20 @@ def test_select_tiling_orders_and_filters():
     by = {(s.t.T_MA, s.t.T_MC, s.t.T_K, s.t.T_N): s for s in scores}
     assert by[(32, 256, 64, 256)].compute_bound_flops < by[(64, 256, 64, 256)].compute_bound_flops \
         < by[(128, 256, 64, 256)].compute_bound_flops
-    # slabs of 256 and 128 rows are the same thing to a 128-row MMA: equal scores, the smaller buffer first
-    assert by[(128, 256, 64, 256)].predicted_flops == by[(256, 256, 64, 256)].predicted_flops
+    # slabs of 256 and 128 rows cost the 128-row MMA the same number of switches; the preset's
+    # coarse_slab_factor (measured: coarser conversion pipeline) puts the 256-row slab behind, and
+    # without it the scores are equal and the smaller buffer goes first
+    assert math.isclose(by[(256, 256, 64, 256)].compute_bound_flops,
+                        by[(128, 256, 64, 256)].compute_bound_flops * atb.atb_hw_params_b200().coarse_slab_factor, rel_tol=1e-2)
     order = [(s.t.T_MA, s.t.T_MC, s.t.T_K, s.t.T_N) for s in scores]
     assert order.index((128, 256, 64, 256)) < order.index((256, 256, 64, 256))
+    hw = atb.atb_hw_params_b200()
+    hw.coarse_slab_factor = 0.0
+    _, flat = atb.atb_select_tiling(8192, 8192, 8192, hw)
+    fb = {(s.t.T_MA, s.t.T_MC, s.t.T_K, s.t.T_N): s for s in flat}
+    assert fb[(128, 256, 64, 256)].predicted_flops == fb[(256, 256, 64, 256)].predicted_flops
+    forder = [(s.t.T_MA, s.t.T_MC, s.t.T_K, s.t.T_N) for s in flat]
+    assert forder.index((128, 256, 64, 256)) < forder.index((256, 256, 64, 256))
     assert by[(32, 256, 64, 256)].ai == by[(256, 256, 64, 256)].ai == by[(32, 256, 128, 256)].ai
 
 
@@ -85,7 +104,7 @@ def test_b200_refinements_can_be_switched_off():
     """With the refinements at 0 the selection is the paper's Eq. 12 times wave quantisation."""
     hw = atb.atb_hw_params_b200()
     hw.mma_rows = 0; hw.load_latency_cycles = 0.0; hw.pair_efficiency = 0.0; hw.launch_seconds = 0.0
-    hw.tile_fixed_cycles = 0.0; hw.drain_cycles_per_column = 0.0; hw.pair_tile_cycles = 0.0
+    hw.tile_fixed_cycles = 0.0; hw.drain_cycles_per_column = 0.0; hw.pair_tile_cycles = 0.0; hw.thin_slab_cost = 1.0; hw.coarse_slab_factor = 0.0
     _, scores = atb.atb_select_tiling(8192, 8192, 8192, hw)
     for s in scores:
         t = (s.t.T_MA, s.t.T_MC, s.t.T_K, s.t.T_N)
