@@ -72,22 +72,31 @@ def measure(shapes: Iterable[Shape], tilings: Optional[Iterable[TilingT]] = None
     expp = torch.randint(125, 130, (exp_bytes,), dtype=torch.uint8, device=dev, generator=g)
     B = torch.randn((kn,), device=dev, generator=g).to(torch.bfloat16)
     C = torch.empty((mn,), dtype=torch.bfloat16, device=dev)
+    def time_one(M, N, K, til, n):
+        for _ in range(2):
+            atb_gemm(M, N, K, *til, mant, expp, B, C, ldb=N, ldc=N)
+        events = []
+        for _ in range(n):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            atb_gemm(M, N, K, *til, mant, expp, B, C, ldb=N, ldc=N)
+            b.record()
+            events.append((a, b))
+        torch.cuda.synchronize()
+        return min(a.elapsed_time(b) for a, b in events)
+
+    # The rate a tiling shows depends a little on what ran just before it (power state), so every shape is
+    # walked twice, in opposite orders, and a tiling keeps its better time.
     records = []
     for (M, N, K) in shapes:
+        best = {}
+        for order in (tilings, tilings[::-1]):
+            for til in order:
+                ms = time_one(M, N, K, til, max(reps // 2, 2))
+                best[til] = min(ms, best.get(til, ms))
         for til in tilings:
-            for _ in range(2):
-                atb_gemm(M, N, K, *til, mant, expp, B, C, ldb=N, ldc=N)
-            events = []
-            for _ in range(reps):
-                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                a.record()
-                atb_gemm(M, N, K, *til, mant, expp, B, C, ldb=N, ldc=N)
-                b.record()
-                events.append((a, b))
-            torch.cuda.synchronize()
-            ms = min(a.elapsed_time(b) for a, b in events)
-            records.append({"M": M, "N": N, "K": K, "tiling": list(til), "ms": ms,
-                            "tflops": 2.0 * M * N * K / ms / 1e9})
+            records.append({"M": M, "N": N, "K": K, "tiling": list(til), "ms": best[til],
+                            "tflops": 2.0 * M * N * K / best[til] / 1e9})
     atb_device_status()
     return records
 
