@@ -236,8 +236,8 @@ typedef struct {
                                      of mma_rows rows, so a slab beyond the first of its bundle costs only this fraction of
                                      a switch: rho_eff = T_MC / mma_rows + (rho - T_MC / mma_rows) * thin_slab_cost
                                      (1 = every slab is a full switch, as in Eq. 14)                                 */
-    double coarse_slab_factor;    /* with mma_rows > 0: factor on Eff_core of slabs larger than mma_rows, which are converted
-                                     by fewer, larger dequantiser groups and pipeline at coarser grain (0 or 1 = none)  */
+    double coarse_slab_factor;    /* with mma_rows > 0: factor on Eff_core of slabs larger than mma_rows: their raw ring has
+                                     fewer, larger buffers and pipelines at coarser grain (0 or 1 = none)              */
 } atb_hw_params_t;
 
 typedef struct {
