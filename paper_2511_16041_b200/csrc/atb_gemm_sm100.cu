@@ -9,7 +9,7 @@
 //   warp 0      TMA producer of B tiles
 //   warp 1      UMMA issuer (one elected lane) and owner of the TMEM allocation
 //   warps 2-5   epilogue: tcgen05.ld -> round to bf16 -> swizzled shared-memory box -> TMA store
-//   warps 6-21  dequantisers, in 2 or 4 groups that take the slabs in turn: raw slab -> bf16,
+//   warps 6-21  dequantisers, in 2 or 4 groups that take the slabs (bundles of thin slabs) in turn: raw slab -> bf16,
 //               K-major, 128-byte-swizzled operand in shared memory (exact: m * 2^(E-133) has at
 //               most 7 significant bits)
 //   warp 22     TMA producer of raw BFP16 A slabs (int8 mantissas + uint8 exponents); a warp of its
@@ -19,8 +19,9 @@
 //   raw A slabs      (n_raw_stages)  producer -> dequantisers  (freed by the dequantisers)
 //   bf16 A groups    (n_groups x 128 rows) dequantisers -> UMMA (freed by tcgen05.commit)
 //   accumulators     (acc_bufs x T_MC/128 row groups in TMEM)  UMMA -> epilogue
-// The UMMA shape is always 128 x T_N x 16.  A slab of T_MA < 128 rows is the unit of loading,
-// dequantising and signalling; 128 / T_MA consecutive slabs fill one 128-row operand group.
+// The UMMA shape is always 128 x T_N x 16.  A slab of T_MA < 128 rows is the unit of loading; the
+// 128 / T_MA consecutive slabs that fill one 128-row operand group are converted and signalled as
+// one bundle (see Cfg::BUNDLE).
 #include <algorithm>
 #include <cmath>
 
