@@ -74,7 +74,10 @@ atb_status_t atb_quantize_bfp16(const float* A_dev, int64_t M, int64_t K, int64_
  * per K-step the T_K x T_N tile of B is loaded once and rho = T_MC / T_MA slabs of A are streamed
  * through it; the T_MC x T_N FP32 accumulator is written out once, after K / T_K steps).
  * FP32 accumulation, one round-to-nearest-even to BF16 at the end.
- *   A_mant_dev, A_exp_dev: the planes described above (16-byte aligned);
+ *   A_mant_dev, A_exp_dev: the planes described above (16-byte aligned); every exponent byte is
+ *               taken as written (element = m * 2^(E-133), exactly, as a bf16 operand: bf16-subnormal for
+ *               E < 7, +-Inf where E = 255 takes it beyond bf16); mantissa -128, which the quantiser never
+ *               writes, is not a valid input;
  *   B_bf16_dev: bf16 B[K][ldb] row-major, ldb >= N, ldb % 8 == 0, 16-byte aligned;
  *   C_bf16_dev: bf16 C[M][ldc] row-major, ldc >= N, ldc % 8 == 0, 16-byte aligned (written).
  * Shapes: M >= 1 (any value), N >= 8 with N % 8 == 0, K >= 16 with K % 16 == 0.  Edge tiles in M, N and

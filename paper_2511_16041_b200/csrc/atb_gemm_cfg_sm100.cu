@@ -46,7 +46,7 @@ struct CfgK {
     static constexpr int LB = ring_bars(NB, DB), LBR = ring_bars(NBR, DB);   // barrier pairs of the B rings
     static constexpr int GROUP_WARPS = 4;
     static constexpr uint32_t SMEM_BYTES = 1024u + (NA + NB) * UNIT_BYTES + (NAR + NBR) * RAW_BYTES + 1024u +
-                                           4u * kEpilogueBoxBytes + 8u * (2 * NA + 2 * NAR + 2 * LB + 2 * LBR + 4) + 16u + 1024u;
+                                           4u * kEpilogueBoxBytes + 8u * (2 * NA + 2 * NAR + 2 * LB + 2 * LBR + 4) + 16u + kScaleTableBytes;
     static_assert(NB % 2 == 0 && LB % 2 == 0, "B tiles are pairs of units");
     static_assert(SMEM_BYTES <= kSmemBudget, "shared memory");
 };
@@ -132,7 +132,7 @@ atb_gemm_cfg_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
     }
     if (threadIdx.x >= kFirstDequantWarp * 32 && threadIdx.x < kFirstDequantWarp * 32 + 256) {
         const uint32_t E = threadIdx.x - kFirstDequantWarp * 32;
-        asm volatile("st.shared.b32 [%0], %1;" ::"r"(scale_lut + E * 4), "r"(scale_table_entry(E)) : "memory");
+        store_scale_table_entry(scale_lut, E);
     }
     tcgen05_fence_before_sync();
     __syncthreads();

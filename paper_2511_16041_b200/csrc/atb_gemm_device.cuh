@@ -41,6 +41,7 @@ constexpr int kFirstDequantWarp = 6;
 constexpr int kMaxStages = 16;
 constexpr int kMaxRingBars = 32;
 constexpr uint32_t kEpilogueBoxBytes = 32 * 128;   // 32 rows x 64 bf16 columns
+constexpr uint32_t kScaleTableBytes = 256u * 8u;  // per exponent: the scale and its offset, see scale_table_entry
 constexpr uint32_t kSmemBudget = 232448;          // 227 KB of dynamic shared memory per CTA
 constexpr uint64_t kWaitTimeoutNs = 2000000000ull;  // every mbarrier wait gives up after 2 s
 
@@ -68,7 +69,7 @@ struct RingPlan {
 
 constexpr uint32_t ring_smem_bytes(uint32_t b_bytes, uint32_t group_bytes, uint32_t raw_bytes, int acc_bars,
                                    int dqg, int bundle, int b, int g, int n_deq, int r) {
-    const uint32_t bars = 8u * (2 * b + 2 * ring_bars(r, dqg * bundle) + 2 * ring_bars(n_deq, dqg) + 2 * acc_bars) + 16u + 1024u;
+    const uint32_t bars = 8u * (2 * b + 2 * ring_bars(r, dqg * bundle) + 2 * ring_bars(n_deq, dqg) + 2 * acc_bars) + 16u + kScaleTableBytes;
     return 1024u + b * b_bytes + g * group_bytes + r * raw_bytes + 1024u + 4u * kEpilogueBoxBytes + bars;
 }
 
@@ -339,25 +340,85 @@ __device__ __forceinline__ WorkItem work_item(int item, const GemmParams& p) {
 //   2. u is positive and non-zero, so fp16 -> bf16 is pure bit arithmetic: drop 3 mantissa bits
 //      (they are zero: u has at most 8 significant bits) and re-bias the exponent by 112 -
 //      (h >> 3) + 0x3800 per half, done for both halves by one mad.hi.u32 (x * 2^29 >> 32).
-//   3. add.bf16x2 subtracts 128 (m, exact: 7 significant bits), mul.bf16x2 scales by the block's
-//      2^(E-133) (from a 256-entry table of packed bf16 pairs: normal for E >= 7, bf16-subnormal
-//      below); the product is exact for every E, subnormal results included.
-// Only the prmt runs on the integer ALU pipe - the pipe the dequantisers saturate first; the other
-// four operations go to the FMA pipe.
-__device__ __forceinline__ uint32_t dequant_pair(uint32_t u, uint32_t selector, uint32_t scale2) {
+//   3. one fma.rn.bf16x2 forms u * s - 128 * s = m * 2^(E-133) with s = 2^(E-133) and -128 * s from
+//      the block's table entry: both products are exact and so is the result (7 significant bits),
+//      bf16-subnormal results included (s is bf16-subnormal for E < 7; no flush to zero).
+// -128 * s is not a bf16 number for E >= 254: a thread that met such a block converts its slots of
+// the slab once more in the two-step form, add.bf16x2 (u - 128, exact) then mul.bf16x2 by s.
+// Only the prmt runs on the integer ALU pipe; the other operations go to the FMA pipe.
+__device__ __forceinline__ uint32_t bf16x2_of_bytes(uint32_t u, uint32_t selector) {
     const uint32_t h2 = __byte_perm(u, 0x64646464u, selector);
-    uint32_t t, b, d, r;
+    uint32_t t, b;
     asm("add.rn.f16x2 %0, %1, %2;" : "=r"(t) : "r"(h2), "r"(0xE400E400u));          // - 1024
     asm("mad.hi.u32 %0, %1, %2, %3;" : "=r"(b) : "r"(t), "r"(0x20000000u), "r"(0x38003800u));
-    asm("add.rn.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(b), "r"(0xC300C300u));          // - 128
+    return b;
+}
+__device__ __forceinline__ uint32_t dequant_pair(uint32_t u, uint32_t selector, uint32_t scale2, uint32_t offset2) {
+    uint32_t r;
+    asm("fma.rn.bf16x2 %0, %1, %2, %3;" : "=r"(r) : "r"(bf16x2_of_bytes(u, selector)), "r"(scale2), "r"(offset2));
+    return r;
+}
+__device__ __forceinline__ uint32_t dequant_pair_two_step(uint32_t u, uint32_t selector, uint32_t scale2) {
+    uint32_t d, r;
+    asm("add.rn.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(bf16x2_of_bytes(u, selector)), "r"(0xC300C300u));   // - 128
     asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(d), "r"(scale2));
     return r;
 }
 
-// Table entry for exponent E: 2^(E-133) as bf16, in both halves of the word.
-__device__ __forceinline__ uint32_t scale_table_entry(uint32_t E) {
+// Table entry for exponent E, 8 bytes: s = 2^(E-133) as bf16 in both halves of the first word,
+// -128 * s = -2^(E-126) in both halves of the second.  For E >= 254 that number does not exist and
+// the second word is 0: the only entries with bit 31 clear.  (The quantiser never writes E = 255;
+// planes from elsewhere that hold it get m * 2^122 like any other block, +-Inf beyond bf16.)
+__device__ __forceinline__ uint2 scale_table_entry(uint32_t E) {
     const uint32_t bits = (E >= 7u) ? ((E - 6u) << 7) : (1u << E);
-    return E == 255u ? 0u : bits * 0x10001u;
+    uint2 e;
+    e.x = bits * 0x10001u;
+    e.y = E >= 254u ? 0u : (0x8000u | ((E + 1u) << 7)) * 0x10001u;
+    return e;
+}
+__device__ __forceinline__ void store_scale_table_entry(uint32_t scale_lut, uint32_t E) {
+    const uint2 e = scale_table_entry(E);
+    asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(scale_lut + E * 8), "r"(e.x), "r"(e.y) : "memory");
+}
+
+// N slots of one thread: 16 mantissa bytes each (w, two's complement) of two blocks with exponents
+// (e & 0xFF, e >> 8) -> two 16-byte stores of bf16 values per slot (addresses st0[i], st1[i]).
+// FAST: the one-fma form; returns the AND of the offsets used, whose bit 31 is clear when a block
+// had E >= 254 - the caller then converts again in the two-step form (FAST = false) before it hands
+// the operand on.  The test stays off the conversion's dependency chain that way.
+template <int N, bool FAST>
+__device__ __forceinline__ uint32_t dequant_slots(const uint4 (&w)[N], const uint32_t (&e)[N], uint32_t scale_lut,
+                                                  const uint32_t (&st0)[N], const uint32_t (&st1)[N]) {
+    uint32_t all = 0xFFFFFFFFu;
+#pragma unroll
+    for (int i = 0; i < N; ++i) {
+        uint32_t s0, c0, s1, c1;
+        asm volatile("ld.shared.v2.b32 {%0, %1}, [%2];" : "=r"(s0), "=r"(c0) : "r"(scale_lut + (e[i] & 0xFFu) * 8));
+        asm volatile("ld.shared.v2.b32 {%0, %1}, [%2];" : "=r"(s1), "=r"(c1) : "r"(scale_lut + (e[i] >> 8) * 8));
+        all &= c0 & c1;
+        const uint32_t u0 = w[i].x ^ 0x80808080u, u1 = w[i].y ^ 0x80808080u;
+        const uint32_t u2 = w[i].z ^ 0x80808080u, u3 = w[i].w ^ 0x80808080u;
+        if constexpr (FAST) {
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(st0[i]),
+                         "r"(dequant_pair(u0, 0x4140u, s0, c0)), "r"(dequant_pair(u0, 0x4342u, s0, c0)),
+                         "r"(dequant_pair(u1, 0x4140u, s0, c0)), "r"(dequant_pair(u1, 0x4342u, s0, c0))
+                         : "memory");
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(st1[i]),
+                         "r"(dequant_pair(u2, 0x4140u, s1, c1)), "r"(dequant_pair(u2, 0x4342u, s1, c1)),
+                         "r"(dequant_pair(u3, 0x4140u, s1, c1)), "r"(dequant_pair(u3, 0x4342u, s1, c1))
+                         : "memory");
+        } else {
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(st0[i]),
+                         "r"(dequant_pair_two_step(u0, 0x4140u, s0)), "r"(dequant_pair_two_step(u0, 0x4342u, s0)),
+                         "r"(dequant_pair_two_step(u1, 0x4140u, s0)), "r"(dequant_pair_two_step(u1, 0x4342u, s0))
+                         : "memory");
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(st1[i]),
+                         "r"(dequant_pair_two_step(u2, 0x4140u, s1)), "r"(dequant_pair_two_step(u2, 0x4342u, s1)),
+                         "r"(dequant_pair_two_step(u3, 0x4140u, s1)), "r"(dequant_pair_two_step(u3, 0x4342u, s1))
+                         : "memory");
+        }
+    }
+    return all;
 }
 
 // Per-thread constants of the dequantiser: thread t of a group owns slot t (16 mantissas = blocks
@@ -379,7 +440,7 @@ struct DequantLane {
 
 // Dequantises one slab: raw mantissas / exponents in shared memory -> bf16 operand rows starting at
 // row `row_base` (a multiple of 32) of the 128-row groups at dst_base.
-template <class C>
+template <class C, bool FAST = true>
 __device__ __forceinline__ void dequant_slab(const DequantLane<C>& ln, uint32_t raw_mant, uint32_t raw_exp, uint32_t scale_lut,
                                              uint32_t dst_base, int row_base, int t, int T_MA_rows) {
     static_assert(C::ROWS_PER_ITER % 8 == 0 && 128 % C::ROWS_PER_ITER == 0, "band height");
@@ -400,33 +461,45 @@ __device__ __forceinline__ void dequant_slab(const DequantLane<C>& ln, uint32_t 
             e[i] = e2;
         }
     }
+    // band i starts i * ROWS_PER_ITER rows further on: possibly in the next 128-row group
+    constexpr uint32_t kBandRows = C::ROWS_PER_ITER;
+    uint32_t all = 0xFFFFFFFFu;
+    if constexpr (C::SLOTS % C::GROUP_THREADS == 0) {
+        constexpr int CHUNK = C::DQ_ITERS < 4 ? C::DQ_ITERS : 4;             // slots converted under one test
+        static_assert(C::DQ_ITERS % CHUNK == 0, "whole chunks");
 #pragma unroll
-    for (int i = 0; i < C::DQ_ITERS; ++i) {
-        if (C::SLOTS % C::GROUP_THREADS == 0 || r0 + i * C::ROWS_PER_ITER < T_MA_rows) {
-            uint32_t s0, s1;
-            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(s0) : "r"(scale_lut + (e[i] & 0xFFu) * 4));
-            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(s1) : "r"(scale_lut + (e[i] >> 8) * 4));
-            const uint32_t u0 = w[i].x ^ 0x80808080u, u1 = w[i].y ^ 0x80808080u;
-            const uint32_t u2 = w[i].z ^ 0x80808080u, u3 = w[i].w ^ 0x80808080u;
-            // band i starts i * ROWS_PER_ITER rows further on: possibly in the next 128-row group
-            constexpr uint32_t kBandRows = C::ROWS_PER_ITER;
-            const uint32_t band = static_cast<uint32_t>((i * kBandRows) >> 7) * C::GROUP_BYTES + static_cast<uint32_t>((i * kBandRows) & 127) * 128u;
-            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(st0 + band),
-                         "r"(dequant_pair(u0, 0x4140u, s0)), "r"(dequant_pair(u0, 0x4342u, s0)),
-                         "r"(dequant_pair(u1, 0x4140u, s0)), "r"(dequant_pair(u1, 0x4342u, s0))
-                         : "memory");
-            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(st1 + band),
-                         "r"(dequant_pair(u2, 0x4140u, s1)), "r"(dequant_pair(u2, 0x4342u, s1)),
-                         "r"(dequant_pair(u3, 0x4140u, s1)), "r"(dequant_pair(u3, 0x4342u, s1))
-                         : "memory");
+        for (int i0 = 0; i0 < C::DQ_ITERS; i0 += CHUNK) {
+            uint4 wc[CHUNK];
+            uint32_t ec[CHUNK], a0[CHUNK], a1[CHUNK];
+#pragma unroll
+            for (int j = 0; j < CHUNK; ++j) {
+                const int i = i0 + j;
+                const uint32_t band = static_cast<uint32_t>((i * kBandRows) >> 7) * C::GROUP_BYTES + static_cast<uint32_t>((i * kBandRows) & 127) * 128u;
+                wc[j] = w[i]; ec[j] = e[i]; a0[j] = st0 + band; a1[j] = st1 + band;
+            }
+            all &= dequant_slots<CHUNK, FAST>(wc, ec, scale_lut, a0, a1);
         }
+    } else {
+#pragma unroll
+        for (int i = 0; i < C::DQ_ITERS; ++i) {
+            if (r0 + i * C::ROWS_PER_ITER < T_MA_rows) {
+                const uint32_t band = static_cast<uint32_t>((i * kBandRows) >> 7) * C::GROUP_BYTES + static_cast<uint32_t>((i * kBandRows) & 127) * 128u;
+                const uint4 wc[1] = {w[i]};
+                const uint32_t ec[1] = {e[i]}, a0[1] = {st0 + band}, a1[1] = {st1 + band};
+                all &= dequant_slots<1, FAST>(wc, ec, scale_lut, a0, a1);
+            }
+        }
+    }
+    if constexpr (FAST) {
+        if (static_cast<int32_t>(all) >= 0)              // a block with E >= 254: rare
+            dequant_slab<C, false>(ln, raw_mant, raw_exp, scale_lut, dst_base, row_base, t, T_MA_rows);
     }
 }
 
 // A bundle of NS consecutive thin slabs (consecutive raw buffers, consecutive row ranges of one
 // 128-row operand group): all loads first, then all conversions and stores, so that a thread has
 // NS * DQ_ITERS slots in flight exactly as with one 128-row slab.
-template <class C, int NS>
+template <class C, int NS, bool FAST = true>
 __device__ __forceinline__ void dequant_bundle(const DequantLane<C>& ln, uint32_t raw0, uint32_t raw_stride, uint32_t mant_bytes,
                                                uint32_t scale_lut, uint32_t dst_base, int row_base0, int t, int slab_rows) {
     static_assert(C::SLOTS % C::GROUP_THREADS == 0, "whole iterations");
@@ -447,28 +520,25 @@ __device__ __forceinline__ void dequant_bundle(const DequantLane<C>& ln, uint32_
             e[s][i] = e2;
         }
     }
+    constexpr int N = NS * C::DQ_ITERS;                  // at most 4: the whole bundle under one test
+    uint4 wc[N];
+    uint32_t ec[N], a0[N], a1[N];
 #pragma unroll
     for (int s = 0; s < NS; ++s) {
         const uint32_t st0 = dst_base + static_cast<uint32_t>(row_base0 + s * slab_rows) * 128u + ln.st_off0;
         const uint32_t st1 = dst_base + static_cast<uint32_t>(row_base0 + s * slab_rows) * 128u + ln.st_off1;
 #pragma unroll
         for (int i = 0; i < C::DQ_ITERS; ++i) {
-            uint32_t s0, s1;
-            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(s0) : "r"(scale_lut + (e[s][i] & 0xFFu) * 4));
-            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(s1) : "r"(scale_lut + (e[s][i] >> 8) * 4));
-            const uint32_t u0 = w[s][i].x ^ 0x80808080u, u1 = w[s][i].y ^ 0x80808080u;
-            const uint32_t u2 = w[s][i].z ^ 0x80808080u, u3 = w[s][i].w ^ 0x80808080u;
             constexpr uint32_t kBandRows = C::ROWS_PER_ITER;
             const uint32_t band = static_cast<uint32_t>((i * kBandRows) & 127) * 128u;     // thin slabs stay inside one group
-            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(st0 + band),
-                         "r"(dequant_pair(u0, 0x4140u, s0)), "r"(dequant_pair(u0, 0x4342u, s0)),
-                         "r"(dequant_pair(u1, 0x4140u, s0)), "r"(dequant_pair(u1, 0x4342u, s0))
-                         : "memory");
-            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(st1 + band),
-                         "r"(dequant_pair(u2, 0x4140u, s1)), "r"(dequant_pair(u2, 0x4342u, s1)),
-                         "r"(dequant_pair(u3, 0x4140u, s1)), "r"(dequant_pair(u3, 0x4342u, s1))
-                         : "memory");
+            wc[s * C::DQ_ITERS + i] = w[s][i]; ec[s * C::DQ_ITERS + i] = e[s][i];
+            a0[s * C::DQ_ITERS + i] = st0 + band; a1[s * C::DQ_ITERS + i] = st1 + band;
         }
+    }
+    const uint32_t all = dequant_slots<N, FAST>(wc, ec, scale_lut, a0, a1);
+    if constexpr (FAST) {
+        if (static_cast<int32_t>(all) >= 0)              // a block with E >= 254: rare
+            dequant_bundle<C, NS, false>(ln, raw0, raw_stride, mant_bytes, scale_lut, dst_base, row_base0, t, slab_rows);
     }
 }
 

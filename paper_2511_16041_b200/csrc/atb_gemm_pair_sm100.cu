@@ -113,7 +113,7 @@ atb_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_c
     }
     if (threadIdx.x >= kFirstDequantWarp * 32 && threadIdx.x < kFirstDequantWarp * 32 + 256) {
         const uint32_t E = threadIdx.x - kFirstDequantWarp * 32;
-        asm volatile("st.shared.b32 [%0], %1;" ::"r"(scale_lut + E * 4), "r"(scale_table_entry(E)) : "memory");
+        store_scale_table_entry(scale_lut, E);
     }
     tcgen05_fence_before_sync();
     __syncthreads();

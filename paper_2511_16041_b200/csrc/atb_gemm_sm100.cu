@@ -101,7 +101,7 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
     const uint32_t deq_full = raw_empty + 8 * C::LR, deq_empty = deq_full + 8 * C::LD;
     const uint32_t acc_full = deq_empty + 8 * C::LD, acc_empty = acc_full + 8 * n_acc;
     const uint32_t misc = acc_empty + 8 * n_acc;             // [0]: TMEM base, [1]: abort flag
-    const uint32_t scale_lut = misc + 16;                    // 256 floats: 2^(E-133)
+    const uint32_t scale_lut = misc + 16;                    // 256 entries of 8 bytes, see scale_table_entry
     volatile uint32_t* const misc_gen = reinterpret_cast<volatile uint32_t*>(smem_gen + (misc - smem_base));
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -125,7 +125,7 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
     }
     if (threadIdx.x >= kFirstDequantWarp * 32 && threadIdx.x < kFirstDequantWarp * 32 + 256) {
         const uint32_t E = threadIdx.x - kFirstDequantWarp * 32;
-        asm volatile("st.shared.b32 [%0], %1;" ::"r"(scale_lut + E * 4), "r"(scale_table_entry(E)) : "memory");
+        store_scale_table_entry(scale_lut, E);
     }
     tcgen05_fence_before_sync();
     __syncthreads();

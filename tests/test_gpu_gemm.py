@@ -127,6 +127,34 @@ def test_permutation_A_returns_permuted_B_bitwise():
     assert np.array_equal(Cg, Bb[perm])
 
 
+def test_largest_exponents_among_ordinary_blocks_every_tiling():
+    """Blocks with E = 253 and 254 (the dequantiser converts a thread's share of a slab a second time,
+    in another form, when it meets E >= 254) and blocks with bf16-subnormal scales, sprinkled among
+    ordinary ones so that some threads of a slab take that path and others do not.  B = 2^j I makes every
+    product a single term: the result must be the dequantised element, exactly, wherever it is a normal
+    bf16 number."""
+    M, K = 520, 256
+    rng = np.random.default_rng(254)
+    mant = rng.integers(-127, 128, (M, K), dtype=np.int8)
+    exp = rng.integers(118, 136, (M, K // 8)).astype(np.uint8)
+    pick = rng.random((M, K // 8))
+    exp[pick < 0.04] = 254
+    exp[(pick >= 0.04) & (pick < 0.07)] = 253
+    exp[(pick >= 0.07) & (pick < 0.10)] = rng.integers(0, 7, int(((pick >= 0.07) & (pick < 0.10)).sum())).astype(np.uint8)
+    exp[300:428] = rng.integers(120, 130, (128, K // 8)).astype(np.uint8)      # a 128-row group without any
+    assert (exp == 254).sum() > 100
+    deq = oracle.dequantize(mant, exp)
+    for shift in (0, 60):
+        Bb = inputs.to_bf16_bits(np.eye(K, dtype=np.float32) * np.float32(2.0 ** shift))
+        want = deq * 2.0 ** shift
+        normal = ((np.abs(want) >= 2.0 ** -126) & (np.abs(want) < 2.0 ** 127)) | (want == 0)
+        assert normal.mean() > 0.85
+        assert shift != 0 or (normal & (want != 0) & (exp.repeat(8, axis=1) == 254)).sum() > 1000
+        for t in supported():
+            got = inputs.bf16_bits_to_f32(run_gemm(mant, exp, Bb, t)).astype(np.float64)
+            assert np.array_equal(got[normal], want[normal]), (t, shift)
+
+
 def test_dequant_every_exponent_through_the_kernel():
     """All 255 block exponents (incl. bf16-subnormal results and the E >= 238 branch) times all
     mantissas, read back through B = 2^j I so that the product stays a normal fp32 / bf16 value."""
