@@ -32,8 +32,10 @@ METRIC = "ATB GEMM TFLOPS (1xB200) at 8192^3 BFP16xBF16"
 DEFAULT_WORKLOAD = "cfg3_8192"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # dram__bytes_read.sum + dram__bytes_write.sum per GEMM launch of the full workload, from the 1-pass ncu
-# capture summarised in profiles/atb_gemm_kernel_dram_traffic_cfg3_8192.md (None where no capture exists).
-NCU_TRAFFIC_BYTES = {"cfg3_8192": 569.5e6 + 116.2e6}
+# captures summarised in profiles/atb_gemm_kernel_dram_traffic_cfg3_8192.md and
+# profiles/atb_gemm_pair_kernel_dram_traffic_cfg3_8192.md (None where no capture exists).
+NCU_TRAFFIC_BYTES = {("cfg3_8192", "atb_gemm_kernel"): 569.5e6 + 116.2e6,
+                     ("cfg3_8192", "atb_gemm_pair_kernel"): 608.2e6 + 117.0e6}
 
 
 def load_peaks():
@@ -335,6 +337,8 @@ def run_ours(args):
         value = aggregate_tflops(flops, world, ms_per_step)
         achieved = flops / (gemm_ms * 1e-3) / 1e12
         T_MA, T_MC, T_K, T_N = tiling_used[0]
+        # T_MC = 256, T_K = 64, T_N = 512 is the tiling that runs on a CTA pair, a kernel of its own
+        gemm_kernel = "atb_gemm_pair_kernel" if (T_MC, T_K, T_N) == (256, 64, 512) else "atb_gemm_kernel"
         line = {
             "metric": METRIC, "value": value, "unit": "TFLOPS", "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
@@ -353,11 +357,11 @@ def run_ours(args):
                     "d2h_bytes_per_step": C_host.numel() * 2, "ms_per_step": e2e_ms, "steps": e2e_steps,
                     "how": "wall clock over pipelined steps: upload, kernels and download of neighbouring steps overlap on three streams"},
             "gpu_launches": 2 * args.steps,
-            "roofline": {"bound": "tensor", "kernel": "atb_gemm_kernel", "achieved": achieved,
+            "roofline": {"bound": "tensor", "kernel": gemm_kernel, "achieved": achieved,
                          "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"],
                          "peak_source": f"{peak_src} cuBLAS bf16 burst",
                          "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"],
-                         "kernel_ms": gemm_ms, "traffic": NCU_TRAFFIC_BYTES.get(name)},
+                         "kernel_ms": gemm_ms, "traffic": NCU_TRAFFIC_BYTES.get((name, gemm_kernel))},
             "quantize": {"bound": "hbm", "achieved": M * K * 5.125 / (quant_ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
                          "unit": "GB/s", "frac": M * K * 5.125 / (quant_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
                          "kernel_ms": quant_ms},

@@ -41,6 +41,7 @@ constexpr int kFirstDequantWarp = 6;
 constexpr int kMaxStages = 16;
 constexpr int kMaxRingBars = 32;
 constexpr uint32_t kEpilogueBoxBytes = 32 * 128;   // 32 rows x 64 bf16 columns
+constexpr uint32_t kSmallBoxBytes = 32 * 64;       // 32 rows x 32 bf16 columns (the CTA-pair kernel)
 constexpr uint32_t kScaleTableBytes = 256u * 8u;  // per exponent: the scale and its offset, see scale_table_entry
 constexpr uint32_t kSmemBudget = 232448;          // 227 KB of dynamic shared memory per CTA
 constexpr uint64_t kWaitTimeoutNs = 2000000000ull;  // every mbarrier wait gives up after 2 s
@@ -68,9 +69,9 @@ struct RingPlan {
 };
 
 constexpr uint32_t ring_smem_bytes(uint32_t b_bytes, uint32_t group_bytes, uint32_t raw_bytes, int acc_bars,
-                                   int dqg, int bundle, int b, int g, int n_deq, int r) {
+                                   int dqg, int bundle, int b, int g, int n_deq, int r, uint32_t box_bytes = kEpilogueBoxBytes) {
     const uint32_t bars = 8u * (2 * b + 2 * ring_bars(r, dqg * bundle) + 2 * ring_bars(n_deq, dqg) + 2 * acc_bars) + 16u + kScaleTableBytes;
-    return 1024u + b * b_bytes + g * group_bytes + r * raw_bytes + 1024u + 4u * kEpilogueBoxBytes + bars;
+    return 1024u + b * b_bytes + g * group_bytes + r * raw_bytes + 1024u + 4u * box_bytes + bars;
 }
 
 // Single-CTA kernel, tiling (T_MA, T_MC, T_K, T_N).
@@ -150,7 +151,7 @@ constexpr RingPlan plan_pair(int slab) {
     pl.tmem_cols = 512;
     const auto total = [=](int b, int g, int r) {
         return ring_smem_bytes(b_bytes, group_bytes, raw_bytes, 2, dqg, slab_bundle(slabs, r, dqg), b, g,
-                               g * (slabs / slab_bundle(slabs, r, dqg)), r);
+                               g * (slabs / slab_bundle(slabs, r, dqg)), r, kSmallBoxBytes);
     };
     const auto bars_ok = [=](int g, int r) {
         return ring_bars(r, dqg * slab_bundle(slabs, r, dqg)) <= kMaxRingBars &&
@@ -166,6 +167,8 @@ constexpr RingPlan plan_pair(int slab) {
     // Spend what is left on bf16 groups, raw slabs (up to 8 K-steps of look-ahead), then B tiles
     // (measured: the dequantised-A ring is the one whose depth pays most).
     while (ng + ng_step <= 4 && bars_ok(ng + ng_step, nr) && total(nb, ng + ng_step, nr) <= kSmemBudget) ng += ng_step;
+    // a fifth group (the epilogue boxes of this kernel are half-size to make room for it): measured +3 %
+    if (ng == 4 && bars_ok(5, nr) && total(nb, 5, nr) <= kSmemBudget) ng = 5;
     while (nr + dqg <= kMaxStages && nr * slab < 8 * 128 && bars_ok(ng, nr + dqg) && total(nb, ng, nr + dqg) <= kSmemBudget) nr += dqg;
     while (nb < 4 && total(nb + 1, ng, nr) <= kSmemBudget) ++nb;
 #if defined(ATB_RINGS_NB) && defined(ATB_RINGS_NG) && defined(ATB_RINGS_NR)
@@ -544,24 +547,26 @@ __device__ __forceinline__ void dequant_bundle(const DequantLane<C>& ln, uint32_
 
 // ---------------------------------------------------------------------------------------------
 // Epilogues of one warp: N_COLS accumulator columns of its 32 TMEM lanes (rows row0 .. row0+31,
-// columns col0 ..) -> C.  `box` is the warp's 4 KB of staging in shared memory.  Rows and columns
+// columns col0 ..) -> C.  `box` is the warp's staging in shared memory.  Rows and columns
 // beyond M, N are clipped by the tensor map of the TMA store.
 // ---------------------------------------------------------------------------------------------
-// BF16 C: tcgen05.ld -> round to bf16 (RNE) -> 128-byte-swizzled 32 x 64 box -> TMA store.
-template <int N_COLS>
+// BF16 C: tcgen05.ld -> round to bf16 (RNE) -> swizzled box of 32 rows x BOX_COLS columns -> TMA store.
+// BOX_COLS = 64: 128-byte rows and swizzle (4 KB); 32: 64-byte rows and swizzle (2 KB).
+template <int N_COLS, int BOX_COLS = 64>
 __device__ __forceinline__ void epilogue_bf16(const CUtensorMap* tm_c, uint32_t t_addr, uint32_t box, int lane, int row0,
                                               int col0, int64_t M, int64_t N) {
-    const uint32_t my_row = box + lane * 128;
-    const uint32_t sw = static_cast<uint32_t>(lane & 7);
+    static_assert(BOX_COLS == 64 || BOX_COLS == 32, "box width");
+    const uint32_t my_row = box + lane * (BOX_COLS * 2);
+    const uint32_t sw = BOX_COLS == 64 ? static_cast<uint32_t>(lane & 7) : (static_cast<uint32_t>(lane >> 1) & 3u);
 #pragma unroll 1
-    for (int c = 0; c < N_COLS / 64; ++c) {
+    for (int c = 0; c < N_COLS / BOX_COLS; ++c) {
         // the previous TMA store of this warp must have finished reading the box
         if (lane == 0) tma_store_wait_read<0>();
         __syncwarp();
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
+        for (int h = 0; h < BOX_COLS / 32; ++h) {
             uint32_t v[32];
-            tmem_ld_32x32b_x32(t_addr + c * 64 + h * 32, v);
+            tmem_ld_32x32b_x32(t_addr + c * BOX_COLS + h * 32, v);
             tmem_ld_wait();
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
@@ -578,8 +583,8 @@ __device__ __forceinline__ void epilogue_bf16(const CUtensorMap* tm_c, uint32_t 
         }
         fence_proxy_async_smem();
         __syncwarp();
-        if (lane == 0 && row0 < M && col0 + c * 64 < N) {   // rows / columns past the edge are clipped
-            tma_store_2d(tm_c, box, col0 + c * 64, row0);
+        if (lane == 0 && row0 < M && col0 + c * BOX_COLS < N) {   // rows / columns past the edge are clipped
+            tma_store_2d(tm_c, box, col0 + c * BOX_COLS, row0);
             tma_store_commit();
         }
     }

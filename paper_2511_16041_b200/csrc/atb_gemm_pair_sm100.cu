@@ -78,7 +78,7 @@ atb_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_c
     constexpr uint32_t raw_off = C::NB * C::B_BYTES + C::NG * C::GROUP_BYTES;
     const uint32_t raw_base = smem_base + raw_off;
     constexpr uint32_t stage_off = (raw_off + C::NR * C::RAW_BYTES + 1023u) & ~1023u;
-    constexpr uint32_t bar_off = stage_off + 4u * kEpilogueBoxBytes;
+    constexpr uint32_t bar_off = stage_off + 4u * kSmallBoxBytes;
     const uint32_t bar_base = smem_base + bar_off;
     const uint32_t b_full = bar_base, b_empty = b_full + 8 * C::NB;
     const uint32_t raw_full = b_empty + 8 * C::NB, raw_empty = raw_full + 8 * C::LR;
@@ -219,13 +219,13 @@ atb_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_c
             int mt, nt;
             tile_coords(tile, p.m_tiles, p.n_tiles, mt, nt);
             const int row0 = mt * 256 + static_cast<int>(rank) * 128 + q * 32;
-            const uint32_t box = smem_base + stage_off + static_cast<uint32_t>(warp - kFirstEpilogueWarp) * kEpilogueBoxBytes;
+            const uint32_t box = smem_base + stage_off + static_cast<uint32_t>(warp - kFirstEpilogueWarp) * kSmallBoxBytes;
             for (int nc = 0; nc < C::N_CHUNKS; ++nc) {
                 if (!(ok = wait_bar_cl(cx, acc_full + 8 * nc, acc_phase, 0x201))) break;
                 tcgen05_fence_after_sync();
                 const int col0 = nt * 512 + nc * C::N_MMA;
                 const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + static_cast<uint32_t>(nc * C::N_MMA);
-                epilogue_bf16<C::N_MMA>(&tm_c, t_addr, box, lane, row0, col0, p.M, p.N);
+                epilogue_bf16<C::N_MMA, 32>(&tm_c, t_addr, box, lane, row0, col0, p.M, p.N);
                 tcgen05_fence_before_sync();
                 __syncwarp();
                 if (lane == 0) mbar_arrive_cluster(mapa_shared(acc_empty + 8 * nc, 0));
@@ -320,7 +320,7 @@ atb_status_t launch_pair_t(const atb::GemmPlan& plan, int64_t M, int64_t N, int6
         return atb::fail(ATB_ERR_CUDA, "cuTensorMapEncodeTiled failed for the exponent plane");
     if (!make_map_2d(&tm_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, B, N, K, ldb * 2, 64, C::T_K, CU_TENSOR_MAP_SWIZZLE_128B))
         return atb::fail(ATB_ERR_CUDA, "cuTensorMapEncodeTiled failed for B");
-    if (!make_map_2d(&tm_c, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Cout, N, M, ldc * 2, 64, 32, CU_TENSOR_MAP_SWIZZLE_128B))
+    if (!make_map_2d(&tm_c, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Cout, N, M, ldc * 2, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B))
         return atb::fail(ATB_ERR_CUDA, "cuTensorMapEncodeTiled failed for C");
 
     PairParams p;

@@ -37,7 +37,7 @@ void atb_hw_params_b200(atb_hw_params_t* hw) {
     hw->delta_cycles = 90.0;                  // per-slab barrier round trip of the dequantisers
     hw->mma_rows = 128;
     hw->load_latency_cycles = 1200.0;
-    hw->pair_efficiency = 0.9;
+    hw->pair_efficiency = 0.95;
     hw->launch_seconds = 1.0e-5;
     hw->tile_fixed_cycles = 3000.0;
     hw->drain_cycles_per_column = 4.0;
@@ -155,6 +155,10 @@ atb_status_t atb_select_tiling(int64_t M, int64_t N, int64_t K, const atb_hw_par
             atb_score_tiling(&h, K, atb_tiling_t{ma > 128 ? 128 : ma, 128, k, n}, &half);
             s.eff_core = half.eff_core;
             s.compute_bound_flops = half.compute_bound_flops;
+            // ... and holds its own half of the tile: Eq. 1's budgets are per CTA
+            s.feasible = half.feasible;
+            s.buf_bytes_used = half.buf_bytes_used;
+            s.acc_bytes_used = half.acc_bytes_used;
             if (hw.pair_efficiency > 0.0) s.compute_bound_flops *= hw.pair_efficiency;
         }
         // Look-ahead of the B ring (Little's law on the buffer of Eq. 1): a stage is busy from the
