@@ -278,7 +278,11 @@ atb_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_c
             fence_proxy_async_smem();
             __syncwarp();
             if (lane == 0) {
-                mbar_arrive_cluster(mapa_shared(deq_full + 8 * rd.bar, 0));
+                // CTA-scope release: the operand this publishes stays in this CTA's shared memory and is
+                // read by this CTA's tensor core (after the proxy fence above) once the leader has seen
+                // the arrival and issued the UMMA.  A cluster-scope release here kept a quarter of the
+                // dequantiser warps in membar stalls (ncu) and cost 1-2 %.
+                mbar_arrive_cluster_cta_release(mapa_shared(deq_full + 8 * rd.bar, 0));
 #pragma unroll
                 for (int i = 0; i < C::BUNDLE; ++i) mbar_arrive(raw_empty + 8 * (rr.bar + i));
             }

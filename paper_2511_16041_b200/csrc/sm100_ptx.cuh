@@ -175,6 +175,12 @@ __device__ __forceinline__ void cluster_sync_all() {
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
     asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
+// The same with CTA-scope release: enough where what the arrival publishes is read inside the arriving
+// CTA (its own shared memory, read by its own tensor core once the peer's thread issues the UMMA), and
+// much cheaper - a cluster-scope release costs every arriving warp a long membar stall.
+__device__ __forceinline__ void mbar_arrive_cluster_cta_release(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cta.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
 // Waits that must observe arrivals made by the peer CTA use cluster-scope acquire.
 __device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
     uint32_t ok;
