@@ -136,11 +136,12 @@ def evaluate(hw: atb_hw_params_t, records: Iterable[dict]) -> Dict[str, float]:
     quality, sq = [], []
     for shape, meas in _by_shape(records).items():
         _, scores = atb_select_tiling(*shape, hw=hw, max_scores=256)
-        pred = {(s.t.T_MA, s.t.T_MC, s.t.T_K, s.t.T_N): s.predicted_flops / 1e12 for s in scores}
+        ranked = [(s.t.T_MA, s.t.T_MC, s.t.T_K, s.t.T_N) for s in scores]      # the selection's own order
+        pred = {t: s.predicted_flops / 1e12 for t, s in zip(ranked, scores)}
         known = {t: v for t, v in meas.items() if t in pred}
         if not known:
             continue
-        pick = max(known, key=lambda t: (pred[t], -t[0]))
+        pick = next(t for t in ranked if t in known)
         quality.append(known[pick] / max(known.values()))
         sq += [(math.log(pred[t]) - math.log(v)) ** 2 for t, v in known.items() if v > 0 and pred[t] > 0]
     return {"pick_quality_mean": sum(quality) / len(quality), "pick_quality_min": min(quality),

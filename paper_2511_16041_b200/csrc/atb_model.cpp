@@ -37,11 +37,11 @@ void atb_hw_params_b200(atb_hw_params_t* hw) {
     hw->delta_cycles = 90.0;                  // per-slab barrier round trip of the dequantisers
     hw->mma_rows = 128;
     hw->load_latency_cycles = 1200.0;
-    hw->pair_efficiency = 0.95;
+    hw->pair_efficiency = 0.97;
     hw->launch_seconds = 1.0e-5;
     hw->tile_fixed_cycles = 3000.0;
     hw->drain_cycles_per_column = 4.0;
-    hw->pair_tile_cycles = 2000.0;
+    hw->pair_tile_cycles = 3000.0;
     // Measured, a bundled slab costs about 0.3 of a switch (rho = 4 reaches 0.97 and rho = 8 0.87 of
     // rho = 2); the fit for pick quality keeps 0.9, because plans with thin slabs also end up with
     // shallower dequantised rings, for which the selection has no term.

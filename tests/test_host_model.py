@@ -145,3 +145,16 @@ def test_per_tile_costs():
         assert (no_pair[t] > b1[t]) == ((t[1], t[2], t[3]) == (256, 64, 512)), t
     # shallow K: the CTA-pair tilings (one accumulator of 512 columns to drain per tile) are not chosen
     assert tuple(atb.atb_select_tiling(8192, 8192, 1024)[0])[3] != 512
+
+
+def test_pair_tilings_are_rated_per_cta_and_chosen_at_deep_k():
+    """A CTA of the pair holds half of the 256 x 512 tile: Eq. 1's budgets apply to that half (the whole
+    accumulator would not fit one SM's tensor memory).  The pair is measured ahead where K is deep and
+    behind where it is shallow (its single accumulator stalls the next tile), and the preset follows."""
+    best, scores = atb.atb_select_tiling(8192, 8192, 8192, max_scores=256)
+    by = {(s.t.T_MA, s.t.T_MC, s.t.T_K, s.t.T_N): s for s in scores}
+    pair = by[(128, 256, 64, 512)]
+    assert pair.feasible == 1 and pair.acc_bytes_used == 128 * 512 * 4
+    assert (best.T_MC, best.T_K, best.T_N) == (256, 64, 512)
+    shallow, _ = atb.atb_select_tiling(8192, 8192, 1024)
+    assert (shallow.T_MC, shallow.T_K, shallow.T_N) == (256, 64, 256)
