@@ -53,6 +53,8 @@ struct PairParams {
     int64_t M, N, K;
     int m_tiles, n_tiles, k_steps;           // tiles of 256 x 512
     unsigned int* error_flag;
+    uint8_t* C_exp;                          // QOUT: exponent plane of C and its padded row count
+    int64_t c_exp_rows;
 };
 
 // Bounded waits with cluster-scope acquire (the arrivals may come from the peer CTA).
@@ -63,7 +65,8 @@ __device__ __forceinline__ bool wait_bar_cl_spin(const Ctx& cx, uint32_t bar, ui
     return wait_bar_t<true, true>(cx, bar, parity, code);
 }
 
-template <int SLAB_ROWS>
+// QOUT: C is written as BFP16 planes by the quantising epilogue (see atb_gemm_bfp16_out).
+template <int SLAB_ROWS, bool QOUT = false>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 atb_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_constant__ CUtensorMap tm_exp,
                      const __grid_constant__ CUtensorMap tm_b, const __grid_constant__ CUtensorMap tm_c,
@@ -225,7 +228,10 @@ atb_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_c
                 tcgen05_fence_after_sync();
                 const int col0 = nt * 512 + nc * C::N_MMA;
                 const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + static_cast<uint32_t>(nc * C::N_MMA);
-                epilogue_bf16<C::N_MMA, 32>(&tm_c, t_addr, box, lane, row0, col0, p.M, p.N);
+                if constexpr (QOUT)
+                    epilogue_bfp16<C::N_MMA>(&tm_c, t_addr, box, lane, row0, col0, p.M, p.N, p.C_exp, p.c_exp_rows);
+                else
+                    epilogue_bf16<C::N_MMA, 32>(&tm_c, t_addr, box, lane, row0, col0, p.M, p.N);
                 tcgen05_fence_before_sync();
                 __syncwarp();
                 if (lane == 0) mbar_arrive_cluster(mapa_shared(acc_empty + 8 * nc, 0));
@@ -310,10 +316,10 @@ atb_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_c
     }
 }
 
-template <int SLAB_ROWS>
+template <int SLAB_ROWS, bool QOUT = false>
 atb_status_t launch_pair_t(const atb::GemmPlan& plan, int64_t M, int64_t N, int64_t K, const int8_t* mant,
                            const uint8_t* exp, const void* B, int64_t ldb, void* Cout, int64_t ldc, int num_sms,
-                           unsigned int* error_flag, cudaStream_t stream) {
+                           unsigned int* error_flag, cudaStream_t stream, uint8_t* C_exp = nullptr) {
     using C = PairCfg<SLAB_ROWS>;
     CUtensorMap tm_mant, tm_exp, tm_b, tm_c;
     const int64_t M_pad = atb::round_up(M, 32);
@@ -324,8 +330,12 @@ atb_status_t launch_pair_t(const atb::GemmPlan& plan, int64_t M, int64_t N, int6
         return atb::fail(ATB_ERR_CUDA, "cuTensorMapEncodeTiled failed for the exponent plane");
     if (!make_map_2d(&tm_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, B, N, K, ldb * 2, 64, C::T_K, CU_TENSOR_MAP_SWIZZLE_128B))
         return atb::fail(ATB_ERR_CUDA, "cuTensorMapEncodeTiled failed for B");
-    if (!make_map_2d(&tm_c, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Cout, N, M, ldc * 2, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B))
+    if (QOUT) {        // int8 mantissa plane C_mant[M][ldc]: boxes of 32 rows x 64 bytes
+        if (!make_map_2d(&tm_c, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Cout, N, M, ldc, 64, 32, CU_TENSOR_MAP_SWIZZLE_64B))
+            return atb::fail(ATB_ERR_CUDA, "cuTensorMapEncodeTiled failed for the mantissa plane of C");
+    } else if (!make_map_2d(&tm_c, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Cout, N, M, ldc * 2, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B)) {
         return atb::fail(ATB_ERR_CUDA, "cuTensorMapEncodeTiled failed for C");
+    }
 
     PairParams p;
     p.M = M; p.N = N; p.K = K;
@@ -333,8 +343,10 @@ atb_status_t launch_pair_t(const atb::GemmPlan& plan, int64_t M, int64_t N, int6
     p.n_tiles = static_cast<int>(atb::ceil_div(N, 512));
     p.k_steps = static_cast<int>(atb::ceil_div(K, C::T_K));
     p.error_flag = error_flag;
+    p.C_exp = C_exp;
+    p.c_exp_rows = M_pad;
 
-    auto kernel = atb_gemm_pair_kernel<SLAB_ROWS>;
+    auto kernel = atb_gemm_pair_kernel<SLAB_ROWS, QOUT>;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(plan.smem_bytes));
     if (e != cudaSuccess) return atb::fail(ATB_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
     const int64_t tiles = static_cast<int64_t>(p.m_tiles) * p.n_tiles;
@@ -352,8 +364,15 @@ namespace atb {
 
 atb_status_t launch_gemm_pair(int T_MA, const GemmPlan& plan, int64_t M, int64_t N, int64_t K, const int8_t* mant,
                               const uint8_t* exp, const void* B, int64_t ldb, void* C, int64_t ldc, int num_sms,
-                              unsigned int* error_flag, void* stream) {
+                              unsigned int* error_flag, void* stream, uint8_t* C_exp) {
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (C_exp) {       // BFP16 output: C is the int8 mantissa plane
+        switch (T_MA) {
+            case 64:  return launch_pair_t<64, true>(plan, M, N, K, mant, exp, B, ldb, C, ldc, num_sms, error_flag, st, C_exp);
+            case 128: return launch_pair_t<128, true>(plan, M, N, K, mant, exp, B, ldb, C, ldc, num_sms, error_flag, st, C_exp);
+        }
+        return atb::fail(ATB_ERR_BAD_TILING, "no pair kernel with the quantising epilogue for T_MA=%d", T_MA);
+    }
     switch (T_MA) {
         case 32:  return launch_pair_t<32>(plan, M, N, K, mant, exp, B, ldb, C, ldc, num_sms, error_flag, st);
         case 64:  return launch_pair_t<64>(plan, M, N, K, mant, exp, B, ldb, C, ldc, num_sms, error_flag, st);

@@ -684,8 +684,9 @@ extern "C" atb_status_t atb_gemm_bfp16_out(int64_t M, int64_t N, int64_t K, int 
     if (M < 1 || N < 16 || N % 16 != 0 || K < 16 || K % 16 != 0 || M > (1ll << 30) || N > (1ll << 30) || K > (1ll << 30))
         return atb::fail(ATB_ERR_BAD_SHAPE, "need M >= 1, N %% 16 == 0, K %% 16 == 0 (got %lld, %lld, %lld)", (long long)M, (long long)N, (long long)K);
     if (ldb < N || ldb % 8 != 0) return atb::fail(ATB_ERR_BAD_SHAPE, "ldb=%lld must be >= N and a multiple of 8", (long long)ldb);
-    if (!splitk_tiling_ok(T_MA, T_MC, T_K, T_N))
-        return atb::fail(ATB_ERR_BAD_TILING, "the quantising epilogue supports T_K = 64, T_MC in {128, 256}, T_N in {128, 256}, T_MA in {64, 128}");
+    const bool pair = atb::is_pair_tiling(T_MC, T_K, T_N) && (T_MA == 64 || T_MA == 128);
+    if (!pair && !splitk_tiling_ok(T_MA, T_MC, T_K, T_N))
+        return atb::fail(ATB_ERR_BAD_TILING, "the quantising epilogue supports T_K = 64, T_MA in {64, 128}, and T_MC in {128, 256} with T_N in {128, 256} or T_MC = 256 with T_N = 512");
     if (!atb::aligned16(A_mant_dev) || !atb::aligned16(A_exp_dev) || !atb::aligned16(B_bf16_dev) || !atb::aligned16(C_mant_dev) ||
         !atb::aligned16(C_exp_dev))
         return atb::fail(ATB_ERR_MISALIGNED, "all device pointers must be 16-byte aligned");
@@ -697,6 +698,9 @@ extern "C" atb_status_t atb_gemm_bfp16_out(int64_t M, int64_t N, int64_t K, int 
     if (st_dev != ATB_OK) return st_dev;
     if (dev->cc_major != 10 || dev->cc_minor != 0)
         return atb::fail(ATB_ERR_UNSUPPORTED_DEVICE, "compute capability %d.%d; this library runs on 10.0 only", dev->cc_major, dev->cc_minor);
+    if (pair)
+        return atb::launch_gemm_pair(T_MA, plan, M, N, K, A_mant_dev, A_exp_dev, B_bf16_dev, ldb, C_mant_dev, N, dev->num_sms,
+                                     dev->error_flag, stream, C_exp_dev);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
 #define ATB_QOUT_CASE(TMA_, TMC_, TN_)                                                                       \
     if (T_MA == TMA_ && T_MC == TMC_ && T_N == TN_)                                                          \

@@ -32,7 +32,7 @@ bool plan_gemm(int T_MA, int T_MC, int T_K, int T_N, GemmPlan* plan);
 inline bool is_pair_tiling(int T_MC, int T_K, int T_N) { return T_MC == 256 && T_N == 512 && T_K == 64; }
 atb_status_t launch_gemm_pair(int T_MA, const GemmPlan& plan, int64_t M, int64_t N, int64_t K, const int8_t* mant,
                               const uint8_t* exp, const void* B, int64_t ldb, void* C, int64_t ldc, int num_sms,
-                              unsigned int* error_flag, void* stream);
+                              unsigned int* error_flag, void* stream, uint8_t* C_exp = nullptr);
 
 // Thin slabs (T_MA < 128) are converted in bundles: the largest power-of-two number of consecutive
 // slabs, at most spg = 128 / T_MA (one operand group), such that the raw ring of n_raw slabs holds a

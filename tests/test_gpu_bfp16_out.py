@@ -19,6 +19,10 @@ from tests.gpu_util import dev, planes_to_dev, bf16_bits_to_dev
 pytestmark = pytest.mark.gpu
 
 TILINGS = [(64, 128, 64, 128), (128, 128, 64, 256), (64, 256, 64, 128), (128, 256, 64, 256), (64, 256, 64, 256)]
+# The CTA-pair tilings have no split-K form to read their FP32 accumulators through.  Their UMMAs add the
+# same products in the same order as the single-CTA 256 x 256 tiling, so their planes are compared with
+# that tiling's bit for bit, and with the FP64 oracle like the others.
+PAIR_TILINGS = [(64, 256, 64, 512), (128, 256, 64, 512)]
 
 
 def fp32_accumulators(M, N, K, tiling, md, ed, Bd):
@@ -58,6 +62,15 @@ def test_planes_equal_the_quantiser_on_the_fp32_accumulators(shape):
         p3 = plane.reshape(-(-N // 64), m_pad, 8)
         assert np.all(p3[:, M:, :] == 0)
         # pin (2): against the FP64 oracle
+        Cq = oracle.dequantize(got_m, got_e)
+        half_step = np.repeat(np.ldexp(1.0, got_e.astype(np.int64) - 134), 8, axis=1)
+        q_err = np.where(np.abs(got_m.astype(np.int64)) == 127, 2.0 * half_step, half_step)
+        assert np.all(np.abs(Cq - Cr) <= q_err + S * 2.0 ** -12), tiling
+    ref_m, ref_plane = run_qout(M, N, K, (128, 256, 64, 256), md, ed, Bd)
+    for tiling in PAIR_TILINGS:
+        got_m, plane = run_qout(M, N, K, tiling, md, ed, Bd)
+        assert np.array_equal(got_m, ref_m) and np.array_equal(plane, ref_plane), tiling
+        got_e = atb.exp_plane_to_logical(plane, M, N)
         Cq = oracle.dequantize(got_m, got_e)
         half_step = np.repeat(np.ldexp(1.0, got_e.astype(np.int64) - 134), 8, axis=1)
         q_err = np.where(np.abs(got_m.astype(np.int64)) == 127, 2.0 * half_step, half_step)

@@ -71,6 +71,18 @@ def test_atb_invariance_bitwise_across_T_MA():
             assert np.array_equal(Cg, ref), (ma, mc, k, n)
 
 
+def test_cta_pair_equals_the_single_cta_tiling_bitwise():
+    """The CTA-pair kernel (T_N = 512) adds the same products in the same order as the single-CTA 256 x 256
+    tiling with the same T_K: every element of C is bit-identical, ragged edges included."""
+    for (M, N, K) in [(512, 1024, 1024), (1000, 1544, 1104)]:
+        A = inputs.make_A("outlier", M, K)
+        Bb = inputs.make_B_bits(K, N, None)
+        mant, exp = oracle.quantize_bfp16(A)
+        ref = run_gemm(mant, exp, Bb, (128, 256, 64, 256))
+        for ma in (32, 64, 128, 256):
+            assert np.array_equal(run_gemm(mant, exp, Bb, (ma, 256, 64, 512)), ref), (M, N, K, ma)
+
+
 def test_rho_that_is_not_a_power_of_two():
     """T_MC = 384 (three 128-row groups): rho = 3, 6 and 12 (the paper's Table 2 uses rho = 6).  Several
     tiles and ragged tails; bitwise equal across T_MA like every other (T_MC, T_K, T_N)."""
