@@ -16,6 +16,8 @@
 //
 // Warp roles are those of the single-CTA kernel: 0 TMA producer of B, 1 UMMA issuer (active in the
 // leader only) + TMEM owner, 2-5 epilogue, 6-21 dequantisers (4 groups of 4 warps), 22 TMA producer of A.
+// The epilogue stages C in boxes of 32 x 32 BF16 (2 KB, half the single-CTA kernel's), which leaves
+// room for a fifth dequantised-operand group.
 #include "atb_gemm_device.cuh"
 
 namespace {
