@@ -250,7 +250,7 @@ def _sampled_rows(M, T_MC, n_random, seed):
 
 @pytest.mark.parametrize("name,tilings", [
     ("cfg2_4096", [(32, 256, 64, 256), (64, 256, 64, 256), (128, 256, 64, 256), (256, 256, 64, 256)]),
-    ("cfg3_8192", ["selected", (256, 256, 64, 256), (128, 256, 64, 512)]),
+    ("cfg3_8192", ["selected", (128, 256, 64, 256), (256, 256, 64, 256), (128, 256, 64, 512)]),
     ("cfg4_ffn_up", ["selected"]),
     ("cfg4_ffn_down", ["selected"]),
 ])
