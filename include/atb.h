@@ -242,6 +242,9 @@ typedef struct {
                                      (1 = every slab is a full switch, as in Eq. 14)                                 */
     double coarse_slab_factor;    /* with mma_rows > 0: factor on Eff_core of slabs larger than mma_rows: their raw ring has
                                      fewer, larger buffers and pipelines at coarser grain (0 or 1 = none)              */
+    double deep_kstep_factor;     /* with mma_rows > 0: factor on Eff_core of tilings with T_K > 64: a dequantiser group then
+                                     converts an mma_rows x T_K unit in one piece, twice the latency per hand-over with
+                                     the same number of buffers (0 or 1 = none)                                        */
 } atb_hw_params_t;
 
 typedef struct {

@@ -46,7 +46,7 @@ class atb_hw_params_t(ctypes.Structure):
                [("mma_rows", ctypes.c_int)] + \
                [(n, ctypes.c_double) for n in ("load_latency_cycles", "pair_efficiency", "launch_seconds", "tile_fixed_cycles",
                                                "drain_cycles_per_column", "pair_tile_cycles", "thin_slab_cost",
-                                               "coarse_slab_factor")]
+                                               "coarse_slab_factor", "deep_kstep_factor")]
 
 
 class atb_tiling_score_t(ctypes.Structure):

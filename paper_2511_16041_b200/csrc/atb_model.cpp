@@ -41,12 +41,13 @@ void atb_hw_params_b200(atb_hw_params_t* hw) {
     hw->launch_seconds = 1.0e-5;
     hw->tile_fixed_cycles = 3000.0;
     hw->drain_cycles_per_column = 4.0;
-    hw->pair_tile_cycles = 3000.0;
+    hw->pair_tile_cycles = 4000.0;
     // Measured, a bundled slab costs about 0.3 of a switch (rho = 4 reaches 0.97 and rho = 8 0.87 of
     // rho = 2); the fit for pick quality keeps 0.9, because plans with thin slabs also end up with
     // shallower dequantised rings, for which the selection has no term.
     hw->thin_slab_cost = 0.9;
     hw->coarse_slab_factor = 0.88;            // measured: 256-row slabs reach a median 0.87 of 128-row slabs
+    hw->deep_kstep_factor = 0.7;              // measured: T_K = 128 reaches 0.62-0.65 of T_K = 64 at T_N = 128, 0.86 at T_N = 64; the look-ahead term carries a part of it already
 }
 
 void atb_hw_params_xdna2(atb_hw_params_t* hw, int precision_config) {
@@ -63,7 +64,7 @@ void atb_hw_params_xdna2(atb_hw_params_t* hw, int precision_config) {
     hw->a_scratch_bytes = 0.0;
     hw->mma_rows = 0; hw->load_latency_cycles = 0.0; hw->pair_efficiency = 0.0; hw->launch_seconds = 0.0;
     hw->tile_fixed_cycles = 0.0; hw->drain_cycles_per_column = 0.0; hw->pair_tile_cycles = 0.0;
-    hw->thin_slab_cost = 1.0; hw->coarse_slab_factor = 0.0;
+    hw->thin_slab_cost = 1.0; hw->coarse_slab_factor = 0.0; hw->deep_kstep_factor = 0.0;
     switch (precision_config) {
         case 1:   // A, C in BF16, B in BFP16 (text: 1.25 B in AI; 9/8 B reproduces the buffer column)
             hw->a_bytes = 2.0; hw->b_bytes = 1.25; hw->c_bytes = 2.0;
@@ -116,6 +117,7 @@ atb_status_t atb_score_tiling(const atb_hw_params_t* hw, int64_t K, atb_tiling_t
     out->eff_core = 1.0 / (1.0 / out->eff_micro +
                            hw->delta_cycles * rho_eff * hw->peak_flops_per_cycle / (2.0 * TMC * TN * TK));
     if (hw->mma_rows > 0 && t.T_MA > hw->mma_rows && hw->coarse_slab_factor > 0.0) out->eff_core *= hw->coarse_slab_factor;
+    if (hw->mma_rows > 0 && t.T_K > 64 && hw->deep_kstep_factor > 0.0) out->eff_core *= hw->deep_kstep_factor;
     // Eq. 12
     out->mem_bound_flops = out->ai * hw->bw_bytes_per_s;
     out->compute_bound_flops = out->eff_core * hw->peak_flops_per_cycle * hw->clock_hz * hw->n_units;

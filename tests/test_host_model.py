@@ -45,6 +45,8 @@ def test_score_matches_oracle_formulas():
                 ec = model.eff_core(T_MC / rho_eff, T_MC, T_K, T_N, hw.peak_flops_per_cycle, em, hw.delta_cycles)
                 if hw.mma_rows > 0 and T_MA > hw.mma_rows and hw.coarse_slab_factor > 0:
                     ec *= hw.coarse_slab_factor
+                if hw.mma_rows > 0 and T_K > 64 and hw.deep_kstep_factor > 0:
+                    ec *= hw.deep_kstep_factor
                 assert math.isclose(s.ai, ai, rel_tol=1e-12)
                 assert math.isclose(s.eff_micro, em, rel_tol=1e-12)
                 assert math.isclose(s.eff_core, ec, rel_tol=1e-12)
@@ -104,7 +106,7 @@ def test_b200_refinements_can_be_switched_off():
     """With the refinements at 0 the selection is the paper's Eq. 12 times wave quantisation."""
     hw = atb.atb_hw_params_b200()
     hw.mma_rows = 0; hw.load_latency_cycles = 0.0; hw.pair_efficiency = 0.0; hw.launch_seconds = 0.0
-    hw.tile_fixed_cycles = 0.0; hw.drain_cycles_per_column = 0.0; hw.pair_tile_cycles = 0.0; hw.thin_slab_cost = 1.0; hw.coarse_slab_factor = 0.0
+    hw.tile_fixed_cycles = 0.0; hw.drain_cycles_per_column = 0.0; hw.pair_tile_cycles = 0.0; hw.thin_slab_cost = 1.0; hw.coarse_slab_factor = 0.0; hw.deep_kstep_factor = 0.0
     _, scores = atb.atb_select_tiling(8192, 8192, 8192, hw)
     for s in scores:
         t = (s.t.T_MA, s.t.T_MC, s.t.T_K, s.t.T_N)
