@@ -273,7 +273,9 @@ atb_status_t atb_score_tiling(const atb_hw_params_t* hw, int64_t K, atb_tiling_t
 /* Tiling selection (Section 5: the trade-off between arithmetic intensity, which wants small T_K
  * and large rho, and core efficiency, which wants the opposite): enumerates the tilings atb_gemm
  * supports, scores each with atb_score_tiling for this (M, N, K) - including the loss from
- * partially filled waves of output tiles over n_units - and returns them best first.
+ * partially filled waves of output tiles over n_units - and returns them best first.  A CTA-pair
+ * tiling (T_MC = 256, T_N = 512) is rated per CTA: feasible, buf_bytes_used, acc_bytes_used, eff_core
+ * and the compute bound are those of the 128-row half tile one CTA holds, with the B tile shared by two.
  *   hw:       NULL = atb_hw_params_b200().
  *   best:     receives the top feasible tiling (may be NULL).
  *   scores:   optional array of *n_scores entries, filled best first; *n_scores receives the
