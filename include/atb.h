@@ -11,7 +11,9 @@
  *     pointers without that suffix are HOST memory.  The library never allocates or frees device
  *     memory and keeps no reference to caller memory after a call returns.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Device work is
- *     asynchronous on that stream; the calls return as soon as it is enqueued.
+ *     asynchronous on that stream; the calls return as soon as it is enqueued.  They only enqueue kernels
+ *     (tensor maps travel by value as kernel parameters), so a sequence of calls can be captured into a
+ *     CUDA graph and replayed on the same buffers.
  *   - Argument errors are returned synchronously and nothing is launched.  No exception or abort
  *     crosses this boundary.  atb_last_error_message() gives a per-thread detail string.
  *   - The device must have compute capability 10.0; there is no fallback of any kind.

@@ -79,3 +79,40 @@ def test_calibration_measures_and_fits_on_this_gpu(tmp_path):
     assert len(records) == 10 and all(r["tflops"] > 10 for r in records)
     values, ev = calibrate.fit(records, {"a_bytes": (3.0, 3.6), "load_latency_cycles": (1200.0, 2000.0)})
     assert set(values) == {"a_bytes", "load_latency_cycles"} and 0.5 < ev["pick_quality_mean"] <= 1.0
+
+
+def test_quantise_and_gemm_capture_into_a_cuda_graph():
+    """The entry points only enqueue work on the given stream (tensor maps travel by value as kernel
+    parameters), so a step can be captured once and replayed: the replay gives the eager result bit for
+    bit, also after the input buffers were refilled."""
+    device = dev()
+    gen = torch.Generator(device=device)
+    gen.manual_seed(5)
+    M, N, K = 1000, 1544, 1104
+    A = torch.randn((M, K), device=device, generator=gen)
+    B = torch.randn((K, N), device=device, generator=gen).to(torch.bfloat16)
+    mant = torch.empty((M, K), dtype=torch.int8, device=device)
+    plane = torch.empty(atb.atb_bfp16_exp_bytes(M, K), dtype=torch.uint8, device=device)
+    eager = torch.empty((M, N), dtype=torch.bfloat16, device=device)
+    replayed = torch.zeros((M, N), dtype=torch.bfloat16, device=device)
+    s = torch.cuda.Stream(device)
+    for tiling in [(128, 256, 64, 256), (128, 256, 64, 512)]:
+        def step(out):
+            atb.atb_quantize_bfp16(A, mant, plane, stream=s)
+            atb.atb_gemm(M, N, K, *tiling, mant, plane, B, out, stream=s)
+        with torch.cuda.stream(s):
+            step(eager)                      # also the warm-up the capture needs
+        s.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=s):
+            step(replayed)
+        for _ in range(2):
+            replayed.zero_()
+            graph.replay()
+            torch.cuda.synchronize()
+            with torch.cuda.stream(s):
+                step(eager)
+            s.synchronize()
+            assert torch.equal(eager, replayed), tiling
+            A.mul_(1.5)                      # new values in the same buffers for the second round
+    atb.atb_device_status()
