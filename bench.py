@@ -12,6 +12,14 @@ against the measured dense-BF16 cuBLAS peak.  ``e2e`` repeats the step with host
 host A and B are copied to the device and C is copied back inside the timed region.
 ``cpu_baseline`` times the FP64 oracle on the host cores on a bounded row sample (a reported
 baseline, not a target).  ``--impl reference`` times that oracle alone.
+
+After the timed region, on one GPU, the line also gets ``ablation`` - the GEMM alone under every T_MA
+of the single-CTA 256 x 256 family and of the CTA-pair 256 x 512 family, the symmetric form first, with
+the best asymmetric rate over the symmetric one - and ``roofline.sustained``: the headline GEMM
+launched back to back for more than 2 s (the GPU settles under its power cap) against the sustained
+cuBLAS figure, with the SM clock sampled meanwhile.
+
+``--gpus N`` without a launcher around it (no WORLD_SIZE in the environment) starts N ranks itself.
 """
 from __future__ import annotations
 
@@ -31,11 +39,33 @@ sys.path.insert(0, ROOT)
 METRIC = "ATB GEMM TFLOPS (1xB200) at 8192^3 BFP16xBF16"
 DEFAULT_WORKLOAD = "cfg3_8192"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# dram__bytes_read.sum + dram__bytes_write.sum per GEMM launch of the full workload, from the 1-pass ncu
-# captures summarised in profiles/atb_gemm_kernel_dram_traffic_cfg3_8192.md and
-# profiles/atb_gemm_pair_kernel_dram_traffic_cfg3_8192.md (None where no capture exists).
-NCU_TRAFFIC_BYTES = {("cfg3_8192", "atb_gemm_kernel"): 569.5e6 + 116.2e6,
-                     ("cfg3_8192", "atb_gemm_pair_kernel"): 608.2e6 + 117.0e6}
+NOMINAL_BF16_TFLOPS = 2250.0        # NVIDIA's dense BF16 figure for B200 (context beside the measured peak)
+# The asymmetric-buffering ablation: for fixed (T_MC, T_K, T_N) only T_MA moves, the first entry of
+# each family is its symmetric form.  On the CTA pair each SM holds 128 rows of the 256-row tile, so
+# T_MA = 128 is symmetric there.
+ABLATION_FAMILIES = {
+    "single_cta_256x256": [(256, 256, 64, 256), (128, 256, 64, 256), (64, 256, 64, 256), (32, 256, 64, 256)],
+    "cta_pair_256x512": [(128, 256, 64, 512), (64, 256, 64, 512), (32, 256, 64, 512)],
+}
+SUSTAINED_SECONDS = 2.2
+
+
+def load_ncu_traffic():
+    """dram__bytes_read.sum + dram__bytes_write.sum per GEMM launch, from the 1-pass ncu captures of the
+    full launch that are summarised beside this table (None where no capture exists)."""
+    try:
+        with open(os.path.join(ROOT, "profiles", "ncu_dram_traffic.json")) as f:
+            rows = json.load(f)["launches"]
+        return {(r["workload"], r["kernel"]): float(r["dram_read_bytes"]) + float(r["dram_write_bytes"]) for r in rows}
+    except Exception:
+        return {}
+
+
+def rho_per_core(t):
+    """rho = T_MC / T_MA as one SM sees it: the CTA-pair tiling keeps 128 of its 256 rows per SM."""
+    T_MA, T_MC, T_K, T_N = t
+    rows = 128 if (T_MC, T_K, T_N) == (256, 64, 512) else T_MC
+    return rows // min(T_MA, rows)
 
 
 def load_peaks():
@@ -193,6 +223,37 @@ def run_reference(args):
     return 0
 
 
+def spawn_ranks(args) -> int:
+    """``python bench.py --gpus N`` outside a launcher: start N ranks of this script, one per GPU, under
+    torch.distributed.run on 127.0.0.1 (the same command line a launcher would use)."""
+    import socket
+    import subprocess
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
+
+
+def run_stub(args) -> int:
+    """--stub-step: the rank plumbing of run_ours (rendezvous, barrier, max over ranks, whole-job figure,
+    one line from rank 0) with a pretend step time instead of GPU work; gloo on CPU."""
+    import torch
+    import torch.distributed as dist
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    if world > 1:
+        dist.init_process_group("gloo")
+        dist.barrier()
+    ms = max_over_ranks([1.0 + rank], torch.device("cpu"), world)[0]
+    if rank == 0:
+        print(json.dumps({"stub": True, "n_gpus": world, "ms_per_step": ms, "value": aggregate_tflops(1e9, world, ms)}))
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -204,6 +265,8 @@ def run_ours(args):
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     if not torch.cuda.is_available():
         raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback of the hot path")
+    if local_rank >= torch.cuda.device_count():
+        raise RuntimeError(f"rank {rank} wants GPU {local_rank} but only {torch.cuda.device_count()} are visible")
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
     if world > 1:
@@ -328,6 +391,55 @@ def run_ours(args):
     stream.synchronize()
     quant_ms = q0.elapsed_time(q1) / 10
 
+    # ---------------- the T_MA ablation and a sustained leg (one GPU only) ----------------
+    ablation = sustained = None
+    if world == 1 and not args.no_ablation:
+        def time_gemm(t, reps):
+            for _ in range(2):
+                atb.atb_gemm(M, N, K, *t, mant, plane, B_dev, C_dev, stream=stream)
+            evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+            for a, b in evs:
+                a.record(stream)
+                atb.atb_gemm(M, N, K, *t, mant, plane, B_dev, C_dev, stream=stream)
+                b.record(stream)
+            stream.synchronize()
+            return min(a.elapsed_time(b) for a, b in evs)
+
+        # every tiling of both families in one process, walked in two opposite orders (what ran just
+        # before moves a rate by a few per cent); a tiling keeps its better time
+        walk = [t for fam in ABLATION_FAMILIES.values() for t in fam]
+        best_ms = {}
+        for order in (walk, walk[::-1]):
+            for t in order:
+                ms = time_gemm(t, 5)
+                best_ms[t] = min(ms, best_ms.get(t, ms))
+        atb.atb_device_status(stream)
+        tf = lambda t: 2.0 * M * N * K / (best_ms[t] * 1e-3) / 1e12
+        ablation = {"how": "atb_gemm alone on the resident planes; both families interleaved in one process, "
+                           "two opposite orders, best of 2 x 5 launches per tiling (CUDA events)",
+                    "families": {}, "atb_over_symmetric": {}}
+        for fam, tilings in ABLATION_FAMILIES.items():
+            ablation["families"][fam] = [{"tiling": list(t), "rho_per_core": rho_per_core(t), "tflops": tf(t)} for t in tilings]
+            ablation["atb_over_symmetric"][fam] = max(tf(t) for t in tilings[1:]) / tf(tilings[0])
+
+        # sustained: the headline GEMM back to back for >= 2 s, so that the GPU settles under its power cap
+        t_head = tiling_used[0]
+        n_launch = max(200, int(SUSTAINED_SECONDS * 1e3 / gemm_ms))
+        s_sampler = ClockSampler(physical_gpu_index(local_rank))
+        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        stream.synchronize()
+        s_sampler.start()
+        s0.record(stream)
+        for _ in range(n_launch):
+            atb.atb_gemm(M, N, K, *t_head, mant, plane, B_dev, C_dev, stream=stream)
+        s1.record(stream)
+        stream.synchronize()
+        s_clocks = s_sampler.stop()
+        atb.atb_device_status(stream)
+        s_ms = s0.elapsed_time(s1)
+        sustained = {"launches": n_launch, "seconds": s_ms * 1e-3,
+                     "achieved": 2.0 * M * N * K * n_launch / (s_ms * 1e-3) / 1e12, "clocks": s_clocks}
+
     total_ms, gemm_ms, e2e_ms, quant_ms = max_over_ranks([total_ms, gemm_ms, e2e_ms, quant_ms], dev, world)
 
     if rank == 0:
@@ -346,7 +458,11 @@ def run_ours(args):
             "config": {"workload": name, "M": M, "N": N, "K": K,
                        "A": f"BFP16 quantised on device from seeded {c['A']} fp32", "B": "bf16, seeded normal",
                        "tiling": {"T_MA": T_MA, "T_MC": T_MC, "T_K": T_K, "T_N": T_N,
-                                  "chosen_by": "flag" if args.tiling else "atb_select_tiling"},
+                                  "chosen_by": "flag" if args.tiling else "atb_select_tiling",
+                                  "rho_per_core": rho_per_core((T_MA, T_MC, T_K, T_N)),
+                                  "note": ("CTA-pair tiling: each SM holds 128 of the 256 rows, so T_MA = 128 buffers "
+                                           "symmetrically per SM and the B tile is shared by two SMs (Eq. 2)")
+                                  if gemm_kernel == "atb_gemm_pair_kernel" else "single-CTA tiling"},
                        "step": "atb_quantize_bfp16 + atb_select_tiling + atb_gemm",
                        "l2": "inputs larger than L2 (A fp32 %d MB, B %d MB, C %d MB per step)" % (
                            M * K * 4 >> 20, K * N * 2 >> 20, M * N * 2 >> 20),
@@ -359,13 +475,24 @@ def run_ours(args):
             "gpu_launches": 2 * args.steps,
             "roofline": {"bound": "tensor", "kernel": gemm_kernel, "achieved": achieved,
                          "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"],
-                         "peak_source": f"{peak_src} cuBLAS bf16 burst",
-                         "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"],
-                         "kernel_ms": gemm_ms, "traffic": NCU_TRAFFIC_BYTES.get((name, gemm_kernel))},
+                         "peak_source": f"{peak_src} cuBLAS bf16 burst (a kernel timed alone, launch by launch)",
+                         "frac_of_nominal": achieved / NOMINAL_BF16_TFLOPS, "nominal_peak": NOMINAL_BF16_TFLOPS,
+                         "kernel_ms": gemm_ms, "traffic": load_ncu_traffic().get((name, gemm_kernel)),
+                         "compulsory_bytes": 1.125 * M * K + 2.0 * K * N + 2.0 * M * N},
             "quantize": {"bound": "hbm", "achieved": M * K * 5.125 / (quant_ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
                          "unit": "GB/s", "frac": M * K * 5.125 / (quant_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
                          "kernel_ms": quant_ms},
         }
+        if sustained is not None:
+            mhz = sustained["clocks"].get("sm_mhz")
+            sustained.update({"peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                              "frac": sustained["achieved"] / peaks["bf16_tflops_sustained"],
+                              "peak_source": f"{peak_src} cuBLAS bf16 back to back under the power cap",
+                              "frac_of_nominal": sustained["achieved"] / NOMINAL_BF16_TFLOPS,
+                              "flop_per_cycle_per_sm": (sustained["achieved"] * 1e12 / (148 * mhz * 1e6)) if mhz else None})
+            line["roofline"]["sustained"] = sustained
+        if ablation is not None:
+            line["ablation"] = ablation
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_oracle_sample(name, args.cpu_seconds)
         print(json.dumps(line))
@@ -477,11 +604,18 @@ def main():
     ap.add_argument("--tiling", type=int, nargs=4, metavar=("T_MA", "T_MC", "T_K", "T_N"), default=None)
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-ablation", action="store_true", help="skip the T_MA ablation and the sustained leg")
+    ap.add_argument("--stub-step", action="store_true",
+                    help="host-only rehearsal of the multi-rank plumbing (gloo, no GPU work); the line is marked as a stub")
     ap.add_argument("--entry", default="gemm", choices=["gemm", "bfp16_out", "config1", "config2"],
                     help="gemm: the headline hot path (default); the others time the further entry points")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        return spawn_ranks(args)
+    if args.stub_step:
+        return run_stub(args)
     if args.entry != "gemm":
         return run_entry(args)
     return run_ours(args)

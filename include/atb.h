@@ -89,6 +89,11 @@ atb_status_t atb_quantize_bfp16(const float* A_dev, int64_t M, int64_t K, int64_
  *          T_MC = 384 gives the ratios that are not powers of two); (T_MC / 128) * T_N <= 512 (the FP32
  *          accumulator must fit the 512 TMEM columns); the shared-memory rings must fit 227 KB.
  *          atb_tiling_supported() tells in advance.
+ *          (T_MC, T_K, T_N) = (256, 64, 512) runs on a pair of SMs (tcgen05 cta_group::2): each SM holds 128
+ *          rows of the tile and the whole 512-column accumulator for them, the B tile is shared by the two
+ *          (the array-level sharing of Eq. 2).  Per SM - the paper's "core" - the accumulator is 128 rows
+ *          tall, so T_MA = 128 is this tiling's SYMMETRIC form (rho per core = 128 / T_MA), only
+ *          T_MA in {32, 64} buffer asymmetrically, and T_MA = 256 does not exist (ATB_ERR_BAD_TILING).
  * For fixed (T_MC, T_K, T_N) the result is bit-identical for every T_MA.
  * Errors: NULL_POINTER, BAD_SHAPE, BAD_TILING, MISALIGNED, UNSUPPORTED_DEVICE, CUDA. */
 atb_status_t atb_gemm(int64_t M, int64_t N, int64_t K, int T_MA, int T_MC, int T_K, int T_N,
@@ -102,7 +107,8 @@ atb_status_t atb_gemm(int64_t M, int64_t N, int64_t K, int T_MA, int T_MC, int T
  * stream.  The paper's hardware cannot do this - Section 2.2: an AIE core has no way to bring partial
  * sums back, so every output tile is fully accumulated in L1 - here partial sums go through L2/HBM.
  * Same operands and rules as atb_gemm.  Tilings: T_K = 64, T_MC in {128, 256}, T_N in {128, 256},
- * T_MA in {64, 128}.  splits in [1, min(64, ceil(K / T_K))].
+ * T_MA in {64, 128}.  splits in [1, min(64, ceil(K / T_K))]; splits * roundup(M, T_MC) must stay below 2^31
+ * (the row coordinate of the partial tiles is a 32-bit TMA coordinate), else ATB_ERR_BAD_SHAPE.
  *   workspace_dev: device memory, 16-byte aligned, at least atb_gemm_splitk_workspace_bytes() bytes;
  *                  fully overwritten; may be reused by the next call on the same stream.
  * Errors: as atb_gemm, plus ATB_ERR_BUFFER_TOO_SMALL. */
@@ -135,6 +141,12 @@ int atb_select_splits(int64_t M, int64_t N, int64_t K, int T_MC, int T_K, int T_
  *   - The call itself performs no cudaMalloc / cudaFree and calls no allocating library routine.
  *   - The first call on each device looks the array's device address up (cudaGetSymbolAddress, with
  *     that device current) and remembers it; make that first call before starting any stream capture.
+ *   - When the array's memory is actually set aside: when the CUDA runtime loads the library's GEMM module
+ *     on a device.  With lazy module loading (the default of recent CUDA versions) that happens inside the
+ *     first GEMM-family call of this library on that device - possibly this one - and it can fail there
+ *     with ATB_ERR_CUDA if the device has less than ATB_NOALLOC_SCRATCH_BYTES free.  So make one priming
+ *     call (any small atb_gemm or this entry point) per device at start-up, BEFORE handing the rest of the
+ *     device memory to a pool; after it, no call of this entry point changes the amount of free memory.
  *   - All calls share the one array and it keeps whatever the last call left there.  Nothing has to be
  *     cleared: every partial sum the reduction reads is written earlier by the same call.  For the same
  *     reason two calls whose kernels can run at the same time on one GPU (different streams, or
@@ -207,9 +219,11 @@ atb_status_t atb_tiling_plan(int T_MA, int T_MC, int T_K, int T_N, atb_plan_t* p
 
 /* Waits for `stream` and reports whether any kernel of this library launched by this process on
  * the current device gave up a bounded wait since the last call (every wait on an mbarrier in the
- * kernels has an iteration limit so that a fault cannot hang a shared GPU).  Returns ATB_OK,
- * ATB_ERR_DEVICE_TIMEOUT (and clears the flag) or ATB_ERR_CUDA.  Debug / test helper: it
- * synchronises. */
+ * kernels gives up after 2 s of the GPU's global timer, so that a fault cannot hang a shared GPU; the
+ * CTA then sets an abort flag, all its roles leave their loops and it frees its tensor memory).
+ * The flag is kept per device and read for the CURRENT device only: call with the device that ran
+ * the kernels current.  Returns ATB_OK, ATB_ERR_DEVICE_TIMEOUT (and clears the flag) or ATB_ERR_CUDA.
+ * Debug / test helper: it synchronises. */
 atb_status_t atb_device_status(void* stream);
 
 /* Parameters of the analytical model of Sections 3-5.  One "unit" is what the paper calls a core

@@ -378,8 +378,7 @@ atb_status_t launch_gemm_pair(int T_MA, const GemmPlan& plan, int64_t M, int64_t
     switch (T_MA) {
         case 32:  return launch_pair_t<32>(plan, M, N, K, mant, exp, B, ldb, C, ldc, num_sms, error_flag, st);
         case 64:  return launch_pair_t<64>(plan, M, N, K, mant, exp, B, ldb, C, ldc, num_sms, error_flag, st);
-        case 128:
-        case 256: return launch_pair_t<128>(plan, M, N, K, mant, exp, B, ldb, C, ldc, num_sms, error_flag, st);
+        case 128: return launch_pair_t<128>(plan, M, N, K, mant, exp, B, ldb, C, ldc, num_sms, error_flag, st);
     }
     return atb::fail(ATB_ERR_BAD_TILING, "no pair kernel for T_MA=%d", T_MA);
 }

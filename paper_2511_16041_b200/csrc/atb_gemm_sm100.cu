@@ -488,7 +488,10 @@ static void fill_plan(const RingPlan& pl, GemmPlan* plan) {
 
 bool plan_gemm(int T_MA, int T_MC, int T_K, int T_N, GemmPlan* plan) {
     if (T_MA <= 0 || T_MC <= 0 || T_MA > T_MC) return false;
-    const RingPlan pl = is_pair_tiling(T_MC, T_K, T_N) ? plan_pair(T_MA > 128 ? 128 : T_MA) : plan_single(T_MA, T_MC, T_K, T_N);
+    // On the CTA pair each SM holds 128 rows of the tile: a slab cannot be taller than that, and
+    // T_MA = 128 is the pair's symmetric form.
+    if (is_pair_tiling(T_MC, T_K, T_N) && T_MA > 128) return false;
+    const RingPlan pl = is_pair_tiling(T_MC, T_K, T_N) ? plan_pair(T_MA) : plan_single(T_MA, T_MC, T_K, T_N);
     if (!pl.ok || !(T_MA == 32 || T_MA == 64 || T_MA == 128 || T_MA == 256)) return false;
     fill_plan(pl, plan);
     return true;
@@ -627,6 +630,10 @@ atb_status_t splitk_validate(int64_t M, int64_t N, int64_t K, int T_MA, int T_MC
         return atb::fail(ATB_ERR_BAD_TILING, "split-K supports T_K = 64, T_MC in {128, 256}, T_N in {128, 256}, T_MA in {64, 128}");
     if (splits < 1 || splits > 64 || splits > atb::ceil_div(K, T_K))
         return atb::fail(ATB_ERR_BAD_SHAPE, "splits=%d must be in [1, min(64, ceil(K / T_K))]", splits);
+    // the partial tiles are addressed by a 32-bit TMA row coordinate split * roundup(M, T_MC) + row
+    if (static_cast<int64_t>(splits) * atb::round_up(M, T_MC) > 0x7FFFFFFFll)
+        return atb::fail(ATB_ERR_BAD_SHAPE, "splits * roundup(M, T_MC) = %lld exceeds 2^31 - 1",
+                         (long long)(static_cast<int64_t>(splits) * atb::round_up(M, T_MC)));
     return ATB_OK;
 }
 

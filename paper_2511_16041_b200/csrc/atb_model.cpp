@@ -10,10 +10,12 @@ extern "C" {
 
 void atb_hw_params_b200(atb_hw_params_t* hw) {
     if (!hw) return;
-    // Constants fitted to measured throughput of atb_gemm on B200: every supported tiling on 16
+    // Constants fitted to measured throughput of atb_gemm on B200: every supported tiling on 15
     // shapes (cubes, shallow and deep K, FFN-like and odd sizes) and 6 tilings on 125 shapes.  The
     // fit maximises what the selection is for - the measured rate of the tiling it picks against the
-    // best measured one: mean 0.98 over the 16 shapes, 0.995 over the 125.
+    // best measured one (paper_2511_16041_b200/calibrate.py repeats the fit on the GPU at hand and
+    // prints that figure).  They are a fit, not the paper's model: the terms beyond Eq. 1, 2, 12-15 are
+    // named in atb_hw_params_t and each can be switched off.
     // One unit = one SM.  Dense BF16 tcgen05 peak: 8192 FLOP per cycle per SM; the clock is the one
     // a tensor-bound kernel settles at under the 1 kW power cap (1.65 PFLOP/s over 148 SMs).
     hw->peak_flops_per_cycle = 8192.0;
@@ -143,7 +145,7 @@ atb_status_t atb_select_tiling(int64_t M, int64_t N, int64_t K, const atb_hw_par
         atb_hw_params_t h = hw;
         if (pair) h.share_rows = hw.share_rows * 2;      // the B tile is shared by the two CTAs (Eq. 2)
         // thin slabs get the bundle discount only as far as this tiling's raw ring lets them be bundled
-        const int slab = pair && ma > 128 ? 128 : ma;
+        const int slab = ma;
         if (hw.mma_rows > 0 && slab < hw.mma_rows) {
             const int spg = hw.mma_rows / slab, b = atb::slab_bundle(spg, plan.n_raw_stages, plan.dq_groups);
             const double full = static_cast<double>(spg) / b;              // full switches per operand group
@@ -154,7 +156,7 @@ atb_status_t atb_select_tiling(int64_t M, int64_t N, int64_t K, const atb_hw_par
         if (pair) {
             // each CTA of the pair runs Eq. 13-15 on its own 128 rows
             atb_tiling_score_t half;
-            atb_score_tiling(&h, K, atb_tiling_t{ma > 128 ? 128 : ma, 128, k, n}, &half);
+            atb_score_tiling(&h, K, atb_tiling_t{ma, 128, k, n}, &half);
             s.eff_core = half.eff_core;
             s.compute_bound_flops = half.compute_bound_flops;
             // ... and holds its own half of the tile: Eq. 1's budgets are per CTA

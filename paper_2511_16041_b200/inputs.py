@@ -150,3 +150,18 @@ def make_config(name: str, seed: int = BASE_SEED, M: int | None = None):
     c = CONFIGS[name]
     m = c["M"] if M is None else M
     return make_A(c["A"], m, c["K"], seed), make_B_bits(c["K"], c["N"], c["b_scale"], seed)
+
+
+SWEEP_SIZES = (1024, 2048, 4096, 8192, 16384)
+
+
+def device_normal(shape, seed: int, tag: int, device, dtype=None):
+    """N(0,1) samples drawn ON THE DEVICE by torch's seeded generator, for the 125-shape sweep, whose
+    operands (up to 1 GB each) would take minutes to draw on the host.  Reproducible for a given torch
+    build; a consumer that needs the values on the host copies them back, so both sides of a comparison
+    always see the same numbers.  fp32, or rounded to ``dtype`` (bf16: torch rounds to nearest even)."""
+    import torch
+    g = torch.Generator(device=device)
+    g.manual_seed((seed * 1000003 + tag) & 0x7FFFFFFFFFFFFFFF)
+    x = torch.randn(shape, device=device, dtype=torch.float32, generator=g)
+    return x if dtype is None else x.to(dtype)

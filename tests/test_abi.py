@@ -48,6 +48,7 @@ def test_tiling_supported_rules():
     assert not ok(64, 128, 32, 128)           # T_K
     assert not ok(64, 128, 64, 96)            # T_N
     assert ok(128, 256, 64, 512) and ok(32, 256, 64, 512) and not ok(128, 256, 128, 512)   # CTA-pair tilings
+    assert not ok(256, 256, 64, 512)          # a CTA of the pair holds 128 rows: no taller slab exists
     # asymmetric buffering is what makes the deep K-step fit next to a 256-wide B tile
     assert not ok(256, 256, 128, 256) and not ok(128, 256, 128, 256) and not ok(64, 256, 128, 256)
     assert ok(32, 256, 128, 256)
@@ -113,3 +114,17 @@ def test_ring_plans_fit_the_budgets():
                     assert p.smem_bytes <= 232448 and p.tmem_columns <= 512
                     assert p.tmem_columns >= p.acc_buffers * (128 if pair else mc) // 128 * tn
     assert n >= 30
+
+
+def test_splitk_rejects_a_partial_tile_row_beyond_32_bits():
+    """The FP32 partial tiles are addressed by a 32-bit row coordinate split * roundup(M, T_MC) + row:
+    shapes whose product leaves that range are refused before anything is launched (host check only;
+    the pointers are never dereferenced)."""
+    lib = atb.load_library()
+    M = 1 << 30
+    big = lambda splits, fn, *tail: fn(M, 8, 128, 128, 256, 64, 128, 16, 16, 16, 8, 16, 8, splits, *tail)
+    assert big(2, lib.atb_gemm_splitk, 16, 0, None) == 2                       # 2 * 2^30 rows: BAD_SHAPE
+    assert "2^31" in atb.atb_last_error_message()
+    assert big(2, lib.atb_gemm_splitk_noalloc, None) == 2
+    assert big(1, lib.atb_gemm_splitk, 16, 0, None) == 7                       # in range: only the workspace is short
+    assert big(1, lib.atb_gemm_splitk_noalloc, None) == 7                      # ... or larger than the built-in array

@@ -79,7 +79,7 @@ def test_cta_pair_equals_the_single_cta_tiling_bitwise():
         Bb = inputs.make_B_bits(K, N, None)
         mant, exp = oracle.quantize_bfp16(A)
         ref = run_gemm(mant, exp, Bb, (128, 256, 64, 256))
-        for ma in (32, 64, 128, 256):
+        for ma in (32, 64, 128):
             assert np.array_equal(run_gemm(mant, exp, Bb, (ma, 256, 64, 512)), ref), (M, N, K, ma)
 
 
@@ -216,7 +216,7 @@ def test_tiny_and_degenerate_shapes():
         mant, exp = oracle.quantize_bfp16(A)
         _check(mant, exp, Bb, (128, 128, 64, 64))
         _check(mant, exp, Bb, (32, 256, 128, 128))
-        _check(mant, exp, Bb, (256, 256, 64, 512))       # CTA-pair kernel on a single partial tile
+        _check(mant, exp, Bb, (128, 256, 64, 512))       # CTA-pair kernel on a single partial tile
 
 
 def test_argument_errors():
@@ -264,7 +264,7 @@ def test_full_size_configs_sampled_rows(name, tilings):
     mant_d, plane_d = atb.atb_quantize_bfp16(Ad)        # the device quantiser feeds the device GEMM
     del Ad
     Bd = bf16_bits_to_dev(Bb)
-    n_rand = 48 if M * N * K > 2 ** 38 else 96
+    n_rand = 512 if name.startswith("cfg4") else 96
     rows = _sampled_rows(M, 256, n_rand, 17)
     mant_o, exp_o = oracle.quantize_bfp16(A[rows])
     del A

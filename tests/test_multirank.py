@@ -59,3 +59,17 @@ def test_single_rank_helpers():
     assert bench.max_over_ranks([3.0, 1.0], torch.device("cpu"), 1) == [3.0, 1.0]
     assert bench.rank_seed(7, 0) == 7 and bench.rank_seed(7, 3) == 10
     assert bench.aggregate_tflops(2.0 * 8192 ** 3, 1, 1.0) == 2.0 * 8192 ** 3 / 1e-3 / 1e12
+
+
+def test_gpus_flag_starts_its_own_ranks():
+    """`python bench.py --gpus 2` with no launcher around it starts two ranks itself; with the stub step
+    (gloo, no GPU work) the line rank 0 prints carries the world size and the slowest rank's time."""
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    p = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--stub-step"],
+                       env=env, capture_output=True, text=True, timeout=300)
+    assert p.returncode == 0, p.stderr[-2000:]
+    lines = [json.loads(l) for l in p.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1                                 # rank 0 alone prints
+    assert lines[0]["stub"] is True and lines[0]["n_gpus"] == 2
+    assert lines[0]["ms_per_step"] == 2.0                  # max over ranks of (1 + rank)
+    assert abs(lines[0]["value"] - 2 * 1e9 / 2e-3 / 1e12) < 1e-12
