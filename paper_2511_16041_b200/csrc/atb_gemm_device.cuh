@@ -44,7 +44,11 @@ constexpr uint32_t kEpilogueBoxBytes = 32 * 128;   // 32 rows x 64 bf16 columns
 constexpr uint32_t kSmallBoxBytes = 32 * 64;       // 32 rows x 32 bf16 columns (the CTA-pair kernel)
 constexpr uint32_t kScaleTableBytes = 256u * 8u;  // per exponent: the scale and its offset, see scale_table_entry
 constexpr uint32_t kSmemBudget = 232448;          // 227 KB of dynamic shared memory per CTA
+#ifdef ATB_TEST_WAIT_NS                             // test build of the timeout path only: a short limit
+constexpr uint64_t kWaitTimeoutNs = ATB_TEST_WAIT_NS;
+#else
 constexpr uint64_t kWaitTimeoutNs = 2000000000ull;  // every mbarrier wait gives up after 2 s
+#endif
 
 // lcm(n, d) for d a power of two: the number of barrier pairs of a ring of n buffers and d groups
 __host__ __device__ constexpr int ring_bars(int n, int d) {
