@@ -560,6 +560,9 @@ template <int N_COLS, int BOX_COLS = 64>
 __device__ __forceinline__ void epilogue_bf16(const CUtensorMap* tm_c, uint32_t t_addr, uint32_t box, int lane, int row0,
                                               int col0, int64_t M, int64_t N) {
     static_assert(BOX_COLS == 64 || BOX_COLS == 32, "box width");
+#ifndef ATB_NO_L2_HINTS
+    const uint64_t store_policy = l2_policy_evict_first();
+#endif
     const uint32_t my_row = box + lane * (BOX_COLS * 2);
     const uint32_t sw = BOX_COLS == 64 ? static_cast<uint32_t>(lane & 7) : (static_cast<uint32_t>(lane >> 1) & 3u);
 #pragma unroll 1
@@ -588,7 +591,11 @@ __device__ __forceinline__ void epilogue_bf16(const CUtensorMap* tm_c, uint32_t 
         fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0 && row0 < M && col0 + c * BOX_COLS < N) {   // rows / columns past the edge are clipped
+#ifndef ATB_NO_L2_HINTS
+            tma_store_2d_hint(tm_c, box, col0 + c * BOX_COLS, row0, store_policy);   // C is not read again: first to leave the L2
+#else
             tma_store_2d(tm_c, box, col0 + c * BOX_COLS, row0);
+#endif
             tma_store_commit();
         }
     }

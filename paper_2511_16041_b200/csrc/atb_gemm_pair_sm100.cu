@@ -160,6 +160,9 @@ atb_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_c
         if (elect_one()) {
             Cursor<C::NR, C::LR> rr;
             bool ok = true;
+#ifndef ATB_NO_L2_HINTS
+            const uint64_t a_policy = l2_policy_evict_last();   // a band's A panels serve wave after wave
+#endif
             for (int tile = cluster_id; ok && tile < total_tiles; tile += n_clusters) {
                 int mt, nt;
                 tile_coords(tile, p.m_tiles, p.n_tiles, mt, nt);
@@ -170,8 +173,13 @@ atb_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_c
                         const uint32_t fr = raw_full + 8 * rr.bar;
                         const uint32_t dst = raw_base + rr.buf() * C::RAW_BYTES;
                         mbar_arrive_expect_tx(fr, C::RAW_BYTES);
+#ifndef ATB_NO_L2_HINTS
+                        tma_load_2d_hint(dst, &tm_mant, k * C::T_K, row0 + s * SLAB_ROWS, fr, a_policy);
+                        tma_load_2d_hint(dst + C::RAW_MANT_BYTES, &tm_exp, row0 + s * SLAB_ROWS, k, fr, a_policy);
+#else
                         tma_load_2d(dst, &tm_mant, k * C::T_K, row0 + s * SLAB_ROWS, fr);
                         tma_load_2d(dst + C::RAW_MANT_BYTES, &tm_exp, row0 + s * SLAB_ROWS, k, fr);
+#endif
                         rr.template advance<1>();
                     }
                 }
@@ -289,8 +297,16 @@ atb_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_c
                 // CTA-scope release: the operand this publishes stays in this CTA's shared memory and is
                 // read by this CTA's tensor core (after the proxy fence above) once the leader has seen
                 // the arrival and issued the UMMA.  A cluster-scope release here kept a quarter of the
-                // dequantiser warps in membar stalls (ncu) and cost 1-2 %.
+                // dequantiser warps in membar stalls (ncu) and cost 1-2 %.  The waiter acquires at cluster
+                // scope, so by the letter of the PTX memory model this release/acquire pair does not
+                // synchronise; it is kept because no thread of the other CTA reads what is published (a
+                // bit-for-bit soak of all slab heights against the single-CTA kernel stands in the test
+                // suite).  -DATB_PAIR_RELEASE_CLUSTER builds the conforming form.
+#ifdef ATB_PAIR_RELEASE_CLUSTER
+                mbar_arrive_cluster(mapa_shared(deq_full + 8 * rd.bar, 0));
+#else
                 mbar_arrive_cluster_cta_release(mapa_shared(deq_full + 8 * rd.bar, 0));
+#endif
 #pragma unroll
                 for (int i = 0; i < C::BUNDLE; ++i) mbar_arrive(raw_empty + 8 * (rr.bar + i));
             }

@@ -164,6 +164,11 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
         if (elect_one()) {
             Cursor<C::NR, C::LR> rr;
             bool ok = true;
+#ifndef ATB_NO_L2_HINTS
+            // The tile walk keeps a band of A row panels in use wave after wave while the B column panels
+            // change: A is asked to stay in the L2 longest.
+            const uint64_t a_policy = l2_policy_evict_last();
+#endif
             for (int item = blockIdx.x; ok && item < total_items; item += gridDim.x) {
                 const WorkItem w = work_item<SPLIT>(item, p);
                 for (int k = w.k_begin; ok && k < w.k_end; ++k) {
@@ -172,8 +177,13 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
                         const uint32_t fr = raw_full + 8 * rr.bar;
                         const uint32_t dst = raw_base + rr.buf() * C::RAW_BYTES;
                         mbar_arrive_expect_tx(fr, C::RAW_BYTES);
+#ifndef ATB_NO_L2_HINTS
+                        tma_load_2d_hint(dst, &tm_mant, k * T_K, w.mt * T_MC + s * T_MA, fr, a_policy);
+                        tma_load_2d_hint(dst + C::RAW_MANT_BYTES, &tm_exp, w.mt * T_MC + s * T_MA, k * (T_K / 64), fr, a_policy);
+#else
                         tma_load_2d(dst, &tm_mant, k * T_K, w.mt * T_MC + s * T_MA, fr);
                         tma_load_2d(dst + C::RAW_MANT_BYTES, &tm_exp, w.mt * T_MC + s * T_MA, k * (T_K / 64), fr);
+#endif
                         rr.template advance<1>();
                     }
                 }

@@ -116,3 +116,39 @@ def test_quantise_and_gemm_capture_into_a_cuda_graph():
             assert torch.equal(eager, replayed), tiling
             A.mul_(1.5)                      # new values in the same buffers for the second round
     atb.atb_device_status()
+
+
+def test_soak_cta_pair_against_single_cta_bitwise():
+    """A bounded soak of the CTA-pair kernel: its dequantisers announce an operand to the leader CTA with
+    a CTA-scope release (the operand is read by the announcing CTA's own tensor core only), which the
+    memory model does not promise to order against the leader's cluster-scope acquire.  Random shapes
+    (ragged edges, one to hundreds of K-steps), the three slab heights of the pair and the single-CTA
+    256 x 256 tiling, which adds the same products in the same order: all four results must be
+    bit-identical, launch after launch."""
+    import random
+    import time
+    g = torch.Generator(device=dev())
+    g.manual_seed(11)
+    rnd = random.Random(5)
+    tilings = [(128, 256, 64, 256), (128, 256, 64, 512), (64, 256, 64, 512), (32, 256, 64, 512)]
+    launches, t_end = 0, time.time() + 12.0
+    while time.time() < t_end or launches < 400:
+        M = rnd.choice([300, 1000, 2048, 4096, 5000])
+        N = rnd.choice([512, 1024, 2048, 4104])
+        K = rnd.choice([16, 64, 448, 1024, 1104, 4096])
+        mant = torch.randint(-127, 128, (M, K), dtype=torch.int8, device=dev(), generator=g)
+        plane = torch.randint(100, 150, (atb.atb_bfp16_exp_bytes(M, K),), dtype=torch.uint8, device=dev(), generator=g)
+        B = torch.randn((K, N), device=dev(), generator=g).to(torch.bfloat16)
+        ref = None
+        for rep in range(6):
+            for t in tilings:
+                C = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device=dev())
+                atb.atb_gemm(M, N, K, *t, mant, plane, B, C)
+                launches += 1
+                if ref is None:
+                    ref = C.view(torch.int16).clone()
+                else:
+                    assert torch.equal(C.view(torch.int16), ref), ((M, N, K), t, rep)
+        atb.atb_device_status()
+        assert bool(torch.isfinite(ref.view(torch.bfloat16).float()).all())
+    assert launches >= 400
