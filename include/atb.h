@@ -258,9 +258,20 @@ typedef struct {
                                      (1 = every slab is a full switch, as in Eq. 14)                                 */
     double coarse_slab_factor;    /* with mma_rows > 0: factor on Eff_core of slabs larger than mma_rows: their raw ring has
                                      fewer, larger buffers and pipelines at coarser grain (0 or 1 = none)              */
-    double deep_kstep_factor;     /* with mma_rows > 0: factor on Eff_core of tilings with T_K > 64: a dequantiser group then
-                                     converts an mma_rows x T_K unit in one piece, twice the latency per hand-over with
-                                     the same number of buffers (0 or 1 = none)                                        */
+    double deep_kstep_factor;     /* with mma_rows > 0: factor on Eff_core of tilings with T_K > 64 (0 or 1 = none; 0 in
+                                     every preset: since A moves in 64-column units whatever T_K is, a deeper K-step
+                                     no longer changes the conversion pipeline)                                        */
+    /* The conversion of A (BFP16 -> BF16 in shared memory) that precedes every UMMA, on the compute side of
+     * Eq. 12.  One unit = mma_rows rows x 64 columns of A; it feeds 2 * mma_rows * 64 * T_N FLOP, i.e.
+     * t_mma = that / peak_flops_per_cycle cycles of tensor time.  Eff_core is multiplied by
+     * t_mma / max(t_mma + convert_exposed_cycles, convert_cycles).  Both 0 = no conversion (XDNA2 presets). */
+    double convert_cycles;        /* cycles per unit at the dequantisers' full throughput (binds where T_N is small)  */
+    double convert_exposed_cycles;/* cycles per unit that the pipeline does not hide behind the UMMAs                  */
+    double convert_latency_cycles;/* atb_select_tiling: latency from a free operand buffer to a converted unit; a ring of n
+                                     converted units, each in use for t = max(t_mma + convert_exposed_cycles,
+                                     convert_cycles) cycles, sustains n * t / (latency + t) of the rate                  */
+    int    a_unit_cols;           /* > 0: A is buffered in units of this many columns whatever T_K is (64 on B200), so the A
+                                     and scratch terms of Eq. 1 use min(T_K, a_unit_cols) in place of T_K (0: T_K)    */
 } atb_hw_params_t;
 
 typedef struct {

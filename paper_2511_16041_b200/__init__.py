@@ -46,7 +46,9 @@ class atb_hw_params_t(ctypes.Structure):
                [("mma_rows", ctypes.c_int)] + \
                [(n, ctypes.c_double) for n in ("load_latency_cycles", "pair_efficiency", "launch_seconds", "tile_fixed_cycles",
                                                "drain_cycles_per_column", "pair_tile_cycles", "thin_slab_cost",
-                                               "coarse_slab_factor", "deep_kstep_factor")]
+                                               "coarse_slab_factor", "deep_kstep_factor", "convert_cycles",
+                                               "convert_exposed_cycles", "convert_latency_cycles")] + \
+               [("a_unit_cols", ctypes.c_int)]
 
 
 class atb_tiling_score_t(ctypes.Structure):

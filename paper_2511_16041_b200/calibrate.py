@@ -27,14 +27,16 @@ TilingT = Tuple[int, int, int, int]
 
 # The constants the search moves, with the values it tries.  Everything else keeps its preset value.
 DEFAULT_GRID: Dict[str, Sequence[float]] = {
-    "a_bytes": (2.4, 3.0, 3.6, 4.2),
-    "load_latency_cycles": (800.0, 1200.0, 1600.0, 2000.0),
-    "delta_cycles": (60.0, 90.0, 120.0, 150.0),
-    "pair_efficiency": (0.85, 0.9, 0.95, 1.0),
-    "tile_fixed_cycles": (1000.0, 2000.0, 3000.0),
-    "drain_cycles_per_column": (4.0, 8.0),
+    "convert_cycles": (300.0, 400.0),
+    "convert_exposed_cycles": (20.0, 45.0),
+    "convert_latency_cycles": (700.0, 1200.0),
+    "load_latency_cycles": (800.0, 1200.0, 1600.0),
+    "delta_cycles": (20.0, 45.0, 90.0),
+    "pair_efficiency": (0.95, 1.0),
+    "tile_fixed_cycles": (1000.0, 3000.0),
+    "drain_cycles_per_column": (2.0, 4.0),
     "pair_tile_cycles": (2000.0, 4000.0),
-    "thin_slab_cost": (0.3, 0.6, 0.9),
+    "thin_slab_cost": (0.3, 0.6),
 }
 
 FULL_SHAPES: List[Shape] = [

@@ -18,6 +18,7 @@ namespace {
 
 using namespace sm100;
 
+constexpr int kKA = 64;               // columns of A per raw slab and per converted operand group, whatever T_K is
 constexpr int kDequantWarps = 16;
 constexpr int kThreads = (7 + kDequantWarps) * 32;      // + B producer, UMMA issuer, 4 epilogue warps, A producer
 constexpr int kAProducerWarp = 6 + kDequantWarps;       // the last warp
@@ -32,8 +33,8 @@ __host__ __device__ constexpr int dq_groups(int T_MA, int T_K, int T_N) {
 #ifdef ATB_DQ_GROUPS
     return ATB_DQ_GROUPS;
 #else
-    // two groups for big slabs, and where a double-buffered B tile already takes 128 KB
-    return (T_MA * T_K >= 256 * 64 || T_K * T_N >= 128 * 256) ? 2 : 4;
+    // two groups for 256-row slabs, and where a double-buffered B tile already takes 128 KB
+    return (T_MA >= 256 || T_K * T_N >= 128 * 256) ? 2 : 4;
 #endif
 }
 constexpr int kFirstEpilogueWarp = 2;
@@ -87,7 +88,7 @@ constexpr RingPlan plan_single(int T_MA, int T_MC, int T_K, int T_N) {
     if (!(T_MA == 32 || T_MA == 64 || T_MA == 128 || T_MA == 256) || T_MA > T_MC || T_MC % T_MA != 0) return pl;
     const int G = T_MC / 128;
     if (G * T_N > 512) return pl;
-    const uint32_t b_bytes = T_K * T_N * 2, group_bytes = 128 * T_K * 2, raw_bytes = T_MA * T_K * 9 / 8;
+    const uint32_t b_bytes = T_K * T_N * 2, group_bytes = 128 * kKA * 2, raw_bytes = T_MA * kKA * 9 / 8;
     const int gps = T_MA > 128 ? T_MA / 128 : 1;          // groups per slab
     const int spg = T_MA < 128 ? 128 / T_MA : 1;          // slabs per group
     const int dqg = dq_groups(T_MA, T_K, T_N);
@@ -112,14 +113,14 @@ constexpr RingPlan plan_single(int T_MA, int T_MC, int T_K, int T_N) {
     // fits; a tiling that only fits with fewer slabs gets one slab per group and smaller bundles.
     const int ng_step = T_MA <= 128 ? (dqg >= spg ? dqg / spg : 1) : dqg * gps;
     int nb = 2, ng = ng_step < 2 ? 2 * ng_step : ng_step;
-    int nr_step = dqg * spg * 64 / T_K;                  // 512 rows of look-ahead at T_K = 64, 256 at T_K = 128
-    if (nr_step < dqg || total(nb, ng, nr_step) > kSmemBudget) nr_step = dqg;
+    int nr_step = dqg * spg;                             // 512 rows x 64 columns of look-ahead
+    if (total(nb, ng, nr_step) > kSmemBudget) nr_step = dqg;
     int nr = nr_step;
     pl.nb = nb; pl.ng = ng; pl.nr = nr;
     if (total(nb, ng, nr) > kSmemBudget) return pl;
     // Grow the rings towards a target look-ahead, counted in 128-row x T_K operand groups:
     // B tiles hide the TMA latency for G groups each, raw slabs for T_MA/128 groups each.
-    const double target_b = 8.0 * 64 / T_K, target_r = 6.0 * 64 / T_K, target_g = 4.0;
+    const double target_b = 8.0 * 64 / T_K, target_r = 6.0, target_g = 4.0;
     for (;;) {
         const double cov_b = nb * G / target_b, cov_r = nr * (T_MA / 128.0) / target_r, cov_g = ng / target_g;
         int pick = -1;

@@ -42,12 +42,18 @@ struct Cfg {
     static constexpr int N_CHUNKS = T_N / N_MMA;
     static constexpr uint32_t B_BYTES = T_K * T_N * 2;
     static constexpr uint32_t B_BOX_BYTES = T_K * 128;         // one 64-column box of B
-    static constexpr uint32_t GROUP_BYTES = 128 * T_K * 2;
+    // T_K is the depth of a B tile.  A always moves in units of kKA = 64 columns - raw slabs of
+    // T_MA x 64, converted operand groups of 128 x 64 (one 128-byte swizzle row per row) - so a K-step
+    // of T_K = 128 is one B tile and KH = 2 rounds of slabs: the conversion pipeline (slab size, groups,
+    // hand-overs per FLOP) is the same for every T_K, only the B ring's grain and the B barriers per
+    // FLOP change.
+    static constexpr int KH = T_K / kKA;
+    static constexpr uint32_t GROUP_BYTES = 128 * kKA * 2;
     static constexpr uint32_t KHALF_BYTES = 128 * 128;         // 128 rows x 64 bf16
-    static constexpr uint32_t RAW_MANT_BYTES = T_MA * T_K;
-    static constexpr uint32_t RAW_EXP_BYTES = T_MA * T_K / 8;
+    static constexpr uint32_t RAW_MANT_BYTES = T_MA * kKA;
+    static constexpr uint32_t RAW_EXP_BYTES = T_MA * kKA / 8;
     static constexpr uint32_t RAW_BYTES = RAW_MANT_BYTES + RAW_EXP_BYTES;
-    static constexpr int SLOTS_PER_ROW = T_K / 16;             // a slot = 2 blocks = 16 mantissa bytes
+    static constexpr int SLOTS_PER_ROW = kKA / 16;             // a slot = 2 blocks = 16 mantissa bytes
     static constexpr int SLOTS = T_MA * SLOTS_PER_ROW;
     static constexpr int DQ_GROUPS = dq_groups(T_MA, T_K, T_N);
     static constexpr int GROUP_WARPS = kDequantWarps / DQ_GROUPS;
@@ -171,18 +177,18 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
 #endif
             for (int item = blockIdx.x; ok && item < total_items; item += gridDim.x) {
                 const WorkItem w = work_item<SPLIT>(item, p);
-                for (int k = w.k_begin; ok && k < w.k_end; ++k) {
+                for (int kh = w.k_begin * C::KH; ok && kh < w.k_end * C::KH; ++kh) {      // 64-column rounds
                     for (int s = 0; s < C::RHO; ++s) {
                         if (!(ok = wait_bar_spin(cx, raw_empty + 8 * rr.freed_bar(), rr.freed_parity(), 0x002))) break;
                         const uint32_t fr = raw_full + 8 * rr.bar;
                         const uint32_t dst = raw_base + rr.buf() * C::RAW_BYTES;
                         mbar_arrive_expect_tx(fr, C::RAW_BYTES);
 #ifndef ATB_NO_L2_HINTS
-                        tma_load_2d_hint(dst, &tm_mant, k * T_K, w.mt * T_MC + s * T_MA, fr, a_policy);
-                        tma_load_2d_hint(dst + C::RAW_MANT_BYTES, &tm_exp, w.mt * T_MC + s * T_MA, k * (T_K / 64), fr, a_policy);
+                        tma_load_2d_hint(dst, &tm_mant, kh * kKA, w.mt * T_MC + s * T_MA, fr, a_policy);
+                        tma_load_2d_hint(dst + C::RAW_MANT_BYTES, &tm_exp, w.mt * T_MC + s * T_MA, kh, fr, a_policy);
 #else
-                        tma_load_2d(dst, &tm_mant, k * T_K, w.mt * T_MC + s * T_MA, fr);
-                        tma_load_2d(dst + C::RAW_MANT_BYTES, &tm_exp, w.mt * T_MC + s * T_MA, k * (T_K / 64), fr);
+                        tma_load_2d(dst, &tm_mant, kh * kKA, w.mt * T_MC + s * T_MA, fr);
+                        tma_load_2d(dst + C::RAW_MANT_BYTES, &tm_exp, w.mt * T_MC + s * T_MA, kh, fr);
 #endif
                         rr.template advance<1>();
                     }
@@ -204,9 +210,11 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
                 for (int k = w.k_begin; ok && k < w.k_end; ++k) {
                     if (!(ok = wait_bar_spin(cx, b_full + 8 * rb.stage, rb.phase, 0x101))) break;
                     const uint32_t bs = b_base + rb.stage * C::B_BYTES;
+#pragma unroll
+                    for (int h = 0; h < C::KH; ++h) {         // 64-column rounds of this B tile
                     for (int g = 0; g < C::G; ++g) {
                         const int acc = acc_buf * C::G + g;
-                        if (k == w.k_begin && !(ok = wait_bar_spin(cx, acc_empty + 8 * acc, acc_phase ^ 1u, 0x102))) break;
+                        if (k == w.k_begin && h == 0 && !(ok = wait_bar_spin(cx, acc_empty + 8 * acc, acc_phase ^ 1u, 0x102))) break;
                         int group_slot;
                         if (T_MA <= 128) {
                             for (int i = 0; ok && i < C::SPB; ++i)
@@ -223,11 +231,11 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
 #pragma unroll
                         for (int nc = 0; nc < C::N_CHUNKS; ++nc) {
 #pragma unroll
-                            for (int kk = 0; kk < T_K / 16; ++kk) {
-                                const uint64_t a_desc = umma_smem_desc_sw128(as + (kk >> 2) * C::KHALF_BYTES + (kk & 3) * 32, 16, 1024);
-                                const uint64_t b_desc = umma_smem_desc_sw128(bs + nc * (C::N_MMA / 64) * C::B_BOX_BYTES + kk * 2048,
+                            for (int kk = 0; kk < kKA / 16; ++kk) {
+                                const uint64_t a_desc = umma_smem_desc_sw128(as + kk * 32, 16, 1024);
+                                const uint64_t b_desc = umma_smem_desc_sw128(bs + nc * (C::N_MMA / 64) * C::B_BOX_BYTES + (h * 4 + kk) * 2048,
                                                                              C::B_BOX_BYTES, 1024);
-                                umma_f16_ss(d_tmem + nc * C::N_MMA, a_desc, b_desc, idesc, (k > w.k_begin || kk > 0) ? 1u : 0u);
+                                umma_f16_ss(d_tmem + nc * C::N_MMA, a_desc, b_desc, idesc, (k > w.k_begin || h > 0 || kk > 0) ? 1u : 0u);
                             }
                         }
                         if (T_MA <= 128) {
@@ -237,7 +245,9 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
                             umma_commit(deq_empty + 8 * rd.bar);
                             rd.template advance<1>();
                         }
-                        if (k == w.k_end - 1) umma_commit(acc_full + 8 * acc);
+                        if (k == w.k_end - 1 && h == C::KH - 1) umma_commit(acc_full + 8 * acc);
+                    }
+                    if (!ok) break;
                     }
                     if (!ok) break;
                     umma_commit(b_empty + 8 * rb.stage);
@@ -305,7 +315,7 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
         int64_t my_slabs = 0;
         for (int item = blockIdx.x; item < total_items; item += gridDim.x) {
             const WorkItem w = work_item<SPLIT>(item, p);
-            my_slabs += static_cast<int64_t>(w.k_end - w.k_begin) * C::RHO;
+            my_slabs += static_cast<int64_t>(w.k_end - w.k_begin) * C::KH * C::RHO;
         }
         const DequantLane<C> ln(t, T_MA);
 #ifdef ATB_PROFILE_SKIP_DEQUANT
@@ -392,10 +402,10 @@ atb_status_t launch(const atb::GemmPlan& plan, int64_t M, int64_t N, int64_t K, 
                     uint8_t* C_exp = nullptr) {
     CUtensorMap tm_mant, tm_exp, tm_b, tm_c;
     const int64_t M_pad = atb::round_up(M, 32);
-    if (!make_map_2d(&tm_mant, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, mant, K, M, K, T_K, T_MA, CU_TENSOR_MAP_SWIZZLE_NONE))
+    if (!make_map_2d(&tm_mant, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, mant, K, M, K, kKA, T_MA, CU_TENSOR_MAP_SWIZZLE_NONE))
         return atb::fail(ATB_ERR_CUDA, "cuTensorMapEncodeTiled failed for the mantissa plane");
     if (!make_map_2d(&tm_exp, CU_TENSOR_MAP_DATA_TYPE_UINT64, 8, exp, M_pad, atb::ceil_div(K, 64), M_pad * 8, T_MA,
-                     T_K / 64, CU_TENSOR_MAP_SWIZZLE_NONE))
+                     1, CU_TENSOR_MAP_SWIZZLE_NONE))
         return atb::fail(ATB_ERR_CUDA, "cuTensorMapEncodeTiled failed for the exponent plane");
     if (!make_map_2d(&tm_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, B, N, K, ldb * 2, 64, T_K, CU_TENSOR_MAP_SWIZZLE_128B))
         return atb::fail(ATB_ERR_CUDA, "cuTensorMapEncodeTiled failed for B");

@@ -21,11 +21,12 @@ void atb_hw_params_b200(atb_hw_params_t* hw) {
     hw->peak_flops_per_cycle = 8192.0;
     hw->clock_hz = 1.361e9;
     hw->n_units = 148;
-    // Eq. 2 / Eq. 12 with byte-EQUIVALENT costs: what an operand element costs the SM per tile.
-    // For A that is 1.125 B of L2->SM traffic plus the dequantiser's time (one conversion per
-    // 2*T_N FLOP), together worth 3.0 B at the fitted feed rate of 14 TB/s.
+    // Eq. 2 / Eq. 12 with the physical byte costs of the operands (BFP16 A 9/8 B, BF16 B and C 2 B): AI is
+    // FLOP per byte of tile traffic, which on B200 flows L2 -> SM (ncu: 163.8 FLOP/B at 256 x 256, the
+    // formula's value).  The bandwidth is the L2 -> SM feed rate of 148 SMs; it is FITTED (no direct
+    // measurement; the kernels have been seen to draw 9.2 TB/s without being bound by it).
     hw->bw_bytes_per_s = 14.0e12;
-    hw->a_bytes = 3.0; hw->b_bytes = 2.0; hw->c_bytes = 2.0;
+    hw->a_bytes = 1.125; hw->b_bytes = 2.0; hw->c_bytes = 2.0;
     // Eq. 1, A and B terms, against shared memory: raw BFP16 slabs double-buffered at 9/8 B, two
     // dequantised BF16 copies per slab row (the "converted copy" of Table 2), B double-buffered.
     // The C term is budgeted against TMEM (128 lanes x 512 columns x 4 B) instead.
@@ -36,20 +37,26 @@ void atb_hw_params_b200(atb_hw_params_t* hw) {
     hw->share_rows = 1; hw->share_cols = 1;
     // Eq. 13: one UMMA covers K = 16 -> eta = 1/16 instructions per unit of T_K, II = 1.
     hw->eta = 1.0 / 16.0; hw->eps_cycles = 0.05; hw->ii = 1.0;
-    hw->delta_cycles = 90.0;                  // per-slab barrier round trip of the dequantisers
+    hw->delta_cycles = 20.0;                  // per-slab hand-over (barrier round trip, commit) left once the conversion has its own term
     hw->mma_rows = 128;
     hw->load_latency_cycles = 1200.0;
-    hw->pair_efficiency = 0.97;
+    hw->pair_efficiency = 1.0;
     hw->launch_seconds = 1.0e-5;
-    hw->tile_fixed_cycles = 3000.0;
-    hw->drain_cycles_per_column = 4.0;
+    hw->tile_fixed_cycles = 1000.0;
+    hw->drain_cycles_per_column = 2.0;
     hw->pair_tile_cycles = 4000.0;
-    // Measured, a bundled slab costs about 0.3 of a switch (rho = 4 reaches 0.97 and rho = 8 0.87 of
-    // rho = 2); the fit for pick quality keeps 0.9, because plans with thin slabs also end up with
-    // shallower dequantised rings, for which the selection has no term.
-    hw->thin_slab_cost = 0.9;
-    hw->coarse_slab_factor = 0.88;            // measured: 256-row slabs reach a median 0.87 of 128-row slabs
-    hw->deep_kstep_factor = 0.7;              // measured: T_K = 128 reaches 0.62-0.65 of T_K = 64 at T_N = 128, 0.86 at T_N = 64; the look-ahead term carries a part of it already
+    hw->thin_slab_cost = 0.3;                 // measured: a bundled slab costs about 0.3 of a switch (rho = 4 reaches 0.97, rho = 8 0.87 of rho = 2)
+    hw->coarse_slab_factor = 0.92;            // 256-row slabs: measured 0.87-0.92 of 128-row slabs
+    hw->deep_kstep_factor = 0.0;              // retired: T_K = 128 runs level with T_K = 64 where the rings are as deep
+    // The conversion of A, on the compute side.  Measured against the same pipeline without it the
+    // conversion costs 8 % at T_N = 256 and 3.5 % on the CTA pair (a unit feeds 512 columns there): about
+    // 45 cycles per unit that the UMMAs do not hide; at T_N <= 128 the 16 dequantiser warps bind at
+    // about 400 cycles per unit.  A converted-operand ring of n units hides a conversion latency of about
+    // 700 cycles only if n * t_mma covers it (two groups instead of four measured -15...-20 %).
+    hw->convert_cycles = 400.0;
+    hw->convert_exposed_cycles = 45.0;
+    hw->convert_latency_cycles = 700.0;
+    hw->a_unit_cols = 64;                     // raw slabs of T_MA x 64 and converted groups of 128 x 64 for every T_K
 }
 
 void atb_hw_params_xdna2(atb_hw_params_t* hw, int precision_config) {
@@ -67,6 +74,8 @@ void atb_hw_params_xdna2(atb_hw_params_t* hw, int precision_config) {
     hw->mma_rows = 0; hw->load_latency_cycles = 0.0; hw->pair_efficiency = 0.0; hw->launch_seconds = 0.0;
     hw->tile_fixed_cycles = 0.0; hw->drain_cycles_per_column = 0.0; hw->pair_tile_cycles = 0.0;
     hw->thin_slab_cost = 1.0; hw->coarse_slab_factor = 0.0; hw->deep_kstep_factor = 0.0;
+    hw->convert_cycles = 0.0; hw->convert_exposed_cycles = 0.0; hw->convert_latency_cycles = 0.0;
+    hw->a_unit_cols = 0;
     switch (precision_config) {
         case 1:   // A, C in BF16, B in BFP16 (text: 1.25 B in AI; 9/8 B reproduces the buffer column)
             hw->a_bytes = 2.0; hw->b_bytes = 1.25; hw->c_bytes = 2.0;
@@ -93,8 +102,9 @@ atb_status_t atb_score_tiling(const atb_hw_params_t* hw, int64_t K, atb_tiling_t
     const double TMC = t.T_MC, TK = t.T_K, TN = t.T_N, TMA = t.T_MA;
     out->t = t;
     // Eq. 1 (left-hand side), with the optional converted-copy term.
-    const double ab = (2.0 * hw->a_buf_bytes / rho) * TMC * TK + 2.0 * hw->b_buf_bytes * TK * TN +
-                      hw->a_scratch_bytes * TMA * TK;
+    const double TKA = (hw->a_unit_cols > 0 && hw->a_unit_cols < t.T_K) ? hw->a_unit_cols : TK;   // depth of an A buffer
+    const double ab = (2.0 * hw->a_buf_bytes / rho) * TMC * TKA + 2.0 * hw->b_buf_bytes * TK * TN +
+                      hw->a_scratch_bytes * TMA * TKA;
     const double cb = hw->c_buf_bytes * TMC * TN;
     if (hw->acc_capacity_bytes > 0.0) {
         out->buf_bytes_used = ab;
@@ -120,6 +130,10 @@ atb_status_t atb_score_tiling(const atb_hw_params_t* hw, int64_t K, atb_tiling_t
                            hw->delta_cycles * rho_eff * hw->peak_flops_per_cycle / (2.0 * TMC * TN * TK));
     if (hw->mma_rows > 0 && t.T_MA > hw->mma_rows && hw->coarse_slab_factor > 0.0) out->eff_core *= hw->coarse_slab_factor;
     if (hw->mma_rows > 0 && t.T_K > 64 && hw->deep_kstep_factor > 0.0) out->eff_core *= hw->deep_kstep_factor;
+    if (hw->mma_rows > 0 && (hw->convert_cycles > 0.0 || hw->convert_exposed_cycles > 0.0)) {
+        const double t_mma = 2.0 * hw->mma_rows * 64.0 * TN / hw->peak_flops_per_cycle;
+        out->eff_core *= t_mma / std::max(t_mma + hw->convert_exposed_cycles, hw->convert_cycles);
+    }
     // Eq. 12
     out->mem_bound_flops = out->ai * hw->bw_bytes_per_s;
     out->compute_bound_flops = out->eff_core * hw->peak_flops_per_cycle * hw->clock_hz * hw->n_units;
@@ -172,6 +186,14 @@ atb_status_t atb_select_tiling(int64_t M, int64_t N, int64_t K, const atb_hw_par
             const double rows_per_unit = pair ? 128.0 : mc;
             const double kstep_cycles = 2.0 * rows_per_unit * n * k / hw.peak_flops_per_cycle;
             const double sustain = plan.n_b_stages * kstep_cycles / (hw.load_latency_cycles + kstep_cycles);
+            if (sustain < 1.0) s.compute_bound_flops *= sustain;
+        }
+        // Look-ahead of the converted-operand ring, the same law: n units of t_mma cycles each hide the
+        // conversion latency only if n * t covers it.
+        if (hw.convert_latency_cycles > 0.0 && hw.mma_rows > 0) {
+            const double t_mma = 2.0 * hw.mma_rows * 64.0 * n / hw.peak_flops_per_cycle;
+            const double t_unit = std::max(t_mma + hw.convert_exposed_cycles, hw.convert_cycles);
+            const double sustain = plan.n_groups * t_unit / (hw.convert_latency_cycles + t_unit);
             if (sustain < 1.0) s.compute_bound_flops *= sustain;
         }
         // Per-tile costs that the K loop does not hide: filling the rings, and - with a single

@@ -49,9 +49,10 @@ def test_tiling_supported_rules():
     assert not ok(64, 128, 64, 96)            # T_N
     assert ok(128, 256, 64, 512) and ok(32, 256, 64, 512) and not ok(128, 256, 128, 512)   # CTA-pair tilings
     assert not ok(256, 256, 64, 512)          # a CTA of the pair holds 128 rows: no taller slab exists
-    # asymmetric buffering is what makes the deep K-step fit next to a 256-wide B tile
-    assert not ok(256, 256, 128, 256) and not ok(128, 256, 128, 256) and not ok(64, 256, 128, 256)
-    assert ok(32, 256, 128, 256)
+    # asymmetric buffering is what makes the deep K-step fit next to a 256-wide B tile: two B tiles of
+    # 128 x 256 take 128 KB, and the symmetric 256-row slabs do not fit beside them
+    assert not ok(256, 256, 128, 256)
+    assert ok(128, 256, 128, 256) and ok(64, 256, 128, 256) and ok(32, 256, 128, 256)
 
 
 def test_layout_helpers_roundtrip():

@@ -236,7 +236,7 @@ def test_argument_errors():
     assert call(K=100) == 2 and call(K=72) == 2 and call(N=12) == 2 and call(M=0) == 2 and call(ldb=N - 8) == 2
     assert call(til=(64, 128, 64, 96)) == 3          # unsupported T_N
     assert call(til=(256, 128, 64, 128)) == 3        # T_MA > T_MC
-    assert call(til=(128, 256, 128, 256)) == 3       # shared-memory rings do not fit
+    assert call(til=(256, 256, 128, 256)) == 3       # shared-memory rings do not fit
     assert call(b=B.data_ptr() + 2) == 4
     assert "T_MA" in atb.atb_last_error_message() or atb.atb_last_error_message() != ""
     torch.cuda.synchronize()

@@ -77,8 +77,8 @@ def test_calibration_measures_and_fits_on_this_gpu(tmp_path):
     tilings = [(128, 256, 64, 256), (64, 256, 64, 256), (128, 128, 64, 256), (128, 256, 64, 128), (128, 256, 64, 512)]
     records = calibrate.measure([(2048, 2048, 2048), (1024, 4096, 1024)], tilings, reps=3)
     assert len(records) == 10 and all(r["tflops"] > 10 for r in records)
-    values, ev = calibrate.fit(records, {"a_bytes": (3.0, 3.6), "load_latency_cycles": (1200.0, 2000.0)})
-    assert set(values) == {"a_bytes", "load_latency_cycles"} and 0.5 < ev["pick_quality_mean"] <= 1.0
+    values, ev = calibrate.fit(records, {"convert_cycles": (300.0, 400.0), "load_latency_cycles": (1200.0, 2000.0)})
+    assert set(values) == {"convert_cycles", "load_latency_cycles"} and 0.5 < ev["pick_quality_mean"] <= 1.0
 
 
 def test_quantise_and_gemm_capture_into_a_cuda_graph():

@@ -47,6 +47,10 @@ def test_score_matches_oracle_formulas():
                     ec *= hw.coarse_slab_factor
                 if hw.mma_rows > 0 and T_K > 64 and hw.deep_kstep_factor > 0:
                     ec *= hw.deep_kstep_factor
+                if hw.mma_rows > 0 and (hw.convert_cycles > 0 or hw.convert_exposed_cycles > 0):
+                    # conversion of A on the compute side: a unit of mma_rows x 64 elements feeds T_N columns
+                    t_mma = 2.0 * hw.mma_rows * 64 * T_N / hw.peak_flops_per_cycle
+                    ec *= t_mma / max(t_mma + hw.convert_exposed_cycles, hw.convert_cycles)
                 assert math.isclose(s.ai, ai, rel_tol=1e-12)
                 assert math.isclose(s.eff_micro, em, rel_tol=1e-12)
                 assert math.isclose(s.eff_core, ec, rel_tol=1e-12)
@@ -54,6 +58,10 @@ def test_score_matches_oracle_formulas():
                 assert math.isclose(s.predicted_flops, perf, rel_tol=1e-12)
                 c_term = hw.c_buf_bytes * T_MC * T_N
                 buf = model.buffer_bytes(T_MA, T_MC, T_K, T_N, hw.a_buf_bytes, hw.b_buf_bytes, 0.0, hw.a_scratch_bytes)
+                if 0 < hw.a_unit_cols < T_K:
+                    # A is buffered 64 columns deep whatever T_K is: Eq. 1's A terms at that depth, the B term at T_K
+                    buf = model.buffer_bytes(T_MA, T_MC, hw.a_unit_cols, T_N, hw.a_buf_bytes, 0.0, 0.0, hw.a_scratch_bytes) + \
+                        model.buffer_bytes(T_MA, T_MC, T_K, T_N, 0.0, hw.b_buf_bytes, 0.0, 0.0)
                 if hw.acc_capacity_bytes > 0:
                     assert math.isclose(s.buf_bytes_used, buf, rel_tol=1e-12)
                     assert math.isclose(s.acc_bytes_used, c_term, rel_tol=1e-12)
@@ -107,6 +115,7 @@ def test_b200_refinements_can_be_switched_off():
     hw = atb.atb_hw_params_b200()
     hw.mma_rows = 0; hw.load_latency_cycles = 0.0; hw.pair_efficiency = 0.0; hw.launch_seconds = 0.0
     hw.tile_fixed_cycles = 0.0; hw.drain_cycles_per_column = 0.0; hw.pair_tile_cycles = 0.0; hw.thin_slab_cost = 1.0; hw.coarse_slab_factor = 0.0; hw.deep_kstep_factor = 0.0
+    hw.convert_cycles = 0.0; hw.convert_exposed_cycles = 0.0; hw.convert_latency_cycles = 0.0
     _, scores = atb.atb_select_tiling(8192, 8192, 8192, hw)
     for s in scores:
         t = (s.t.T_MA, s.t.T_MC, s.t.T_K, s.t.T_N)
