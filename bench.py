@@ -538,17 +538,17 @@ def run_entry(args):
         call = lambda: atb.atb_gemm_bfp16_out(M, N, K, *tiling, mant, plane, B_dev, Cm, Ce, stream=stream)
     else:
         Bt_m, Bt_e = atb.atb_quantize_bfp16(B_dev.float().t().contiguous())      # planes of B transposed, once
-        tiling = (128, 256, 64, 256)
+        tiling = tuple(args.tiling) if args.tiling else (128, 256, 64, 256)      # T_MA is free, the rest fixed
         if args.entry == "config1":
             A16 = A_dev.to(torch.bfloat16)
             C = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
-            kernel, what, quantises = "atb_gemm_cfg_kernel<A bf16, C bf16>", "atb_gemm_config(1)", False
-            call = lambda: atb.atb_gemm_config(1, M, N, K, A16, None, Bt_m, Bt_e, C, stream=stream)
+            kernel, what, quantises = "atb_gemm_cfg_kernel<A bf16, C bf16>", "atb_gemm_config_tiled(1)", False
+            call = lambda: atb.atb_gemm_config_tiled(1, M, N, K, *tiling, A16, None, Bt_m, Bt_e, C, stream=stream)
         else:
             Cm = torch.empty((M, N), dtype=torch.int8, device=dev)
             Ce = torch.empty(atb.atb_bfp16_exp_bytes(M, N), dtype=torch.uint8, device=dev)
-            kernel, what, quantises = "atb_gemm_cfg_kernel<A BFP16, C BFP16>", "atb_quantize_bfp16 + atb_gemm_config(2)", True
-            call = lambda: atb.atb_gemm_config(2, M, N, K, mant, plane, Bt_m, Bt_e, Cm, Ce, stream=stream)
+            kernel, what, quantises = "atb_gemm_cfg_kernel<A BFP16, C BFP16>", "atb_quantize_bfp16 + atb_gemm_config_tiled(2)", True
+            call = lambda: atb.atb_gemm_config_tiled(2, M, N, K, *tiling, mant, plane, Bt_m, Bt_e, Cm, Ce, stream=stream)
     torch.cuda.synchronize()
 
     def step(ev=None):

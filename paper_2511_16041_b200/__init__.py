@@ -71,7 +71,7 @@ class Tiling(NamedTuple):
 
 EXPORTED_SYMBOLS = [
     "atb_status_string", "atb_last_error_message", "atb_bfp16_mant_bytes", "atb_bfp16_exp_bytes",
-    "atb_quantize_bfp16", "atb_gemm", "atb_gemm_bfp16_out", "atb_gemm_config", "atb_gemm_splitk", "atb_gemm_splitk_workspace_bytes", "atb_select_splits",
+    "atb_quantize_bfp16", "atb_gemm", "atb_gemm_bfp16_out", "atb_gemm_config", "atb_gemm_config_tiled", "atb_gemm_splitk", "atb_gemm_splitk_workspace_bytes", "atb_select_splits",
     "atb_gemm_splitk_noalloc",
     "atb_tiling_supported", "atb_tiling_plan", "atb_device_status",
     "atb_hw_params_b200", "atb_hw_params_xdna2", "atb_score_tiling", "atb_select_tiling",
@@ -103,6 +103,8 @@ def load_library():
     lib.atb_gemm_bfp16_out.argtypes = [i64, i64, i64, ci, ci, ci, ci, vp, vp, vp, i64, vp, vp, vp]
     lib.atb_gemm_config.restype = ci
     lib.atb_gemm_config.argtypes = [ci, i64, i64, i64, vp, vp, i64, vp, vp, vp, vp, i64, vp]
+    lib.atb_gemm_config_tiled.restype = ci
+    lib.atb_gemm_config_tiled.argtypes = [ci, i64, i64, i64, ci, ci, ci, ci, vp, vp, i64, vp, vp, vp, vp, i64, vp]
     lib.atb_gemm_splitk.restype = ci
     lib.atb_gemm_splitk.argtypes = [i64, i64, i64, ci, ci, ci, ci, vp, vp, vp, i64, vp, i64, ci, vp, ctypes.c_size_t, vp]
     lib.atb_gemm_splitk_noalloc.restype = ci
@@ -250,11 +252,33 @@ def atb_gemm_bfp16_out(M, N, K, T_MA, T_MC, T_K, T_N, A_mant, A_exp, B, C_mant=N
     return C_mant, C_exp
 
 
-def atb_gemm_config(config, M, N, K, A, A_exp, Bt_mant, Bt_exp, C=None, C_exp=None, stream=None):
-    """The paper's precision configurations with the BFP16 operand on the B side (planes of B transposed).
+def atb_gemm_config_tiled(config, M, N, K, T_MA, T_MC, T_K, T_N, A, A_exp, Bt_mant, Bt_exp, C=None, C_exp=None, stream=None):
+    """The paper's precision configurations with the BFP16 operand on the B side (planes of B transposed),
+    A streamed in slabs of ``T_MA`` rows (``T_MC, T_K, T_N`` = 256, 64, 256).
 
     ``config=1``: ``A`` is a bf16 ``[M, K]`` tensor (``A_exp=None``); returns bf16 ``C``.
     ``config=2``: ``A`` / ``A_exp`` are BFP16 planes; returns ``(C_mant, C_exp)``."""
+    import torch
+    dev = Bt_mant.device
+    if config == 1:
+        if C is None:
+            C = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
+        _check(load_library().atb_gemm_config_tiled(1, M, N, K, T_MA, T_MC, T_K, T_N, _dev_ptr(A), None, A.stride(0),
+                                                    _dev_ptr(Bt_mant), _dev_ptr(Bt_exp), _dev_ptr(C), None, C.stride(0),
+                                                    _stream_ptr(stream)))
+        return C
+    if C is None:
+        C = torch.empty((M, N), dtype=torch.int8, device=dev)
+    if C_exp is None:
+        C_exp = torch.empty(atb_bfp16_exp_bytes(M, N), dtype=torch.uint8, device=dev)
+    _check(load_library().atb_gemm_config_tiled(config, M, N, K, T_MA, T_MC, T_K, T_N, _dev_ptr(A),
+                                                _dev_ptr(A_exp) if A_exp is not None else None, K, _dev_ptr(Bt_mant),
+                                                _dev_ptr(Bt_exp), _dev_ptr(C), _dev_ptr(C_exp), N, _stream_ptr(stream)))
+    return C, C_exp
+
+
+def atb_gemm_config(config, M, N, K, A, A_exp, Bt_mant, Bt_exp, C=None, C_exp=None, stream=None):
+    """``atb_gemm_config_tiled`` at the tiling (128, 256, 64, 256); goes through the C entry of the same name."""
     import torch
     dev = Bt_mant.device
     if config == 1:

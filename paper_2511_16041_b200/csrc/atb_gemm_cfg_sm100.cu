@@ -10,10 +10,15 @@
 // K-major form the UMMA takes for its N-side operand; the dequantised tile is laid out like the
 // dequantised A slabs of atb_gemm_kernel and read with a K-major descriptor.
 //
-// Fixed tiling: T_MA = 128, T_MC = 256, T_K = 64, T_N = 256 (rho = 2).  Units of 128 rows x 64 K
-// flow through the rings: two A units and two B units per K-step.
+// Tiling: T_MC = 256, T_K = 64, T_N = 256, and T_MA in {32, 64, 128, 256} (rho = 8, 4, 2, 1): A is the
+// streamed operand, as in the paper, and T_MA is the height of the slabs it is buffered in - the unit
+// of loading (one TMA box and, for BFP16 A, one raw-ring buffer with its own barrier per slab).  The
+// UMMA consumes 128-row operand units; slabs thinner than that are gathered (BF16 A: the boxes of a
+// unit land side by side under one barrier; BFP16 A: a dequantiser group converts the slabs of a unit
+// as one bundle), a 256-row slab is two units under one barrier.  For fixed data the result is
+// bit-identical for every T_MA.
 //   warp 0      TMA producer of raw B units (mantissa box + exponent box)
-//   warp 22     TMA producer of A units: raw BFP16 (config 2) or BF16 straight into the operand
+//   warp 22     TMA producer of A slabs: raw BFP16 (config 2) or BF16 straight into the operand
 //               ring, K-major with the 128-byte swizzle (config 1: nothing to convert)
 //   warp 1      UMMA issuer: 128 x 256 x 16, both operands K-major
 //   warps 2-5   epilogue (BF16 or quantising BFP16, shared with atb_gemm_kernel)
@@ -26,28 +31,40 @@ namespace {
 
 __device__ unsigned int g_cfg_error_flag = 0;
 
-struct CfgDq {                                         // what dequant_slab needs to know
-    static constexpr int SLOTS_PER_ROW = 4, SLOTS = 128 * 4, GROUP_THREADS = 128;
-    static constexpr int DQ_ITERS = 4, ROWS_PER_ITER = 32;
+template <int ROWS>
+struct CfgDq {                                         // what dequant_slab needs to know about a slab of ROWS rows
+    static constexpr int SLOTS_PER_ROW = 4, SLOTS = ROWS * 4, GROUP_THREADS = 128;
+    static constexpr int DQ_ITERS = (SLOTS + GROUP_THREADS - 1) / GROUP_THREADS, ROWS_PER_ITER = 32;
     static constexpr uint32_t KHALF_BYTES = 128 * 128, GROUP_BYTES = 128 * 128;
 };
 
-template <bool A_Q>
+template <int T_MA, bool A_Q>
 struct CfgK {
-    static constexpr int T_K = 64, T_N = 256;
+    static constexpr int T_K = 64, T_N = 256, T_MC = 256;
+    static_assert(T_MA == 32 || T_MA == 64 || T_MA == 128 || T_MA == 256, "slab height");
+    static constexpr int RHO = T_MC / T_MA;                           // slabs of A per K-step
+    static constexpr int SPG = T_MA < 128 ? 128 / T_MA : 1;           // slabs per 128-row operand unit
+    static constexpr int GPS = T_MA > 128 ? T_MA / 128 : 1;           // operand units per slab
     static constexpr uint32_t UNIT_BYTES = 128 * 128;                 // 128 rows x 64 bf16
-    static constexpr uint32_t RAW_MANT_BYTES = 128 * 64, RAW_BYTES = RAW_MANT_BYTES + 128 * 8;
+    static constexpr uint32_t RAW_MANT_BYTES = 128 * 64, RAW_BYTES = RAW_MANT_BYTES + 128 * 8;      // a raw B unit
+    static constexpr uint32_t SLAB_MANT_BYTES = T_MA * 64, SLAB_RAW_BYTES = SLAB_MANT_BYTES + T_MA * 8;
+    static constexpr uint32_t SLAB_BF16_BYTES = T_MA * 128;           // a BF16 slab of A
     static constexpr int DA = A_Q ? 2 : 0, DB = 4 - DA;               // dequantiser groups per stream
     static constexpr int NA = 4;                                      // operand units of A in shared memory
-    static constexpr int NAR = A_Q ? 4 : 0;                           // raw A units
+    static constexpr int NAH = NA / GPS;                              // ... counted in hand-overs (a 256-row slab is one)
+    static constexpr int NAS = A_Q ? (T_MA <= 128 ? 4 * SPG : 2) : 0; // raw A slabs: 512 rows of look-ahead
+    static constexpr int LAR = A_Q ? ring_bars(NAS, DA * SPG) : 0;    // barrier pairs of the raw A ring (bundles of SPG slabs)
+    static constexpr int LAH = A_Q ? ring_bars(NAH, DA) : NAH;        // barrier pairs of the A operand ring
     // A converted B tile (two units) is held for a whole K-step, by both row groups: three tiles
     // where shared memory allows (config 1), two otherwise.
     static constexpr int NB = A_Q ? 4 : 6, NBR = 4;                   // operand / raw units of B
     static constexpr int LB = ring_bars(NB, DB), LBR = ring_bars(NBR, DB);   // barrier pairs of the B rings
     static constexpr int GROUP_WARPS = 4;
-    static constexpr uint32_t SMEM_BYTES = 1024u + (NA + NB) * UNIT_BYTES + (NAR + NBR) * RAW_BYTES + 1024u +
-                                           4u * kEpilogueBoxBytes + 8u * (2 * NA + 2 * NAR + 2 * LB + 2 * LBR + 4) + 16u + kScaleTableBytes;
+    static constexpr uint32_t SMEM_BYTES = 1024u + (NA + NB) * UNIT_BYTES + NAS * SLAB_RAW_BYTES + NBR * RAW_BYTES + 1024u +
+                                           4u * kEpilogueBoxBytes + 8u * (2 * LAH + 2 * LAR + 2 * LB + 2 * LBR + 4) + 16u + kScaleTableBytes;
     static_assert(NB % 2 == 0 && LB % 2 == 0, "B tiles are pairs of units");
+    static_assert(!A_Q || (NAS % (DA * SPG) == 0 && LAR % SPG == 0), "whole bundles per dequantiser group");
+    static_assert(LAH <= kMaxRingBars && LAR <= kMaxRingBars, "barrier count");
     static_assert(SMEM_BYTES <= kSmemBudget, "shared memory");
 };
 
@@ -59,51 +76,68 @@ struct CfgParams {
     unsigned int* error_flag;
 };
 
-// One dequantiser group on one BFP16 stream: units arrive in ring order, the group takes every D-th.
-template <int D, int NR, int ND>
-__device__ __forceinline__ void dequant_stream(const Ctx& cx, int my, int64_t units, int t, int lane, uint32_t raw_full,
+// One dequantiser group on one BFP16 stream of slabs of ROWS rows.  Hand-over units arrive in ring order
+// and the group takes every D-th: a bundle of 128 / ROWS thin slabs that fill one 128-row operand
+// unit, one 128-row slab, or one 256-row slab that fills two units.  NRS raw slabs, NDH hand-overs in
+// the operand ring.
+template <int ROWS, int D, int NRS, int NDH>
+__device__ __forceinline__ void dequant_stream(const Ctx& cx, int my, int64_t handovers, int t, int lane, uint32_t raw_full,
                                                uint32_t raw_empty, uint32_t deq_full, uint32_t deq_empty,
                                                uint32_t raw_base, uint32_t deq_base, uint32_t scale_lut, unsigned code) {
-    constexpr uint32_t kRaw = 128 * 64 + 128 * 8, kMant = 128 * 64;
-    const DequantLane<CfgDq> ln(t, 128);
-    Cursor<NR, ring_bars(NR, D)> rr;
-    Cursor<ND, ring_bars(ND, D)> rd;
-    rr.start_at(my);
+    using Dq = CfgDq<ROWS>;
+    constexpr int SPG = ROWS < 128 ? 128 / ROWS : 1, GPS = ROWS > 128 ? ROWS / 128 : 1;
+    constexpr uint32_t kMant = ROWS * 64, kRaw = kMant + ROWS * 8;
+    const DequantLane<Dq> ln(t, ROWS);
+    Cursor<NRS, ring_bars(NRS, D * SPG)> rr;
+    Cursor<NDH, ring_bars(NDH, D)> rd;
+    rr.start_at(my * SPG);
     rd.start_at(my);
-    for (int64_t n = my; n < units; n += D) {
-        if (!wait_bar(cx, raw_full + 8 * rr.bar, rr.phase, code | 1u)) break;
-        if (!wait_bar(cx, deq_empty + 8 * rd.freed_bar(), rd.freed_parity(), code | 2u)) break;
-        const uint32_t raw = raw_base + rr.buf() * kRaw;
-        dequant_slab<CfgDq>(ln, raw, raw + kMant, scale_lut, deq_base + rd.buf() * CfgDq::GROUP_BYTES, 0, t, 128);
+    for (int64_t n = my; n < handovers; n += D) {
+        bool ok = true;
+#pragma unroll
+        for (int i = 0; i < SPG; ++i) ok = ok && wait_bar(cx, raw_full + 8 * (rr.bar + i), rr.phase, code | 1u);
+        ok = ok && wait_bar(cx, deq_empty + 8 * rd.freed_bar(), rd.freed_parity(), code | 2u);
+        if (!ok) break;
+        const uint32_t dst = deq_base + rd.buf() * GPS * Dq::GROUP_BYTES;
+        if constexpr (SPG > 1 && SPG * Dq::DQ_ITERS <= 4) {
+            dequant_bundle<Dq, SPG>(ln, raw_base + rr.buf() * kRaw, kRaw, kMant, scale_lut, dst, 0, t, ROWS);
+        } else {
+#pragma unroll
+            for (int i = 0; i < SPG; ++i) {
+                const uint32_t raw = raw_base + (rr.buf() + i) * kRaw;
+                dequant_slab<Dq>(ln, raw, raw + kMant, scale_lut, dst, i * ROWS, t, ROWS);
+            }
+        }
         fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) {
             mbar_arrive(deq_full + 8 * rd.bar);
-            mbar_arrive(raw_empty + 8 * rr.bar);
+#pragma unroll
+            for (int i = 0; i < SPG; ++i) mbar_arrive(raw_empty + 8 * (rr.bar + i));
         }
-        rr.template advance<D>();
+        rr.template advance<D * SPG>();
         rd.template advance<D>();
     }
 }
 
-template <bool A_Q, bool C_Q>
+template <int T_MA, bool A_Q, bool C_Q>
 __global__ void __launch_bounds__(kThreads, 1)
 atb_gemm_cfg_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_a_exp,
                     const __grid_constant__ CUtensorMap tm_b, const __grid_constant__ CUtensorMap tm_b_exp,
                     const __grid_constant__ CUtensorMap tm_c, const CfgParams p) {
-    using C = CfgK<A_Q>;
+    using C = CfgK<T_MA, A_Q>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* const smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
     const uint32_t a_base = smem_base;                                           // operand units of A
     const uint32_t b_base = a_base + C::NA * C::UNIT_BYTES;                      // operand units of B
     const uint32_t a_raw_base = b_base + C::NB * C::UNIT_BYTES;
-    const uint32_t b_raw_base = a_raw_base + C::NAR * C::RAW_BYTES;
-    constexpr uint32_t stage_off = ((C::NA + C::NB) * C::UNIT_BYTES + (C::NAR + C::NBR) * C::RAW_BYTES + 1023u) & ~1023u;
+    const uint32_t b_raw_base = a_raw_base + C::NAS * C::SLAB_RAW_BYTES;
+    constexpr uint32_t stage_off = ((C::NA + C::NB) * C::UNIT_BYTES + C::NAS * C::SLAB_RAW_BYTES + C::NBR * C::RAW_BYTES + 1023u) & ~1023u;
     const uint32_t bar_base = smem_base + stage_off + 4u * kEpilogueBoxBytes;
-    const uint32_t a_full = bar_base, a_empty = a_full + 8 * C::NA;
-    const uint32_t ar_full = a_empty + 8 * C::NA, ar_empty = ar_full + 8 * C::NAR;
-    const uint32_t b_full = ar_empty + 8 * C::NAR, b_empty = b_full + 8 * C::LB;
+    const uint32_t a_full = bar_base, a_empty = a_full + 8 * C::LAH;
+    const uint32_t ar_full = a_empty + 8 * C::LAH, ar_empty = ar_full + 8 * C::LAR;
+    const uint32_t b_full = ar_empty + 8 * C::LAR, b_empty = b_full + 8 * C::LB;
     const uint32_t br_full = b_empty + 8 * C::LB, br_empty = br_full + 8 * C::LBR;
     const uint32_t acc_full = br_empty + 8 * C::LBR, acc_empty = acc_full + 8 * 2;
     const uint32_t misc = acc_empty + 8 * 2;                 // [0]: TMEM base, [1]: abort flag
@@ -114,8 +148,8 @@ atb_gemm_cfg_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
     Ctx cx{misc_gen + 1, p.error_flag};
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < C::NA; ++i) { mbar_init(a_full + 8 * i, A_Q ? C::GROUP_WARPS : 1); mbar_init(a_empty + 8 * i, 1); }
-        for (int i = 0; i < C::NAR; ++i) { mbar_init(ar_full + 8 * i, 1); mbar_init(ar_empty + 8 * i, C::GROUP_WARPS); }
+        for (int i = 0; i < C::LAH; ++i) { mbar_init(a_full + 8 * i, A_Q ? C::GROUP_WARPS : 1); mbar_init(a_empty + 8 * i, 1); }
+        for (int i = 0; i < C::LAR; ++i) { mbar_init(ar_full + 8 * i, 1); mbar_init(ar_empty + 8 * i, C::GROUP_WARPS); }
         for (int i = 0; i < C::LB; ++i) { mbar_init(b_full + 8 * i, C::GROUP_WARPS); mbar_init(b_empty + 8 * i, 1); }
         for (int i = 0; i < C::LBR; ++i) { mbar_init(br_full + 8 * i, 1); mbar_init(br_empty + 8 * i, C::GROUP_WARPS); }
         for (int i = 0; i < 2; ++i) { mbar_init(acc_full + 8 * i, 1); mbar_init(acc_empty + 8 * i, 4); }
@@ -166,36 +200,41 @@ atb_gemm_cfg_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
         // ================================ TMA producer: A units ========================
         if (elect_one()) {
             bool ok = true;
-            if (A_Q) {
-                Cursor<(C::NAR > 0 ? C::NAR : 1), ring_bars((C::NAR > 0 ? C::NAR : 1), (C::DA > 0 ? C::DA : 1))> rr;
+            if constexpr (A_Q) {
+                // raw BFP16 slabs of T_MA rows, each with its own buffer and barrier
+                Cursor<C::NAS, C::LAR> rr;
                 for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
                     int mt, nt;
                     tile_coords(tile, p.m_tiles, p.n_tiles, mt, nt);
                     for (int k = 0; ok && k < p.k_steps; ++k) {
-                        for (int u = 0; u < 2; ++u) {
+                        for (int sl = 0; sl < C::RHO; ++sl) {
                             if (!(ok = wait_bar_spin(cx, ar_empty + 8 * rr.freed_bar(), rr.freed_parity(), 0x002))) break;
                             const uint32_t fr = ar_full + 8 * rr.bar;
-                            const uint32_t dst = a_raw_base + rr.buf() * C::RAW_BYTES;
-                            mbar_arrive_expect_tx(fr, C::RAW_BYTES);
-                            tma_load_2d(dst, &tm_a, k * C::T_K, mt * 256 + u * 128, fr);
-                            tma_load_2d(dst + C::RAW_MANT_BYTES, &tm_a_exp, mt * 256 + u * 128, k, fr);
+                            const uint32_t dst = a_raw_base + rr.buf() * C::SLAB_RAW_BYTES;
+                            mbar_arrive_expect_tx(fr, C::SLAB_RAW_BYTES);
+                            tma_load_2d(dst, &tm_a, k * C::T_K, mt * 256 + sl * T_MA, fr);
+                            tma_load_2d(dst + C::SLAB_MANT_BYTES, &tm_a_exp, mt * 256 + sl * T_MA, k, fr);
                             rr.template advance<1>();
                         }
                     }
                 }
             } else {
-                // BF16 A: the TMA box is the UMMA operand (K-major, 128-byte swizzle)
+                // BF16 A: the TMA boxes are the UMMA operand (K-major, 128-byte swizzle).  One barrier per
+                // hand-over: the slabs of a 128-row unit land side by side; a 256-row slab is two units.
                 Ring ra;
                 for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
                     int mt, nt;
                     tile_coords(tile, p.m_tiles, p.n_tiles, mt, nt);
                     for (int k = 0; ok && k < p.k_steps; ++k) {
-                        for (int u = 0; u < 2; ++u) {
+                        for (int h = 0; h < 2 / C::GPS; ++h) {       // hand-overs of this K-step
                             if (!(ok = wait_bar_spin(cx, a_empty + 8 * ra.stage, ra.phase ^ 1u, 0x002))) break;
                             const uint32_t fa = a_full + 8 * ra.stage;
-                            mbar_arrive_expect_tx(fa, C::UNIT_BYTES);
-                            tma_load_2d(a_base + ra.stage * C::UNIT_BYTES, &tm_a, k * C::T_K, mt * 256 + u * 128, fa);
-                            ra.advance(C::NA);
+                            mbar_arrive_expect_tx(fa, C::GPS * C::UNIT_BYTES);
+#pragma unroll
+                            for (int sl = 0; sl < C::SPG; ++sl)
+                                tma_load_2d(a_base + ra.stage * C::GPS * C::UNIT_BYTES + sl * C::SLAB_BF16_BYTES, &tm_a, k * C::T_K,
+                                            mt * 256 + h * C::GPS * 128 + sl * T_MA, fa);
+                            ra.advance(C::NAH);
                         }
                     }
                 }
@@ -205,7 +244,7 @@ atb_gemm_cfg_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
         // ================================ UMMA issuer =================================
         if (elect_one()) {
             constexpr uint32_t idesc = umma_idesc_bf16_f32(128, 256, false, false);   // both operands K-major
-            Ring ra;
+            Cursor<C::NAH, C::LAH> ra;               // hand-overs of A: one per 128-row unit, or per 256-row slab
             Cursor<C::NB, C::LB> rb;                 // first unit of the B tile; the second follows it
             uint32_t acc_phase = 0;
             bool ok = true;
@@ -217,17 +256,19 @@ atb_gemm_cfg_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
                     const uint32_t bs = b_base + rb.buf() * C::UNIT_BYTES;
                     for (int g = 0; g < 2; ++g) {
                         if (k == 0 && !(ok = wait_bar_spin(cx, acc_empty + 8 * g, acc_phase ^ 1u, 0x102))) break;
-                        if (!(ok = wait_bar_spin(cx, a_full + 8 * ra.stage, ra.phase, 0x103))) break;
+                        if ((g % C::GPS) == 0 && !(ok = wait_bar_spin(cx, a_full + 8 * ra.bar, ra.phase, 0x103))) break;
                         tcgen05_fence_after_sync();
-                        const uint32_t as = a_base + ra.stage * C::UNIT_BYTES;
+                        const uint32_t as = a_base + (ra.buf() * C::GPS + (g % C::GPS)) * C::UNIT_BYTES;
 #pragma unroll
                         for (int kk = 0; kk < C::T_K / 16; ++kk) {
                             const uint64_t a_desc = umma_smem_desc_sw128(as + kk * 32, 16, 1024);
                             const uint64_t b_desc = umma_smem_desc_sw128(bs + kk * 32, 16, 1024);
                             umma_f16_ss(tmem_base + static_cast<uint32_t>(g * 256), a_desc, b_desc, idesc, (k > 0 || kk > 0) ? 1u : 0u);
                         }
-                        umma_commit(a_empty + 8 * ra.stage);
-                        ra.advance(C::NA);
+                        if ((g % C::GPS) == C::GPS - 1) {
+                            umma_commit(a_empty + 8 * ra.bar);
+                            ra.template advance<1>();
+                        }
                         if (k == p.k_steps - 1) umma_commit(acc_full + 8 * g);
                     }
                     if (!ok) break;
@@ -263,14 +304,15 @@ atb_gemm_cfg_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
     } else {
         // ================================ dequantisers ================================
         const int group = (threadIdx.x - kFirstDequantWarp * 32) / 128, t = (threadIdx.x - kFirstDequantWarp * 32) % 128;
-        int64_t units = 0;
+        int64_t units = 0;                            // 128-row units per stream over this CTA's tiles
         for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) units += 2 * static_cast<int64_t>(p.k_steps);
         if (A_Q && group < C::DA) {
-            dequant_stream<(C::DA > 0 ? C::DA : 1), (C::NAR > 0 ? C::NAR : 1), C::NA>(
-                cx, group, units, t, lane, ar_full, ar_empty, a_full, a_empty, a_raw_base, a_base, scale_lut, 0x300);
+            if constexpr (A_Q)
+                dequant_stream<T_MA, C::DA, C::NAS, C::NAH>(cx, group, units / C::GPS, t, lane, ar_full, ar_empty, a_full, a_empty,
+                                                            a_raw_base, a_base, scale_lut, 0x300);
         } else {
-            dequant_stream<C::DB, C::NBR, C::NB>(cx, group - C::DA, units, t, lane, br_full, br_empty, b_full, b_empty,
-                                                 b_raw_base, b_base, scale_lut, 0x310);
+            dequant_stream<128, C::DB, C::NBR, C::NB>(cx, group - C::DA, units, t, lane, br_full, br_empty, b_full, b_empty,
+                                                      b_raw_base, b_base, scale_lut, 0x310);
         }
     }
 
@@ -288,20 +330,20 @@ atb_gemm_cfg_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
 std::mutex g_cfg_mutex;
 unsigned int* g_cfg_flag_addr[64] = {};
 
-template <bool A_Q, bool C_Q>
+template <int T_MA, bool A_Q, bool C_Q>
 atb_status_t launch_cfg(int64_t M, int64_t N, int64_t K, const void* A, const uint8_t* A_exp, int64_t lda,
                         const int8_t* Bt_mant, const uint8_t* Bt_exp, void* Cout, uint8_t* C_exp, int64_t ldc,
                         int num_sms, unsigned int* error_flag, cudaStream_t stream) {
-    using C = CfgK<A_Q>;
+    using C = CfgK<T_MA, A_Q>;
     CUtensorMap tm_a, tm_a_exp, tm_b, tm_b_exp, tm_c;
     const int64_t M_pad = atb::round_up(M, 32), N_pad = atb::round_up(N, 32);
     if (A_Q) {
-        if (!make_map_2d(&tm_a, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, A, K, M, K, 64, 128, CU_TENSOR_MAP_SWIZZLE_NONE) ||
-            !make_map_2d(&tm_a_exp, CU_TENSOR_MAP_DATA_TYPE_UINT64, 8, A_exp, M_pad, atb::ceil_div(K, 64), M_pad * 8, 128, 1,
+        if (!make_map_2d(&tm_a, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, A, K, M, K, 64, T_MA, CU_TENSOR_MAP_SWIZZLE_NONE) ||
+            !make_map_2d(&tm_a_exp, CU_TENSOR_MAP_DATA_TYPE_UINT64, 8, A_exp, M_pad, atb::ceil_div(K, 64), M_pad * 8, T_MA, 1,
                          CU_TENSOR_MAP_SWIZZLE_NONE))
             return atb::fail(ATB_ERR_CUDA, "cuTensorMapEncodeTiled failed for the planes of A");
     } else {
-        if (!make_map_2d(&tm_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, A, K, M, lda * 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B))
+        if (!make_map_2d(&tm_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, A, K, M, lda * 2, 64, T_MA, CU_TENSOR_MAP_SWIZZLE_128B))
             return atb::fail(ATB_ERR_CUDA, "cuTensorMapEncodeTiled failed for A");
         tm_a_exp = tm_a;                                   // unused
     }
@@ -323,7 +365,7 @@ atb_status_t launch_cfg(int64_t M, int64_t N, int64_t K, const void* A, const ui
     p.C_exp = C_exp;
     p.c_exp_rows = M_pad;
     p.error_flag = error_flag;
-    auto kernel = atb_gemm_cfg_kernel<A_Q, C_Q>;
+    auto kernel = atb_gemm_cfg_kernel<T_MA, A_Q, C_Q>;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(C::SMEM_BYTES));
     if (e != cudaSuccess) return atb::fail(ATB_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
     const int64_t tiles = static_cast<int64_t>(p.m_tiles) * p.n_tiles;
@@ -336,12 +378,15 @@ atb_status_t launch_cfg(int64_t M, int64_t N, int64_t K, const void* A, const ui
 
 }  // namespace
 
-extern "C" atb_status_t atb_gemm_config(int config, int64_t M, int64_t N, int64_t K,
-                                        const void* A_dev, const uint8_t* A_exp_dev, int64_t lda,
-                                        const int8_t* Bt_mant_dev, const uint8_t* Bt_exp_dev,
-                                        void* C_dev, uint8_t* C_exp_dev, int64_t ldc, void* stream) {
+extern "C" atb_status_t atb_gemm_config_tiled(int config, int64_t M, int64_t N, int64_t K, int T_MA, int T_MC, int T_K, int T_N,
+                                              const void* A_dev, const uint8_t* A_exp_dev, int64_t lda,
+                                              const int8_t* Bt_mant_dev, const uint8_t* Bt_exp_dev,
+                                              void* C_dev, uint8_t* C_exp_dev, int64_t ldc, void* stream) {
     atb::clear_error();
     if (config != 1 && config != 2) return atb::fail(ATB_ERR_BAD_TILING, "config=%d: 1 (A BF16, B BFP16, C BF16) or 2 (all BFP16)", config);
+    if (T_MC != 256 || T_K != 64 || T_N != 256 || !(T_MA == 32 || T_MA == 64 || T_MA == 128 || T_MA == 256))
+        return atb::fail(ATB_ERR_BAD_TILING, "the precision configurations run T_MC = 256, T_K = 64, T_N = 256 with T_MA in {32, 64, 128, 256} "
+                                             "(got T_MA=%d, T_MC=%d, T_K=%d, T_N=%d)", T_MA, T_MC, T_K, T_N);
     if (!A_dev || !Bt_mant_dev || !Bt_exp_dev || !C_dev || (config == 2 && (!A_exp_dev || !C_exp_dev)))
         return atb::fail(ATB_ERR_NULL_POINTER, "operand pointers must be non-NULL");
     if (M < 1 || N < 16 || N % 16 != 0 || K < 16 || K % 16 != 0 || M > (1ll << 30) || N > (1ll << 30) || K > (1ll << 30))
@@ -370,9 +415,24 @@ extern "C" atb_status_t atb_gemm_config(int config, int64_t M, int64_t N, int64_
         flag = g_cfg_flag_addr[dev];
     }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (config == 1)
-        return launch_cfg<false, false>(M, N, K, A_dev, nullptr, lda, Bt_mant_dev, Bt_exp_dev, C_dev, nullptr, ldc, sms, flag, st);
-    return launch_cfg<true, true>(M, N, K, A_dev, A_exp_dev, K, Bt_mant_dev, Bt_exp_dev, C_dev, C_exp_dev, N, sms, flag, st);
+#define ATB_CFG_CASE(TMA_)                                                                                                     \
+    case TMA_:                                                                                                                 \
+        if (config == 1)                                                                                                       \
+            return launch_cfg<TMA_, false, false>(M, N, K, A_dev, nullptr, lda, Bt_mant_dev, Bt_exp_dev, C_dev, nullptr, ldc, sms, flag, st); \
+        return launch_cfg<TMA_, true, true>(M, N, K, A_dev, A_exp_dev, K, Bt_mant_dev, Bt_exp_dev, C_dev, C_exp_dev, N, sms, flag, st);
+    switch (T_MA) {
+        ATB_CFG_CASE(32) ATB_CFG_CASE(64) ATB_CFG_CASE(128) ATB_CFG_CASE(256)
+    }
+#undef ATB_CFG_CASE
+    return atb::fail(ATB_ERR_BAD_TILING, "no kernel for T_MA=%d", T_MA);
+}
+
+extern "C" atb_status_t atb_gemm_config(int config, int64_t M, int64_t N, int64_t K,
+                                        const void* A_dev, const uint8_t* A_exp_dev, int64_t lda,
+                                        const int8_t* Bt_mant_dev, const uint8_t* Bt_exp_dev,
+                                        void* C_dev, uint8_t* C_exp_dev, int64_t ldc, void* stream) {
+    return atb_gemm_config_tiled(config, M, N, K, 128, 256, 64, 256, A_dev, A_exp_dev, lda, Bt_mant_dev, Bt_exp_dev, C_dev,
+                                 C_exp_dev, ldc, stream);
 }
 
 namespace atb {

@@ -116,3 +116,69 @@ def test_argument_errors():
     assert lib.atb_gemm_config(1, 256, 264, 256, p, None, 256, p, p, p, None, 264, None) == 2  # N % 16
     assert lib.atb_gemm_config(2, 256, 256, 256, p, None, 256, p, p, p, p, 256, None) == 1     # config 2 needs A_exp
     assert lib.atb_gemm_config(1, 256, 256, 256, p, None, 250, p, p, p, None, 256, None) == 2  # lda
+
+
+SLAB_HEIGHTS = (256, 128, 64, 32)            # T_MA: the symmetric form first, then rho = 2, 4, 8
+
+
+@pytest.mark.parametrize("shape", [(512, 512, 512), (300, 272, 448), (1000, 528, 1104), (2048, 1040, 2064)])
+def test_config1_every_slab_height_bitwise_and_against_the_definition(shape):
+    """A streamed in slabs of T_MA rows through the resident BFP16 tile of B (the orientation of the
+    paper's own experiment): only buffer lifetimes change with T_MA, so every slab height gives the
+    same bits, ragged edges included, and those bits pass the acceptance rule of the plain product."""
+    M, N, K = shape
+    A_bits = inputs.to_bf16_bits(inputs.make_A("laplace", M, K))
+    A64 = inputs.bf16_bits_to_f32(A_bits).astype(np.float64)
+    Bt_mant, Bt_exp = make_Bt_planes(K, N, 3)
+    Cr, S = ref_product(A64, Bt_mant, Bt_exp)
+    bm, be = planes_to_dev(Bt_mant, Bt_exp)
+    Ad = bf16_bits_to_dev(A_bits)
+    ref = None
+    for ma in SLAB_HEIGHTS:
+        C = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device=dev())
+        atb.atb_gemm_config_tiled(1, M, N, K, ma, 256, 64, 256, Ad, None, bm, be, C)
+        atb.atb_device_status()
+        bits = bf16_dev_to_bits(C)
+        if ref is None:
+            ref = bits
+            bad, ratio = oracle.check_tolerance(bits, Cr, S)
+            assert bad == 0 and ratio < 0.75, (shape, ma, bad, ratio)
+        assert np.array_equal(bits, ref), (shape, ma)
+
+
+@pytest.mark.parametrize("shape", [(512, 512, 512), (300, 272, 448), (1000, 528, 1104)])
+def test_config2_every_slab_height_bitwise(shape):
+    """All-BFP16 configuration: raw slabs of T_MA rows, each with its own buffer and barrier, converted
+    in bundles (thin slabs) or as two operand units (256 rows).  The BFP16 planes of C are bit-identical
+    for every slab height, and equal to those of the fixed-tiling entry point."""
+    M, N, K = shape
+    A = inputs.make_A("outlier", M, K)
+    am, ae = oracle.quantize_bfp16(A)
+    Bt_mant, Bt_exp = make_Bt_planes(K, N, 7)
+    amd, aed = planes_to_dev(am, ae)
+    bm, be = planes_to_dev(Bt_mant, Bt_exp)
+    Cm0, Ce0 = atb.atb_gemm_config(2, M, N, K, amd, aed, bm, be)
+    atb.atb_device_status()
+    # the reference entry itself against the definition (half a quantisation step, a whole one where saturated)
+    Cr, S = ref_product(oracle.dequantize(am, ae), Bt_mant, Bt_exp)
+    got_e = atb.exp_plane_to_logical(Ce0.cpu().numpy(), M, N)
+    got_m = Cm0.cpu().numpy()
+    half_step = np.repeat(np.ldexp(1.0, got_e.astype(np.int64) - 134), 8, axis=1)
+    q_err = np.where(np.abs(got_m.astype(np.int64)) == 127, 2.0 * half_step, half_step)
+    assert np.all(np.abs(oracle.dequantize(got_m, got_e) - Cr) <= q_err + S * 2.0 ** -12), shape
+    for ma in SLAB_HEIGHTS:
+        Cm = torch.full((M, N), 55, dtype=torch.int8, device=dev())
+        Ce = torch.full((atb.atb_bfp16_exp_bytes(M, N),), 199, dtype=torch.uint8, device=dev())
+        atb.atb_gemm_config_tiled(2, M, N, K, ma, 256, 64, 256, amd, aed, bm, be, Cm, Ce)
+        atb.atb_device_status()
+        assert torch.equal(Cm, Cm0) and torch.equal(Ce, Ce0), (shape, ma)
+
+
+def test_config_tiled_rejects_other_tilings():
+    lib = atb.load_library()
+    t = torch.zeros(256 * 256, dtype=torch.int8, device=dev())
+    p = t.data_ptr()
+    ok = lambda til: lib.atb_gemm_config_tiled(1, 256, 256, 256, *til, p, None, 256, p, p, p, None, 256, None)
+    assert ok((128, 256, 64, 256)) == 0 and ok((32, 256, 64, 256)) == 0
+    assert ok((128, 256, 64, 128)) == 3 and ok((128, 128, 64, 256)) == 3 and ok((48, 256, 64, 256)) == 3 and ok((128, 256, 128, 256)) == 3
+    torch.cuda.synchronize()
