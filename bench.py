@@ -538,16 +538,19 @@ def run_entry(args):
         call = lambda: atb.atb_gemm_bfp16_out(M, N, K, *tiling, mant, plane, B_dev, Cm, Ce, stream=stream)
     else:
         Bt_m, Bt_e = atb.atb_quantize_bfp16(B_dev.float().t().contiguous())      # planes of B transposed, once
-        tiling = tuple(args.tiling) if args.tiling else (128, 256, 64, 256)      # T_MA is free, the rest fixed
+        # T_MA is free; T_MC = 512 is the CTA pair that shares the converted B tile, 256 one SM
+        tiling = tuple(args.tiling) if args.tiling else (128, 512, 64, 256)
         if args.entry == "config1":
             A16 = A_dev.to(torch.bfloat16)
             C = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
-            kernel, what, quantises = "atb_gemm_cfg_kernel<A bf16, C bf16>", "atb_gemm_config_tiled(1)", False
+            form = "CTA pair" if tiling[1] == 512 else "single CTA"
+            kernel, what, quantises = f"atb_gemm_cfg_kernel<A bf16, C bf16, {form}>", "atb_gemm_config_tiled(1)", False
             call = lambda: atb.atb_gemm_config_tiled(1, M, N, K, *tiling, A16, None, Bt_m, Bt_e, C, stream=stream)
         else:
             Cm = torch.empty((M, N), dtype=torch.int8, device=dev)
             Ce = torch.empty(atb.atb_bfp16_exp_bytes(M, N), dtype=torch.uint8, device=dev)
-            kernel, what, quantises = "atb_gemm_cfg_kernel<A BFP16, C BFP16>", "atb_quantize_bfp16 + atb_gemm_config_tiled(2)", True
+            form = "CTA pair" if tiling[1] == 512 else "single CTA"
+            kernel, what, quantises = f"atb_gemm_cfg_kernel<A BFP16, C BFP16, {form}>", "atb_quantize_bfp16 + atb_gemm_config_tiled(2)", True
             call = lambda: atb.atb_gemm_config_tiled(2, M, N, K, *tiling, mant, plane, Bt_m, Bt_e, Cm, Ce, stream=stream)
     torch.cuda.synchronize()
 

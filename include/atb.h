@@ -191,8 +191,9 @@ atb_status_t atb_gemm_bfp16_out(int64_t M, int64_t N, int64_t K, int T_MA, int T
  *   C_dev:       config 1: bf16 C[M][ldc] (ldc >= N, ldc % 8 == 0), C_exp_dev = NULL;
  *                config 2: int8 mantissas [M][N] and the exponent plane in C_exp_dev, as
  *                atb_gemm_bfp16_out writes them (ldc is ignored).
- * Shapes: M >= 1, N % 16 == 0, K % 16 == 0.  atb_gemm_config runs the tiling T_MA = 128, T_MC = 256,
- * T_K = 64, T_N = 256.  Errors as for atb_gemm; an unknown config is ATB_ERR_BAD_TILING. */
+ * Shapes: M >= 1, N % 16 == 0, K % 16 == 0.  atb_gemm_config runs T_MA = 128, T_K = 64, T_N = 256 on a pair of SMs
+ * (T_MC = 512, see atb_gemm_config_tiled) where M > 256 and on one SM (T_MC = 256) otherwise; the result does
+ * not depend on that choice.  Errors as for atb_gemm; an unknown config is ATB_ERR_BAD_TILING. */
 atb_status_t atb_gemm_config(int config, int64_t M, int64_t N, int64_t K,
                              const void* A_dev, const uint8_t* A_exp_dev, int64_t lda,
                              const int8_t* Bt_mant_dev, const uint8_t* Bt_exp_dev,
@@ -200,9 +201,14 @@ atb_status_t atb_gemm_config(int config, int64_t M, int64_t N, int64_t K,
 /* The same with the asymmetric-buffering knob of Section 3 in the paper's own orientation (the experiment
  * of Section 6.1 / Table 1: the BFP16 tile of B stays put, A streams through it in slabs of T_MA rows):
  * T_MA in {32, 64, 128, 256} is the height of the slabs A is loaded and buffered in - one TMA box and, for a
- * BFP16 A, one raw buffer with its own barrier per slab; T_MA = 256 = T_MC is the symmetric form.  T_MC = 256,
- * T_K = 64 and T_N = 256 are the only values accepted for the other three (else ATB_ERR_BAD_TILING).
- * For fixed operands the result is bit-identical for every T_MA. */
+ * BFP16 A, one raw buffer with its own barrier per slab.  T_K = 64 and T_N = 256 are fixed; T_MC is
+ *   256: one SM holds the 256 x 256 accumulator and converts the whole B tile once per K-step;
+ *   512: a pair of SMs (tcgen05 cta_group::2) holds 256 rows each and shares the B tile - each converts half of
+ *        it, so a converted B element feeds 512 rows (the array-level sharing of Section 3.2, Eq. 2, applied to
+ *        the resident operand) and the conversions per FLOP halve.
+ * Per SM - the paper's "core" - the accumulator is 256 rows tall in both forms, so rho per core = 256 / T_MA
+ * and T_MA = 256 is the symmetric form of both.  Any other (T_MC, T_K, T_N) is ATB_ERR_BAD_TILING.
+ * For fixed operands the result is bit-identical for every T_MA and for both values of T_MC. */
 atb_status_t atb_gemm_config_tiled(int config, int64_t M, int64_t N, int64_t K, int T_MA, int T_MC, int T_K, int T_N,
                                    const void* A_dev, const uint8_t* A_exp_dev, int64_t lda,
                                    const int8_t* Bt_mant_dev, const uint8_t* Bt_exp_dev,

@@ -254,7 +254,8 @@ def atb_gemm_bfp16_out(M, N, K, T_MA, T_MC, T_K, T_N, A_mant, A_exp, B, C_mant=N
 
 def atb_gemm_config_tiled(config, M, N, K, T_MA, T_MC, T_K, T_N, A, A_exp, Bt_mant, Bt_exp, C=None, C_exp=None, stream=None):
     """The paper's precision configurations with the BFP16 operand on the B side (planes of B transposed),
-    A streamed in slabs of ``T_MA`` rows (``T_MC, T_K, T_N`` = 256, 64, 256).
+    A streamed in slabs of ``T_MA`` rows; ``T_K, T_N`` = 64, 256 and ``T_MC`` = 256 (one SM) or 512 (a CTA pair
+    that shares the converted B tile).
 
     ``config=1``: ``A`` is a bf16 ``[M, K]`` tensor (``A_exp=None``); returns bf16 ``C``.
     ``config=2``: ``A`` / ``A_exp`` are BFP16 planes; returns ``(C_mant, C_exp)``."""
@@ -278,7 +279,8 @@ def atb_gemm_config_tiled(config, M, N, K, T_MA, T_MC, T_K, T_N, A, A_exp, Bt_ma
 
 
 def atb_gemm_config(config, M, N, K, A, A_exp, Bt_mant, Bt_exp, C=None, C_exp=None, stream=None):
-    """``atb_gemm_config_tiled`` at the tiling (128, 256, 64, 256); goes through the C entry of the same name."""
+    """``atb_gemm_config_tiled`` with 128-row slabs, on a CTA pair where M > 256; goes through the C entry of the
+    same name."""
     import torch
     dev = Bt_mant.device
     if config == 1:

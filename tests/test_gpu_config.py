@@ -119,13 +119,15 @@ def test_argument_errors():
 
 
 SLAB_HEIGHTS = (256, 128, 64, 32)            # T_MA: the symmetric form first, then rho = 2, 4, 8
+FORMS = (256, 512)                           # T_MC: one SM, or a CTA pair that shares the converted B tile
 
 
 @pytest.mark.parametrize("shape", [(512, 512, 512), (300, 272, 448), (1000, 528, 1104), (2048, 1040, 2064)])
 def test_config1_every_slab_height_bitwise_and_against_the_definition(shape):
     """A streamed in slabs of T_MA rows through the resident BFP16 tile of B (the orientation of the
-    paper's own experiment): only buffer lifetimes change with T_MA, so every slab height gives the
-    same bits, ragged edges included, and those bits pass the acceptance rule of the plain product."""
+    paper's own experiment): only buffer lifetimes change with T_MA, and only who converts which half of
+    the B tile changes between one SM and a CTA pair, so every slab height in either form gives the same
+    bits, ragged edges included, and those bits pass the acceptance rule of the plain product."""
     M, N, K = shape
     A_bits = inputs.to_bf16_bits(inputs.make_A("laplace", M, K))
     A64 = inputs.bf16_bits_to_f32(A_bits).astype(np.float64)
@@ -134,16 +136,17 @@ def test_config1_every_slab_height_bitwise_and_against_the_definition(shape):
     bm, be = planes_to_dev(Bt_mant, Bt_exp)
     Ad = bf16_bits_to_dev(A_bits)
     ref = None
-    for ma in SLAB_HEIGHTS:
-        C = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device=dev())
-        atb.atb_gemm_config_tiled(1, M, N, K, ma, 256, 64, 256, Ad, None, bm, be, C)
-        atb.atb_device_status()
-        bits = bf16_dev_to_bits(C)
-        if ref is None:
-            ref = bits
-            bad, ratio = oracle.check_tolerance(bits, Cr, S)
-            assert bad == 0 and ratio < 0.75, (shape, ma, bad, ratio)
-        assert np.array_equal(bits, ref), (shape, ma)
+    for mc in FORMS:
+        for ma in SLAB_HEIGHTS:
+            C = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device=dev())
+            atb.atb_gemm_config_tiled(1, M, N, K, ma, mc, 64, 256, Ad, None, bm, be, C)
+            atb.atb_device_status()
+            bits = bf16_dev_to_bits(C)
+            if ref is None:
+                ref = bits
+                bad, ratio = oracle.check_tolerance(bits, Cr, S)
+                assert bad == 0 and ratio < 0.75, (shape, ma, bad, ratio)
+            assert np.array_equal(bits, ref), (shape, ma, mc)
 
 
 @pytest.mark.parametrize("shape", [(512, 512, 512), (300, 272, 448), (1000, 528, 1104)])
@@ -166,12 +169,13 @@ def test_config2_every_slab_height_bitwise(shape):
     half_step = np.repeat(np.ldexp(1.0, got_e.astype(np.int64) - 134), 8, axis=1)
     q_err = np.where(np.abs(got_m.astype(np.int64)) == 127, 2.0 * half_step, half_step)
     assert np.all(np.abs(oracle.dequantize(got_m, got_e) - Cr) <= q_err + S * 2.0 ** -12), shape
-    for ma in SLAB_HEIGHTS:
-        Cm = torch.full((M, N), 55, dtype=torch.int8, device=dev())
-        Ce = torch.full((atb.atb_bfp16_exp_bytes(M, N),), 199, dtype=torch.uint8, device=dev())
-        atb.atb_gemm_config_tiled(2, M, N, K, ma, 256, 64, 256, amd, aed, bm, be, Cm, Ce)
-        atb.atb_device_status()
-        assert torch.equal(Cm, Cm0) and torch.equal(Ce, Ce0), (shape, ma)
+    for mc in FORMS:
+        for ma in SLAB_HEIGHTS:
+            Cm = torch.full((M, N), 55, dtype=torch.int8, device=dev())
+            Ce = torch.full((atb.atb_bfp16_exp_bytes(M, N),), 199, dtype=torch.uint8, device=dev())
+            atb.atb_gemm_config_tiled(2, M, N, K, ma, mc, 64, 256, amd, aed, bm, be, Cm, Ce)
+            atb.atb_device_status()
+            assert torch.equal(Cm, Cm0) and torch.equal(Ce, Ce0), (shape, ma, mc)
 
 
 def test_config_tiled_rejects_other_tilings():
@@ -179,6 +183,36 @@ def test_config_tiled_rejects_other_tilings():
     t = torch.zeros(256 * 256, dtype=torch.int8, device=dev())
     p = t.data_ptr()
     ok = lambda til: lib.atb_gemm_config_tiled(1, 256, 256, 256, *til, p, None, 256, p, p, p, None, 256, None)
-    assert ok((128, 256, 64, 256)) == 0 and ok((32, 256, 64, 256)) == 0
+    assert ok((128, 256, 64, 256)) == 0 and ok((32, 256, 64, 256)) == 0 and ok((128, 512, 64, 256)) == 0
+    assert ok((128, 384, 64, 256)) == 3 and ok((128, 512, 64, 512)) == 3
     assert ok((128, 256, 64, 128)) == 3 and ok((128, 128, 64, 256)) == 3 and ok((48, 256, 64, 256)) == 3 and ok((128, 256, 128, 256)) == 3
     torch.cuda.synchronize()
+
+
+@pytest.mark.parametrize("shape", [(8192, 4096, 1024), (4200, 4112, 2064)])
+def test_pair_form_equals_single_cta_form_at_full_launch_size(shape):
+    """Several waves of tiles over all 148 SMs (74 CTA pairs), ragged edges in the second shape: the planes
+    / the bf16 C of the CTA-pair form equal those of the single-CTA form bit for bit, for both
+    configurations, and sampled rows of config 1 pass the acceptance rule of the plain product."""
+    M, N, K = shape
+    g = torch.Generator(device=dev())
+    g.manual_seed(5)
+    A32 = torch.randn((M, K), device=dev(), generator=g)
+    Bt32 = torch.randn((N, K), device=dev(), generator=g)
+    A16 = A32.to(torch.bfloat16)
+    am, ae = atb.atb_quantize_bfp16(A32)
+    bm, be = atb.atb_quantize_bfp16(Bt32)
+    C1 = {mc: atb.atb_gemm_config_tiled(1, M, N, K, 128, mc, 64, 256, A16, None, bm, be) for mc in FORMS}
+    C2 = {mc: atb.atb_gemm_config_tiled(2, M, N, K, 64, mc, 64, 256, am, ae, bm, be) for mc in FORMS}
+    atb.atb_device_status()
+    assert torch.equal(C1[256].view(torch.int16), C1[512].view(torch.int16))
+    assert torch.equal(C2[256][0], C2[512][0]) and torch.equal(C2[256][1], C2[512][1])
+    rows = np.unique(np.concatenate([np.arange(0, M, 512), np.arange(255, M, 512), np.arange(256, M, 512), [M - 1],
+                                     np.random.default_rng(1).integers(0, M, 48)]))
+    rows_d = torch.from_numpy(rows).to(dev())
+    A64 = inputs.bf16_bits_to_f32(A16[rows_d].view(torch.int16).cpu().numpy().view(np.uint16)).astype(np.float64)
+    Bt_mant = bm.cpu().numpy()
+    Bt_exp = atb.exp_plane_to_logical(be.cpu().numpy(), N, K)
+    Cr, S = ref_product(A64, Bt_mant, Bt_exp)
+    bad, ratio = oracle.check_tolerance(C1[512][rows_d].view(torch.int16).cpu().numpy().view(np.uint16), Cr, S)
+    assert bad == 0 and ratio < 0.75, (shape, bad, ratio)
