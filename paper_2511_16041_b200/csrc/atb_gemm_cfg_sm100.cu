@@ -94,7 +94,8 @@ struct CfgK {
 };
 
 struct CfgParams {
-    int64_t M, N, K;
+    int64_t M, N, K, ldc;
+    __nv_bfloat16* C;                        // bf16 C[M][ldc] (config 1)
     int m_tiles, n_tiles, k_steps;
     uint8_t* C_exp;
     int64_t c_exp_rows;
@@ -373,7 +374,7 @@ atb_gemm_cfg_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
                 const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + static_cast<uint32_t>(g * 256);
                 const uint32_t box = smem_base + stage_off + static_cast<uint32_t>(warp - kFirstEpilogueWarp) * kEpilogueBoxBytes;
                 if (C_Q) epilogue_bfp16<C::T_N>(&tm_c, t_addr, box, lane, row0, col0, p.M, p.N, p.C_exp, p.c_exp_rows);
-                else epilogue_bf16<C::T_N>(&tm_c, t_addr, box, lane, row0, col0, p.M, p.N);
+                else epilogue_bf16<C::T_N>(&tm_c, p.C, p.ldc, t_addr, box, lane, row0, col0, p.M, p.N);
                 tcgen05_fence_before_sync();
                 __syncwarp();
                 if (lane == 0) {
@@ -454,7 +455,8 @@ atb_status_t launch_cfg(int64_t M, int64_t N, int64_t K, const void* A, const ui
         return atb::fail(ATB_ERR_CUDA, "cuTensorMapEncodeTiled failed for C");
     }
     CfgParams p;
-    p.M = M; p.N = N; p.K = K;
+    p.M = M; p.N = N; p.K = K; p.ldc = ldc;
+    p.C = static_cast<__nv_bfloat16*>(Cout);
     p.m_tiles = static_cast<int>(atb::ceil_div(M, C::T_MC));
     p.n_tiles = static_cast<int>(atb::ceil_div(N, C::T_N));
     p.k_steps = static_cast<int>(atb::ceil_div(K, C::T_K));

@@ -42,7 +42,10 @@ constexpr int kFirstDequantWarp = 6;
 constexpr int kMaxStages = 16;
 constexpr int kMaxRingBars = 32;
 constexpr uint32_t kEpilogueBoxBytes = 32 * 128;   // 32 rows x 64 bf16 columns
-constexpr uint32_t kSmallBoxBytes = 32 * 64;       // 32 rows x 32 bf16 columns (the CTA-pair kernel)
+// The CTA-pair kernel stages C in full-size boxes (128-byte rows) where 64- and 128-row slabs leave room
+// for them, and in half-size boxes under 32-row slabs, whose deeper raw ring needs the space.
+constexpr int pair_box_cols(int slab) { return slab >= 64 ? 64 : 32; }
+constexpr uint32_t pair_box_bytes(int slab) { return 32u * pair_box_cols(slab) * 2u; }
 constexpr uint32_t kScaleTableBytes = 256u * 8u;  // per exponent: the scale and its offset, see scale_table_entry
 constexpr uint32_t kSmemBudget = 232448;          // 227 KB of dynamic shared memory per CTA
 #ifdef ATB_TEST_WAIT_NS                             // test build of the timeout path only: a short limit
@@ -156,7 +159,7 @@ constexpr RingPlan plan_pair(int slab) {
     pl.tmem_cols = 512;
     const auto total = [=](int b, int g, int r) {
         return ring_smem_bytes(b_bytes, group_bytes, raw_bytes, 2, dqg, slab_bundle(slabs, r, dqg), b, g,
-                               g * (slabs / slab_bundle(slabs, r, dqg)), r, kSmallBoxBytes);
+                               g * (slabs / slab_bundle(slabs, r, dqg)), r, pair_box_bytes(slab));
     };
     const auto bars_ok = [=](int g, int r) {
         return ring_bars(r, dqg * slab_bundle(slabs, r, dqg)) <= kMaxRingBars &&
@@ -172,9 +175,9 @@ constexpr RingPlan plan_pair(int slab) {
     // Spend what is left on bf16 groups, raw slabs (up to 8 K-steps of look-ahead), then B tiles
     // (measured: the dequantised-A ring is the one whose depth pays most).
     while (ng + ng_step <= 4 && bars_ok(ng + ng_step, nr) && total(nb, ng + ng_step, nr) <= kSmemBudget) ng += ng_step;
-    // a fifth group (the epilogue boxes of this kernel are half-size to make room for it): measured +3 %
-    if (ng == 4 && bars_ok(5, nr) && total(nb, 5, nr) <= kSmemBudget) ng = 5;
     while (nr + dqg <= kMaxStages && nr * slab < 8 * 128 && bars_ok(ng, nr + dqg) && total(nb, ng, nr + dqg) <= kSmemBudget) nr += dqg;
+    // a fifth group where it still fits (under 32-row slabs, whose epilogue boxes are half-size): measured +3 % there
+    if (ng == 4 && bars_ok(5, nr) && total(nb, 5, nr) <= kSmemBudget) ng = 5;
     while (nb < 4 && total(nb + 1, ng, nr) <= kSmemBudget) ++nb;
 #if defined(ATB_RINGS_NB) && defined(ATB_RINGS_NG) && defined(ATB_RINGS_NR)
     if (ATB_RINGS_NB >= 2 && ATB_RINGS_NG >= 1 && ATB_RINGS_NR >= 1 && bars_ok(ATB_RINGS_NG, ATB_RINGS_NR) &&
@@ -552,52 +555,98 @@ __device__ __forceinline__ void dequant_bundle(const DequantLane<C>& ln, uint32_
 
 // ---------------------------------------------------------------------------------------------
 // Epilogues of one warp: N_COLS accumulator columns of its 32 TMEM lanes (rows row0 .. row0+31,
-// columns col0 ..) -> C.  `box` is the warp's staging in shared memory.  Rows and columns
-// beyond M, N are clipped by the tensor map of the TMA store.
+// columns col0 ..) -> C.  `box` is the warp's staging in shared memory.
 // ---------------------------------------------------------------------------------------------
-// BF16 C: tcgen05.ld -> round to bf16 (RNE) -> swizzled box of 32 rows x BOX_COLS columns -> TMA store.
-// BOX_COLS = 64: 128-byte rows and swizzle (4 KB); 32: 64-byte rows and swizzle (2 KB).
-template <int N_COLS, int BOX_COLS = 64>
-__device__ __forceinline__ void epilogue_bf16(const CUtensorMap* tm_c, uint32_t t_addr, uint32_t box, int lane, int row0,
-                                              int col0, int64_t M, int64_t N) {
-    static_assert(BOX_COLS == 64 || BOX_COLS == 32, "box width");
-#ifndef ATB_NO_L2_HINTS
-    const uint64_t store_policy = l2_policy_evict_first();
+// BF16 C: tcgen05.ld -> round to bf16 (RNE) -> swizzled box of 32 rows x BOX_COLS columns in shared
+// memory -> global memory.  BOX_COLS = 64: 128-byte rows (4 KB); 32: 64-byte rows (2 KB).
+// The accumulator is read 32 columns at a time; the load of the next 32 columns is issued as soon as
+// the current ones are packed to bf16, so that its latency passes behind the staging and the stores.
+// Two ways out of the box (measured: the single-CTA kernels are faster with the TMA store - one instruction in a
+// warp that competes with the dequantisers for issue slots -, the CTA-pair kernel, whose 128 x 512 accumulator
+// takes longest to drain, with direct stores: +4 % at K = 1024, +1 % at K = 8192):
+//   TMA store   one instruction per box; costs about 5.5 cycles per row whatever the row carries (23 B per
+//               cycle and SM at 128-byte rows, half of that at 64-byte rows); edges are clipped by the tensor map.
+//   direct      the warp reads the box back row-wise and writes 16-byte chunks: 8 (4) lanes cover one row
+//               segment, so every store instruction writes full 128-byte (64-byte) runs; rows and columns
+//               beyond M, N are skipped (N is a multiple of 8: a 16-byte chunk is inside or outside).
+#ifndef ATB_EPILOGUE_DIRECT          // tuning builds: -DATB_EPILOGUE_DIRECT=0|1, -DATB_EPILOGUE_DIRECT_PAIR=0|1
+#define ATB_EPILOGUE_DIRECT 0
 #endif
+#ifndef ATB_EPILOGUE_DIRECT_PAIR
+#define ATB_EPILOGUE_DIRECT_PAIR 1
+#endif
+template <int N_COLS, int BOX_COLS = 64, bool DIRECT = (ATB_EPILOGUE_DIRECT != 0)>
+__device__ __forceinline__ void epilogue_bf16(const CUtensorMap* tm_c, __nv_bfloat16* __restrict__ C, int64_t ldc, uint32_t t_addr,
+                                              uint32_t box, int lane, int row0, int col0, int64_t M, int64_t N) {
+    static_assert(BOX_COLS == 64 || BOX_COLS == 32, "box width");
+    constexpr int CPR = BOX_COLS / 8;                  // 16-byte chunks per row of the box
+    constexpr int RPI = 32 / CPR;                      // rows one store instruction of the warp covers (direct)
+    constexpr uint32_t kSwMask = CPR - 1;
+    constexpr int HALVES = BOX_COLS / 32, N_LOADS = N_COLS / 32;
     const uint32_t my_row = box + lane * (BOX_COLS * 2);
     const uint32_t sw = BOX_COLS == 64 ? static_cast<uint32_t>(lane & 7) : (static_cast<uint32_t>(lane >> 1) & 3u);
-#pragma unroll 1
-    for (int c = 0; c < N_COLS / BOX_COLS; ++c) {
-        // the previous TMA store of this warp must have finished reading the box
-        if (lane == 0) tma_store_wait_read<0>();
-        __syncwarp();
-#pragma unroll
-        for (int h = 0; h < BOX_COLS / 32; ++h) {
-            uint32_t v[32];
-            tmem_ld_32x32b_x32(t_addr + c * BOX_COLS + h * 32, v);
-            tmem_ld_wait();
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                uint32_t o[4];
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(v[j * 8 + 2 * e]),
-                                                              __uint_as_float(v[j * 8 + 2 * e + 1]));
-                    o[e] = *reinterpret_cast<uint32_t*>(&b2);
-                }
-                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(my_row + ((static_cast<uint32_t>(h * 4 + j) ^ sw) << 4)),
-                             "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]) : "memory");
-            }
-        }
-        fence_proxy_async_smem();
-        __syncwarp();
-        if (lane == 0 && row0 < M && col0 + c * BOX_COLS < N) {   // rows / columns past the edge are clipped
+    const int och = lane % CPR, orow = lane / CPR;     // direct: this lane copies chunk och of rows orow, orow + RPI, ...
 #ifndef ATB_NO_L2_HINTS
-            tma_store_2d_hint(tm_c, box, col0 + c * BOX_COLS, row0, store_policy);   // C is not read again: first to leave the L2
-#else
-            tma_store_2d(tm_c, box, col0 + c * BOX_COLS, row0);
+    const uint64_t store_policy = l2_policy_evict_first();   // C is not read again: first to leave the L2
 #endif
-            tma_store_commit();
+    uint32_t v[32];
+    tmem_ld_32x32b_x32(t_addr, v);
+#pragma unroll 1
+    for (int l = 0; l < N_LOADS; ++l) {
+        const int c = l / HALVES, h = l % HALVES;
+        tmem_ld_wait_for(v);
+        uint32_t o[16];
+#pragma unroll
+        for (int e = 0; e < 16; ++e) {
+            __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(v[2 * e]), __uint_as_float(v[2 * e + 1]));
+            o[e] = *reinterpret_cast<uint32_t*>(&b2);
+        }
+        if (l + 1 < N_LOADS) tmem_ld_32x32b_x32(t_addr + (l + 1) * 32, v);       // in flight during what follows
+        if (h == 0) {
+            // the box is free again: the TMA store that read it has finished / every lane has copied its part out
+            if constexpr (!DIRECT) { if (lane == 0) tma_store_wait_read<0>(); }
+            __syncwarp();
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(my_row + ((static_cast<uint32_t>(h * 4 + j) ^ sw) << 4)),
+                         "r"(o[4 * j]), "r"(o[4 * j + 1]), "r"(o[4 * j + 2]), "r"(o[4 * j + 3]) : "memory");
+        if (h != HALVES - 1) continue;
+        if constexpr (!DIRECT) {
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0 && row0 < M && col0 + c * BOX_COLS < N) {   // rows / columns past the edge are clipped
+#ifndef ATB_NO_L2_HINTS
+                tma_store_2d_hint(tm_c, box, col0 + c * BOX_COLS, row0, store_policy);
+#else
+                tma_store_2d(tm_c, box, col0 + c * BOX_COLS, row0);
+#endif
+                tma_store_commit();
+            }
+        } else {
+            __syncwarp();
+            const int64_t col = static_cast<int64_t>(col0) + c * BOX_COLS + och * 8;
+            __nv_bfloat16* dst = C + (static_cast<int64_t>(row0) + orow) * ldc + col;
+            const int rows_left = static_cast<int>(min(M - row0 - orow, static_cast<int64_t>(32)));     // rows r < rows_left exist
+            uint32_t src = box + static_cast<uint32_t>(orow) * (BOX_COLS * 2);
+#pragma unroll
+            for (int i = 0; i < CPR; ++i) {
+                // row r = i * RPI + orow: with 64-byte rows RPI = 8 and r's swizzle term is orow's; with 128-byte rows RPI = 4
+                const uint32_t rsw = BOX_COLS == 64 ? static_cast<uint32_t>((i * RPI + orow) & 7) : (static_cast<uint32_t>(orow >> 1) & 3u);
+                uint32_t o0, o1, o2, o3;
+                asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(o0), "=r"(o1), "=r"(o2), "=r"(o3)
+                             : "r"(src + (((static_cast<uint32_t>(och) ^ rsw) & kSwMask) << 4)));
+                if (i * RPI < rows_left && col < N) {
+#ifndef ATB_NO_L2_HINTS
+                    asm volatile("st.global.L2::cache_hint.v4.b32 [%0], {%1, %2, %3, %4}, %5;" ::"l"(dst), "r"(o0), "r"(o1), "r"(o2), "r"(o3),
+                                 "l"(store_policy) : "memory");
+#else
+                    asm volatile("st.global.v4.b32 [%0], {%1, %2, %3, %4};" ::"l"(dst), "r"(o0), "r"(o1), "r"(o2), "r"(o3) : "memory");
+#endif
+                }
+                dst += static_cast<int64_t>(RPI) * ldc;
+                src += RPI * (BOX_COLS * 2);
+            }
         }
     }
 }

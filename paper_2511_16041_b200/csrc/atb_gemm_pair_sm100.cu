@@ -16,8 +16,8 @@
 //
 // Warp roles are those of the single-CTA kernel: 0 TMA producer of B, 1 UMMA issuer (active in the
 // leader only) + TMEM owner, 2-5 epilogue, 6-21 dequantisers (4 groups of 4 warps), 22 TMA producer of A.
-// The epilogue stages C in boxes of 32 x 32 BF16 (2 KB, half the single-CTA kernel's), which leaves
-// room for a fifth dequantised-operand group.
+// The epilogue stages C in boxes of 32 x 64 BF16 and writes them out with plain coalesced stores (under
+// 32-row slabs: boxes of 32 x 32, which leaves room for a fifth dequantised-operand group).
 #include "atb_gemm_device.cuh"
 
 namespace {
@@ -30,6 +30,8 @@ struct PairCfg {
     static constexpr uint32_t B_BYTES = 4 * B_BOX_BYTES;       // this CTA's half: 2 chunks x 128 columns
     static constexpr uint32_t GROUP_BYTES = 128 * T_K * 2;
     static constexpr uint32_t KHALF_BYTES = 128 * 128;
+    static constexpr int BOX_COLS = pair_box_cols(SLAB_ROWS);   // epilogue staging box of a warp: 32 rows x BOX_COLS bf16
+    static constexpr uint32_t BOX_BYTES = pair_box_bytes(SLAB_ROWS);
     static constexpr uint32_t RAW_MANT_BYTES = SLAB_ROWS * T_K;
     static constexpr uint32_t RAW_EXP_BYTES = SLAB_ROWS * T_K / 8;
     static constexpr uint32_t RAW_BYTES = RAW_MANT_BYTES + RAW_EXP_BYTES;
@@ -52,7 +54,8 @@ struct PairCfg {
 };
 
 struct PairParams {
-    int64_t M, N, K;
+    int64_t M, N, K, ldc;
+    __nv_bfloat16* C;                        // bf16 C[M][ldc] (not used by the quantising epilogue)
     int m_tiles, n_tiles, k_steps;           // tiles of 256 x 512
     unsigned int* error_flag;
     uint8_t* C_exp;                          // QOUT: exponent plane of C and its padded row count
@@ -83,7 +86,7 @@ atb_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_c
     constexpr uint32_t raw_off = C::NB * C::B_BYTES + C::NG * C::GROUP_BYTES;
     const uint32_t raw_base = smem_base + raw_off;
     constexpr uint32_t stage_off = (raw_off + C::NR * C::RAW_BYTES + 1023u) & ~1023u;
-    constexpr uint32_t bar_off = stage_off + 4u * kSmallBoxBytes;
+    constexpr uint32_t bar_off = stage_off + 4u * C::BOX_BYTES;
     const uint32_t bar_base = smem_base + bar_off;
     const uint32_t b_full = bar_base, b_empty = b_full + 8 * C::NB;
     const uint32_t raw_full = b_empty + 8 * C::NB, raw_empty = raw_full + 8 * C::LR;
@@ -232,7 +235,7 @@ atb_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_c
             int mt, nt;
             tile_coords(tile, p.m_tiles, p.n_tiles, mt, nt);
             const int row0 = mt * 256 + static_cast<int>(rank) * 128 + q * 32;
-            const uint32_t box = smem_base + stage_off + static_cast<uint32_t>(warp - kFirstEpilogueWarp) * kSmallBoxBytes;
+            const uint32_t box = smem_base + stage_off + static_cast<uint32_t>(warp - kFirstEpilogueWarp) * C::BOX_BYTES;
             for (int nc = 0; nc < C::N_CHUNKS; ++nc) {
                 if (!(ok = wait_bar_cl(cx, acc_full + 8 * nc, acc_phase, 0x201))) break;
                 tcgen05_fence_after_sync();
@@ -241,7 +244,7 @@ atb_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_c
                 if constexpr (QOUT)
                     epilogue_bfp16<C::N_MMA>(&tm_c, t_addr, box, lane, row0, col0, p.M, p.N, p.C_exp, p.c_exp_rows);
                 else
-                    epilogue_bf16<C::N_MMA, 32>(&tm_c, t_addr, box, lane, row0, col0, p.M, p.N);
+                    epilogue_bf16<C::N_MMA, C::BOX_COLS, (ATB_EPILOGUE_DIRECT_PAIR != 0)>(&tm_c, p.C, p.ldc, t_addr, box, lane, row0, col0, p.M, p.N);
                 tcgen05_fence_before_sync();
                 __syncwarp();
                 if (lane == 0) mbar_arrive_cluster(mapa_shared(acc_empty + 8 * nc, 0));
@@ -351,12 +354,14 @@ atb_status_t launch_pair_t(const atb::GemmPlan& plan, int64_t M, int64_t N, int6
     if (QOUT) {        // int8 mantissa plane C_mant[M][ldc]: boxes of 32 rows x 64 bytes
         if (!make_map_2d(&tm_c, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Cout, N, M, ldc, 64, 32, CU_TENSOR_MAP_SWIZZLE_64B))
             return atb::fail(ATB_ERR_CUDA, "cuTensorMapEncodeTiled failed for the mantissa plane of C");
-    } else if (!make_map_2d(&tm_c, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Cout, N, M, ldc * 2, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B)) {
+    } else if (!make_map_2d(&tm_c, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Cout, N, M, ldc * 2, C::BOX_COLS, 32,
+                            C::BOX_COLS == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B)) {
         return atb::fail(ATB_ERR_CUDA, "cuTensorMapEncodeTiled failed for C");
     }
 
     PairParams p;
-    p.M = M; p.N = N; p.K = K;
+    p.M = M; p.N = N; p.K = K; p.ldc = ldc;
+    p.C = static_cast<__nv_bfloat16*>(Cout);
     p.m_tiles = static_cast<int>(atb::ceil_div(M, 256));
     p.n_tiles = static_cast<int>(atb::ceil_div(N, 512));
     p.k_steps = static_cast<int>(atb::ceil_div(K, C::T_K));

@@ -298,7 +298,7 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
                 } else if (QOUT) {
                     epilogue_bfp16<T_N>(&tm_c, t_addr, box, lane, row0, col0, p.M, p.N, p.C_exp, p.c_exp_rows);
                 } else {
-                    epilogue_bf16<T_N>(&tm_c, t_addr, box, lane, row0, col0, p.M, p.N);
+                    epilogue_bf16<T_N>(&tm_c, p.C, p.ldc, t_addr, box, lane, row0, col0, p.M, p.N);
                 }
                 tcgen05_fence_before_sync();
                 __syncwarp();
