@@ -94,7 +94,12 @@ atb_status_t atb_quantize_bfp16(const float* A_dev, int64_t M, int64_t K, int64_
  *          (the array-level sharing of Eq. 2).  Per SM - the paper's "core" - the accumulator is 128 rows
  *          tall, so T_MA = 128 is this tiling's SYMMETRIC form (rho per core = 128 / T_MA), only
  *          T_MA in {32, 64} buffer asymmetrically, and T_MA = 256 does not exist (ATB_ERR_BAD_TILING).
- * For fixed (T_MC, T_K, T_N) the result is bit-identical for every T_MA.
+ * For fixed (T_MC, T_K, T_N) the result is bit-identical for every T_MA, and every call with the same
+ * arguments on the same GPU model gives the same bits.  Between different (T_MC, T_K, T_N) results agree
+ * within FP32 rounding, not bit for bit: a persistent CTA walks K upwards for one of its tiles and downwards
+ * for the next (the next wave of tiles then starts on data the L2 still holds), so the order of a tile's
+ * additions depends on its place in the walk; only where no CTA computes more than one tile do all
+ * tilings with the same T_K add in the same order.
  * Errors: NULL_POINTER, BAD_SHAPE, BAD_TILING, MISALIGNED, UNSUPPORTED_DEVICE, CUDA. */
 atb_status_t atb_gemm(int64_t M, int64_t N, int64_t K, int T_MA, int T_MC, int T_K, int T_N,
                       const int8_t* A_mant_dev, const uint8_t* A_exp_dev,

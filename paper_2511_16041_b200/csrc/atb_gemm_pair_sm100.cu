@@ -141,11 +141,13 @@ atb_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_c
         if (elect_one()) {
             Ring rb;
             bool ok = true;
-            for (int tile = cluster_id; ok && tile < total_tiles; tile += n_clusters) {
+            int it = 0;
+            for (int tile = cluster_id; ok && tile < total_tiles; tile += n_clusters, ++it) {
                 int mt, nt;
                 tile_coords(tile, p.m_tiles, p.n_tiles, mt, nt);
                 const int colb = nt * 512 + static_cast<int>(rank) * 128;
-                for (int k = 0; ok && k < p.k_steps; ++k) {
+                for (int k0 = 0; ok && k0 < p.k_steps; ++k0) {
+                    const int k = serpentine_k(it, k0, 0, p.k_steps);
                     if (!(ok = wait_bar_cl_spin(cx, b_empty + 8 * rb.stage, rb.phase ^ 1u, 0x001))) break;
                     // both halves of the B tile are credited to the leader's barrier
                     if (leader) mbar_arrive_expect_tx(b_full + 8 * rb.stage, 2 * C::B_BYTES);
@@ -166,11 +168,13 @@ atb_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_c
 #ifndef ATB_NO_L2_HINTS
             const uint64_t a_policy = l2_policy_evict_last();   // a band's A panels serve wave after wave
 #endif
-            for (int tile = cluster_id; ok && tile < total_tiles; tile += n_clusters) {
+            int it = 0;
+            for (int tile = cluster_id; ok && tile < total_tiles; tile += n_clusters, ++it) {
                 int mt, nt;
                 tile_coords(tile, p.m_tiles, p.n_tiles, mt, nt);
                 const int row0 = mt * 256 + static_cast<int>(rank) * 128;
-                for (int k = 0; ok && k < p.k_steps; ++k) {
+                for (int k0 = 0; ok && k0 < p.k_steps; ++k0) {
+                    const int k = serpentine_k(it, k0, 0, p.k_steps);
                     for (int s = 0; s < C::SLABS; ++s) {
                         if (!(ok = wait_bar_cl_spin(cx, raw_empty + 8 * rr.freed_bar(), rr.freed_parity(), 0x002))) break;
                         const uint32_t fr = raw_full + 8 * rr.bar;

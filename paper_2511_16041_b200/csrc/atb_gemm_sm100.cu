@@ -149,9 +149,11 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
         if (elect_one()) {
             Ring rb;
             bool ok = true;
-            for (int item = blockIdx.x; ok && item < total_items; item += gridDim.x) {
+            int it = 0;
+            for (int item = blockIdx.x; ok && item < total_items; item += gridDim.x, ++it) {
                 const WorkItem w = work_item<SPLIT>(item, p);
-                for (int k = w.k_begin; ok && k < w.k_end; ++k) {
+                for (int k0 = w.k_begin; ok && k0 < w.k_end; ++k0) {
+                    const int k = serpentine_k(it, k0, w.k_begin, w.k_end);
                     if (!(ok = wait_bar_spin(cx, b_empty + 8 * rb.stage, rb.phase ^ 1u, 0x001))) break;
                     const uint32_t fb = b_full + 8 * rb.stage;
                     mbar_arrive_expect_tx(fb, C::B_BYTES);
@@ -175,9 +177,12 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
             // change: A is asked to stay in the L2 longest.
             const uint64_t a_policy = l2_policy_evict_last();
 #endif
-            for (int item = blockIdx.x; ok && item < total_items; item += gridDim.x) {
+            int it = 0;
+            for (int item = blockIdx.x; ok && item < total_items; item += gridDim.x, ++it) {
                 const WorkItem w = work_item<SPLIT>(item, p);
-                for (int kh = w.k_begin * C::KH; ok && kh < w.k_end * C::KH; ++kh) {      // 64-column rounds
+                for (int kh0 = w.k_begin * C::KH; ok && kh0 < w.k_end * C::KH; ++kh0) {      // 64-column rounds
+                    // (a downward walk keeps the two rounds of a T_K = 128 step in their upward order)
+                    const int kh = serpentine_k(it, kh0 / C::KH, w.k_begin, w.k_end) * C::KH + kh0 % C::KH;
                     for (int s = 0; s < C::RHO; ++s) {
                         if (!(ok = wait_bar_spin(cx, raw_empty + 8 * rr.freed_bar(), rr.freed_parity(), 0x002))) break;
                         const uint32_t fr = raw_full + 8 * rr.bar;

@@ -73,7 +73,8 @@ def test_atb_invariance_bitwise_across_T_MA():
 
 def test_cta_pair_equals_the_single_cta_tiling_bitwise():
     """The CTA-pair kernel (T_N = 512) adds the same products in the same order as the single-CTA 256 x 256
-    tiling with the same T_K: every element of C is bit-identical, ragged edges included."""
+    tiling with the same T_K wherever no CTA computes more than one tile (a CTA's second tile walks K
+    downwards): every element of C is bit-identical, ragged edges included."""
     for (M, N, K) in [(512, 1024, 1024), (1000, 1544, 1104)]:
         A = inputs.make_A("outlier", M, K)
         Bb = inputs.make_B_bits(K, N, None)
