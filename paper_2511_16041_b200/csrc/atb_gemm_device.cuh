@@ -319,6 +319,8 @@ __device__ __forceinline__ void tile_coords(int tile, int m_tiles, int n_tiles, 
     const int rows = min(16, m_tiles - band * 16);
     mt = band * 16 + i % rows;
     nt = i / rows;
+    // odd bands walk the columns backwards: they start on the B panels the band before them ended on
+    if (band & 1) nt = n_tiles - 1 - nt;
 }
 
 // K-step that a CTA loads `k0` steps into its `it`-th work item over [k_begin, k_end): every other work
