@@ -574,6 +574,91 @@ __device__ __forceinline__ void dequant_bundle(const DequantLane<C>& ln, uint32_
 }
 
 // ---------------------------------------------------------------------------------------------
+// The dequantiser role of atb_gemm_kernel and atb_gemm_pair_kernel: one warp of dequantiser group
+// `my_group` (thread `t` of the group).  The group does not need to know tiles or K-steps: slabs arrive in
+// ring order, so it takes every DQ_GROUPS-th bundle of the CTA's stream of `my_slabs` raw slabs, waits for the
+// raw slabs and for a free place in the operand ring, converts, and hands the operand on.
+// C: the kernel's compile-time configuration (slab height SLAB_ROWS, bundle, ring depths and barrier counts).
+// PAIR: the operand is announced on the leader CTA's barrier and the waits use cluster-scope acquire.
+// ---------------------------------------------------------------------------------------------
+template <class C, bool PAIR>
+__device__ __forceinline__ void dequantiser_role(const Ctx& cx, int t, int my_group, int warp, int lane, int64_t my_slabs,
+                                                 uint32_t raw_full, uint32_t raw_empty, uint32_t deq_full, uint32_t deq_empty,
+                                                 uint32_t raw_base, uint32_t deq_base, uint32_t scale_lut) {
+    constexpr int SLAB = C::SLAB_ROWS;
+    const DequantLane<C> ln(t, SLAB);
+#ifdef ATB_PROFILE_SKIP_DEQUANT
+    // diagnostic: the operand ring holds fixed pseudo-random bf16 values (zeros would lower the
+    // tensor cores' power and flatter the clock)
+    for (uint32_t i = threadIdx.x - kFirstDequantWarp * 32; i < C::NG * C::GROUP_BYTES / 4; i += kDequantWarps * 32) {
+        uint32_t h = (i + 1u) * 2654435761u; h ^= h >> 15; h *= 2246822519u; h ^= h >> 13;
+        const uint32_t v = (h & 0x807F807Fu) | 0x3F003F00u;          // +-[0.5, 1) in both halves
+        asm volatile("st.shared.b32 [%0], %1;" ::"r"(deq_base + i * 4), "r"(v) : "memory");
+    }
+    fence_proxy_async_smem();
+#endif
+    Cursor<C::NR, C::LR> rr;
+    Cursor<C::ND, C::LD> rd;
+    rr.start_at(my_group * C::BUNDLE);
+    rd.start_at(my_group);
+    for (int64_t n = static_cast<int64_t>(my_group) * C::BUNDLE; n < my_slabs; n += C::DQ_GROUPS * C::BUNDLE) {
+        bool ok = true;
+#pragma unroll
+        for (int i = 0; i < C::BUNDLE; ++i)        // bars and buffers of a bundle are consecutive
+            ok = ok && wait_bar_t<false, PAIR>(cx, raw_full + 8 * (rr.bar + i), rr.phase, 0x301);
+        ok = ok && wait_bar_t<false, PAIR>(cx, deq_empty + 8 * rd.freed_bar(), rd.freed_parity(), 0x302);
+        if (!ok) break;
+#ifndef ATB_PROFILE_SKIP_DEQUANT    // diagnostic: the pipeline without the conversion work (results are wrong)
+        // all slots of the bundle in flight at once where that is at most four per thread (registers)
+        if constexpr (C::BUNDLE > 1 && C::SLOTS % C::GROUP_THREADS == 0 && C::BUNDLE * C::DQ_ITERS <= 4) {
+            dequant_bundle<C, C::BUNDLE>(ln, raw_base + rr.buf() * C::RAW_BYTES, C::RAW_BYTES, C::RAW_MANT_BYTES, scale_lut,
+                                         deq_base + (rd.buf() / C::SPB) * C::GROUP_BYTES, (rd.buf() % C::SPB) * C::BUNDLE * SLAB, t, SLAB);
+        } else {
+#pragma unroll
+            for (int i = 0; i < C::BUNDLE; ++i) {
+                const uint32_t raw = raw_base + (rr.buf() + i) * C::RAW_BYTES;
+                const uint32_t dst_base = deq_base + (SLAB <= 128 ? rd.buf() / C::SPB : rd.buf() * C::GPS) * C::GROUP_BYTES;
+                dequant_slab<C>(ln, raw, raw + C::RAW_MANT_BYTES, scale_lut, dst_base,
+                                SLAB <= 128 ? ((rd.buf() % C::SPB) * C::BUNDLE + i) * SLAB : 0, t, SLAB);
+            }
+        }
+#endif
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+            if constexpr (PAIR) {
+                // CTA-scope release: the operand this publishes stays in this CTA's shared memory and is
+                // read by this CTA's tensor core (after the proxy fence above) once the leader has seen
+                // the arrival and issued the UMMA.  A cluster-scope release here kept a quarter of the
+                // dequantiser warps in membar stalls (ncu) and cost 1-2 %.  The waiter acquires at cluster
+                // scope, so by the letter of the PTX memory model this release/acquire pair does not
+                // synchronise; it is kept because no thread of the other CTA reads what is published (a
+                // bit-for-bit soak of all slab heights against the single-CTA kernel stands in the test
+                // suite).  -DATB_PAIR_RELEASE_CLUSTER builds the conforming form.
+#ifdef ATB_PAIR_RELEASE_CLUSTER
+                mbar_arrive_cluster(mapa_shared(deq_full + 8 * rd.bar, 0));
+#else
+                mbar_arrive_cluster_cta_release(mapa_shared(deq_full + 8 * rd.bar, 0));
+#endif
+            } else {
+#ifdef ATB_TEST_WITHHOLD_DEQ_ARRIVAL
+                // Test build of the timeout path only: the first dequantiser warp of CTA 0 keeps back its very
+                // first arrival, so the issuer's bounded wait for that operand runs out, the CTA aborts, every
+                // role returns and atb_device_status reports it.  No UMMA or copy depends on the missing arrival.
+                if (!(blockIdx.x == 0 && warp == kFirstDequantWarp && n == 0))
+#endif
+                mbar_arrive(deq_full + 8 * rd.bar);
+            }
+#pragma unroll
+            for (int i = 0; i < C::BUNDLE; ++i) mbar_arrive(raw_empty + 8 * (rr.bar + i));
+        }
+        rr.template advance<C::DQ_GROUPS * C::BUNDLE>();
+        rd.template advance<C::DQ_GROUPS>();
+    }
+    (void)warp;
+}
+
+// ---------------------------------------------------------------------------------------------
 // Epilogues of one warp: N_COLS accumulator columns of its 32 TMEM lanes (rows row0 .. row0+31,
 // columns col0 ..) -> C.  `box` is the warp's staging in shared memory.
 // ---------------------------------------------------------------------------------------------

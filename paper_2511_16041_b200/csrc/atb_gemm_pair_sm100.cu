@@ -22,10 +22,12 @@
 
 namespace {
 
-template <int SLAB_ROWS>
+template <int SLAB_ROWS_T>
 struct PairCfg {
+    static constexpr int SLAB_ROWS = SLAB_ROWS_T;              // rows of a raw A slab (T_MA)
     static constexpr int T_K = 64, N_MMA = 256, N_CHUNKS = 2, ROWS = 128;
     static constexpr int SLABS = ROWS / SLAB_ROWS;             // slabs per CTA and K-step
+    static constexpr int GPS = 1;                              // a slab never spans operand groups here
     static constexpr uint32_t B_BOX_BYTES = T_K * 128;         // 64 columns x 64 rows of bf16
     static constexpr uint32_t B_BYTES = 4 * B_BOX_BYTES;       // this CTA's half: 2 chunks x 128 columns
     static constexpr uint32_t GROUP_BYTES = 128 * T_K * 2;
@@ -262,64 +264,8 @@ atb_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_c
         // slabs arrive in ring order: a group takes every DQ_GROUPS-th slab of this CTA's stream
         int64_t my_slabs = 0;
         for (int tile = cluster_id; tile < total_tiles; tile += n_clusters) my_slabs += static_cast<int64_t>(p.k_steps) * C::SLABS;
-        const DequantLane<C> ln(t, SLAB_ROWS);
-#ifdef ATB_PROFILE_SKIP_DEQUANT
-        // diagnostic: the operand ring holds fixed pseudo-random bf16 values (zeros would lower the
-        // tensor cores' power and flatter the clock)
-        for (uint32_t i = threadIdx.x - kFirstDequantWarp * 32; i < C::NG * C::GROUP_BYTES / 4; i += kDequantWarps * 32) {
-            uint32_t h = (i + 1u) * 2654435761u; h ^= h >> 15; h *= 2246822519u; h ^= h >> 13;
-            const uint32_t v = (h & 0x807F807Fu) | 0x3F003F00u;          // +-[0.5, 1) in both halves
-            asm volatile("st.shared.b32 [%0], %1;" ::"r"(deq_base + i * 4), "r"(v) : "memory");
-        }
-        fence_proxy_async_smem();
-#endif
-        Cursor<C::NR, C::LR> rr;
-        Cursor<C::ND, C::LD> rd;
-        rr.start_at(my_group * C::BUNDLE);
-        rd.start_at(my_group);
-        for (int64_t n = static_cast<int64_t>(my_group) * C::BUNDLE; n < my_slabs; n += C::DQ_GROUPS * C::BUNDLE) {
-            bool ok = true;
-#pragma unroll
-            for (int i = 0; i < C::BUNDLE; ++i)        // bars and buffers of a bundle are consecutive
-                ok = ok && wait_bar_cl(cx, raw_full + 8 * (rr.bar + i), rr.phase, 0x301);
-            ok = ok && wait_bar_cl(cx, deq_empty + 8 * rd.freed_bar(), rd.freed_parity(), 0x302);
-            if (!ok) break;
-            const uint32_t dst_base = deq_base + (rd.buf() / C::SPB) * C::GROUP_BYTES;
-            const int row_base0 = (rd.buf() % C::SPB) * C::BUNDLE * SLAB_ROWS;
-#ifndef ATB_PROFILE_SKIP_DEQUANT    // diagnostic: the pipeline without the conversion work (results are wrong)
-            if constexpr (C::BUNDLE > 1 && C::SLOTS % C::GROUP_THREADS == 0 && C::BUNDLE * C::DQ_ITERS <= 4) {
-                dequant_bundle<C, C::BUNDLE>(ln, raw_base + rr.buf() * C::RAW_BYTES, C::RAW_BYTES, C::RAW_MANT_BYTES, scale_lut,
-                                             dst_base, row_base0, t, SLAB_ROWS);
-            } else {
-#pragma unroll
-                for (int i = 0; i < C::BUNDLE; ++i) {
-                    const uint32_t raw = raw_base + (rr.buf() + i) * C::RAW_BYTES;
-                    dequant_slab<C>(ln, raw, raw + C::RAW_MANT_BYTES, scale_lut, dst_base, row_base0 + i * SLAB_ROWS, t, SLAB_ROWS);
-                }
-            }
-#endif
-            fence_proxy_async_smem();
-            __syncwarp();
-            if (lane == 0) {
-                // CTA-scope release: the operand this publishes stays in this CTA's shared memory and is
-                // read by this CTA's tensor core (after the proxy fence above) once the leader has seen
-                // the arrival and issued the UMMA.  A cluster-scope release here kept a quarter of the
-                // dequantiser warps in membar stalls (ncu) and cost 1-2 %.  The waiter acquires at cluster
-                // scope, so by the letter of the PTX memory model this release/acquire pair does not
-                // synchronise; it is kept because no thread of the other CTA reads what is published (a
-                // bit-for-bit soak of all slab heights against the single-CTA kernel stands in the test
-                // suite).  -DATB_PAIR_RELEASE_CLUSTER builds the conforming form.
-#ifdef ATB_PAIR_RELEASE_CLUSTER
-                mbar_arrive_cluster(mapa_shared(deq_full + 8 * rd.bar, 0));
-#else
-                mbar_arrive_cluster_cta_release(mapa_shared(deq_full + 8 * rd.bar, 0));
-#endif
-#pragma unroll
-                for (int i = 0; i < C::BUNDLE; ++i) mbar_arrive(raw_empty + 8 * (rr.bar + i));
-            }
-            rr.template advance<C::DQ_GROUPS * C::BUNDLE>();
-            rd.template advance<C::DQ_GROUPS>();
-        }
+        dequantiser_role<C, true>(cx, t, my_group, warp, lane, my_slabs, raw_full, raw_empty, deq_full, deq_empty, raw_base, deq_base,
+                                  scale_lut);
     }
 
     // ---- teardown: the peer may still arrive on this CTA's barriers until it gets here ----

@@ -34,6 +34,7 @@ __device__ unsigned int g_gemm_error_flag = 0;
 
 template <int T_MA, int T_MC, int T_K, int T_N>
 struct Cfg {
+    static constexpr int SLAB_ROWS = T_MA;
     static constexpr int G = T_MC / 128;                       // 128-row groups per output tile
     static constexpr int RHO = T_MC / T_MA;                    // slabs per K-step
     static constexpr int SPG = (T_MA < 128) ? 128 / T_MA : 1;  // slabs per group
@@ -322,59 +323,8 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
             const WorkItem w = work_item<SPLIT>(item, p);
             my_slabs += static_cast<int64_t>(w.k_end - w.k_begin) * C::KH * C::RHO;
         }
-        const DequantLane<C> ln(t, T_MA);
-#ifdef ATB_PROFILE_SKIP_DEQUANT
-        // diagnostic: the operand ring holds fixed pseudo-random bf16 values (zeros would lower the
-        // tensor cores' power and flatter the clock)
-        for (uint32_t i = threadIdx.x - kFirstDequantWarp * 32; i < C::NG * C::GROUP_BYTES / 4; i += kDequantWarps * 32) {
-            uint32_t h = (i + 1u) * 2654435761u; h ^= h >> 15; h *= 2246822519u; h ^= h >> 13;
-            const uint32_t v = (h & 0x807F807Fu) | 0x3F003F00u;          // +-[0.5, 1) in both halves
-            asm volatile("st.shared.b32 [%0], %1;" ::"r"(deq_base + i * 4), "r"(v) : "memory");
-        }
-        fence_proxy_async_smem();
-#endif
-        Cursor<C::NR, C::LR> rr;
-        Cursor<C::ND, C::LD> rd;
-        rr.start_at(my_group * C::BUNDLE);
-        rd.start_at(my_group);
-        for (int64_t n = static_cast<int64_t>(my_group) * C::BUNDLE; n < my_slabs; n += C::DQ_GROUPS * C::BUNDLE) {
-            bool ok = true;
-#pragma unroll
-            for (int i = 0; i < C::BUNDLE; ++i)        // bars and buffers of a bundle are consecutive
-                ok = ok && wait_bar(cx, raw_full + 8 * (rr.bar + i), rr.phase, 0x301);
-            ok = ok && wait_bar(cx, deq_empty + 8 * rd.freed_bar(), rd.freed_parity(), 0x302);
-            if (!ok) break;
-#ifndef ATB_PROFILE_SKIP_DEQUANT    // diagnostic: the pipeline without the conversion work (results are wrong)
-            // all slots of the bundle in flight at once where that is at most four per thread (registers)
-            if constexpr (C::BUNDLE > 1 && C::SLOTS % C::GROUP_THREADS == 0 && C::BUNDLE * C::DQ_ITERS <= 4) {
-                dequant_bundle<C, C::BUNDLE>(ln, raw_base + rr.buf() * C::RAW_BYTES, C::RAW_BYTES, C::RAW_MANT_BYTES, scale_lut,
-                                             deq_base + (rd.buf() / C::SPB) * C::GROUP_BYTES, (rd.buf() % C::SPB) * C::BUNDLE * T_MA, t, T_MA);
-            } else {
-#pragma unroll
-                for (int i = 0; i < C::BUNDLE; ++i) {
-                    const uint32_t raw = raw_base + (rr.buf() + i) * C::RAW_BYTES;
-                    const uint32_t dst_base = deq_base + (T_MA <= 128 ? rd.buf() / C::SPB : rd.buf() * C::GPS) * C::GROUP_BYTES;
-                    dequant_slab<C>(ln, raw, raw + C::RAW_MANT_BYTES, scale_lut, dst_base,
-                                    T_MA <= 128 ? ((rd.buf() % C::SPB) * C::BUNDLE + i) * T_MA : 0, t, T_MA);
-                }
-            }
-#endif
-            fence_proxy_async_smem();
-            __syncwarp();
-            if (lane == 0) {
-#ifdef ATB_TEST_WITHHOLD_DEQ_ARRIVAL
-                // Test build of the timeout path only: the first dequantiser warp of CTA 0 keeps back its very
-                // first arrival, so the issuer's bounded wait for that operand runs out, the CTA aborts, every
-                // role returns and atb_device_status reports it.  No UMMA or copy depends on the missing arrival.
-                if (!(blockIdx.x == 0 && warp == kFirstDequantWarp && n == 0))
-#endif
-                mbar_arrive(deq_full + 8 * rd.bar);
-#pragma unroll
-                for (int i = 0; i < C::BUNDLE; ++i) mbar_arrive(raw_empty + 8 * (rr.bar + i));
-            }
-            rr.template advance<C::DQ_GROUPS * C::BUNDLE>();
-            rd.template advance<C::DQ_GROUPS>();
-        }
+        dequantiser_role<C, false>(cx, t, my_group, warp, lane, my_slabs, raw_full, raw_empty, deq_full, deq_empty, raw_base, deq_base,
+                                   scale_lut);
     }
 
     // ---- teardown: on the abort path give copies and MMAs in flight time to land first ----
