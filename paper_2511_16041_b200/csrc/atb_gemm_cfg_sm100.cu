@@ -86,6 +86,13 @@ struct CfgK {
     static constexpr int NB = PAIR ? 4 : (A_Q ? 4 : 6), NBR = 4;      // operand / raw units of B
     static constexpr int LB = stream_bars(NB, UB, IPK), LBR = stream_bars(NBR, UB, IPK);
     static constexpr int GROUP_WARPS = 4;
+    // Tile-rows per band of the tile walk (tile_coords): the streamed A is the heavier operand here (BF16 in config 1),
+    // so a wave should cover few row panels and many column panels of the BFP16 B.
+#ifdef ATB_CFG_BAND
+    static constexpr int BAND = ATB_CFG_BAND;
+#else
+    static constexpr int BAND = PAIR ? 4 : 8;
+#endif
     static constexpr uint32_t SMEM_BYTES = 1024u + (NA + NB) * UNIT_BYTES + NAS * SLAB_RAW_BYTES + NBR * RAW_BYTES + 1024u +
                                            4u * kEpilogueBoxBytes + 8u * (2 * LAH + 2 * LAR + 2 * LB + 2 * LBR + 4) + 16u + kScaleTableBytes;
     static_assert(NB % UB == 0 && LB % UB == 0, "B tiles are whole groups of units");
@@ -244,7 +251,7 @@ atb_gemm_cfg_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
             bool ok = true;
             for (int tile = first_tile; ok && tile < total_tiles; tile += tile_step) {
                 int mt, nt;
-                tile_coords(tile, p.m_tiles, p.n_tiles, mt, nt);
+                tile_coords<C::BAND>(tile, p.m_tiles, p.n_tiles, mt, nt);
                 // this CTA's units of the tile: both (single CTA) or unit `rank` (pair)
                 const int n0 = nt * C::T_N + (PAIR ? static_cast<int>(rank) * 128 : 0);
                 for (int k = 0; ok && k < p.k_steps; ++k) {
@@ -269,7 +276,7 @@ atb_gemm_cfg_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
                 Cursor<C::NAS, C::LAR> rr;
                 for (int tile = first_tile; ok && tile < total_tiles; tile += tile_step) {
                     int mt, nt;
-                    tile_coords(tile, p.m_tiles, p.n_tiles, mt, nt);
+                    tile_coords<C::BAND>(tile, p.m_tiles, p.n_tiles, mt, nt);
                     const int row0 = mt * C::T_MC + row_off;
                     for (int k = 0; ok && k < p.k_steps; ++k) {
                         for (int sl = 0; sl < C::RHO; ++sl) {
@@ -290,7 +297,7 @@ atb_gemm_cfg_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
                 Ring ra;
                 for (int tile = first_tile; ok && tile < total_tiles; tile += tile_step) {
                     int mt, nt;
-                    tile_coords(tile, p.m_tiles, p.n_tiles, mt, nt);
+                    tile_coords<C::BAND>(tile, p.m_tiles, p.n_tiles, mt, nt);
                     const int row0 = mt * C::T_MC + row_off;
                     for (int k = 0; ok && k < p.k_steps; ++k) {
                         for (int h = 0; h < C::HA; ++h) {            // hand-overs of this K-step
@@ -365,7 +372,7 @@ atb_gemm_cfg_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
         bool ok = true;
         for (int tile = first_tile; ok && tile < total_tiles; tile += tile_step, acc_phase ^= 1u) {
             int mt, nt;
-            tile_coords(tile, p.m_tiles, p.n_tiles, mt, nt);
+            tile_coords<C::BAND>(tile, p.m_tiles, p.n_tiles, mt, nt);
             for (int g = 0; g < 2; ++g) {
                 if (!(ok = wait_bar_t<false, PAIR>(cx, acc_full + 8 * g, acc_phase, 0x201))) break;
                 tcgen05_fence_after_sync();

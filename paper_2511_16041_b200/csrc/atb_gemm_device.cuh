@@ -311,13 +311,18 @@ __device__ __forceinline__ bool wait_bar_spin(const Ctx& cx, uint32_t bar, uint3
     return wait_bar_t<true, false>(cx, bar, parity, code);
 }
 
+// BAND tile-rows per band: the CTAs of a wave (148 tiles, or 74 pair tiles) cover BAND row panels of the
+// operand on the M side and 148 / BAND column panels of the other; the bytes a wave pulls through the L2 are
+// least where the two sides weigh the same, BAND^2 = units * (bytes of a column panel) / (bytes of a row panel).
+// atb_gemm (BFP16 row panels of 256 rows against BF16 column panels of 256 or 512 columns): 16.
+template <int BAND = 16>
 __device__ __forceinline__ void tile_coords(int tile, int m_tiles, int n_tiles, int& mt, int& nt) {
-    // Bands of 16 tile-rows, column-major inside a band: the CTAs of one wave share a few
+    // Bands of BAND tile-rows, column-major inside a band: the CTAs of one wave share a few
     // A row-panels and B column-panels in L2.
-    const int per_band = 16 * n_tiles;
+    const int per_band = BAND * n_tiles;
     const int band = tile / per_band, i = tile - band * per_band;
-    const int rows = min(16, m_tiles - band * 16);
-    mt = band * 16 + i % rows;
+    const int rows = min(BAND, m_tiles - band * BAND);
+    mt = band * BAND + i % rows;
     nt = i / rows;
     // odd bands walk the columns backwards: they start on the B panels the band before them ended on
     if (band & 1) nt = n_tiles - 1 - nt;
