@@ -94,7 +94,7 @@ struct CfgK {
     static constexpr int BAND = PAIR ? 4 : 8;
 #endif
     static constexpr uint32_t SMEM_BYTES = 1024u + (NA + NB) * UNIT_BYTES + NAS * SLAB_RAW_BYTES + NBR * RAW_BYTES + 1024u +
-                                           4u * kEpilogueBoxBytes + 8u * (2 * LAH + 2 * LAR + 2 * LB + 2 * LBR + 4) + 16u + kScaleTableBytes;
+                                           4u * kEpilogueBoxBytes + 8u * (2 * LAH + 2 * LAR + 2 * LB + 2 * LBR + 4) + 16u;
     static_assert(NB % UB == 0 && LB % UB == 0, "B tiles are whole groups of units");
     static_assert(LAH <= kMaxRingBars && LAR <= kMaxRingBars && LB <= kMaxRingBars && LBR <= kMaxRingBars, "barrier count");
     static_assert(SMEM_BYTES <= kSmemBudget, "shared memory");
@@ -130,7 +130,7 @@ struct RingPos {
 template <int ROWS, int NRS, int LR, int NDH, int LD, bool PAIR>
 __device__ __forceinline__ bool dequant_job(const Ctx& cx, int64_t x, int t, int lane, uint32_t raw_full, uint32_t raw_empty,
                                             uint32_t deq_full, uint32_t deq_empty, uint32_t raw_base, uint32_t deq_base,
-                                            uint32_t scale_lut, unsigned code) {
+                                            unsigned code) {
     using Dq = CfgDq<ROWS>;
     constexpr int SPG = ROWS < 128 ? 128 / ROWS : 1, GPS = ROWS > 128 ? ROWS / 128 : 1;
     constexpr uint32_t kMant = ROWS * 64, kRaw = kMant + ROWS * 8;
@@ -144,12 +144,12 @@ __device__ __forceinline__ bool dequant_job(const Ctx& cx, int64_t x, int t, int
     if (!ok) return false;
     const uint32_t dst = deq_base + rd.buf * GPS * Dq::GROUP_BYTES;
     if constexpr (SPG > 1 && SPG * Dq::DQ_ITERS <= 4) {
-        dequant_bundle<Dq, SPG>(ln, raw_base + rr.buf * SPG * kRaw, kRaw, kMant, scale_lut, dst, 0, t, ROWS);
+        dequant_bundle<Dq, SPG>(ln, raw_base + rr.buf * SPG * kRaw, kRaw, kMant, dst, 0, t, ROWS);
     } else {
 #pragma unroll
         for (int i = 0; i < SPG; ++i) {
             const uint32_t raw = raw_base + (rr.buf * SPG + i) * kRaw;
-            dequant_slab<Dq>(ln, raw, raw + kMant, scale_lut, dst, i * ROWS, t, ROWS);
+            dequant_slab<Dq>(ln, raw, raw + kMant, dst, i * ROWS, t, ROWS);
         }
     }
     fence_proxy_async_smem();
@@ -201,7 +201,6 @@ atb_gemm_cfg_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
     const uint32_t br_full = b_empty + 8 * C::LB, br_empty = br_full + 8 * C::LBR;
     const uint32_t acc_full = br_empty + 8 * C::LBR, acc_empty = acc_full + 8 * 2;
     const uint32_t misc = acc_empty + 8 * 2;                 // [0]: TMEM base, [1]: abort flag
-    const uint32_t scale_lut = misc + 16;
     volatile uint32_t* const misc_gen = reinterpret_cast<volatile uint32_t*>(smem_gen + (misc - smem_base));
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -228,10 +227,6 @@ atb_gemm_cfg_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
     if (warp == 1) {
         if constexpr (PAIR) { tmem_alloc_pair(misc, 512u); tmem_relinquish_pair(); }
         else { tmem_alloc(misc, 512u); tmem_relinquish(); }
-    }
-    if (threadIdx.x >= kFirstDequantWarp * 32 && threadIdx.x < kFirstDequantWarp * 32 + 256) {
-        const uint32_t E = threadIdx.x - kFirstDequantWarp * 32;
-        store_scale_table_entry(scale_lut, E);
     }
     tcgen05_fence_before_sync();
     __syncthreads();
@@ -407,10 +402,10 @@ atb_gemm_cfg_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
             if (A_Q && j < C::JA) {
                 if constexpr (A_Q)
                     ok = dequant_job<T_MA, C::NAS, C::LAR, C::NAH, C::LAH, PAIR>(cx, ks * C::HA + j, t, lane, ar_full, ar_empty, a_full, a_empty,
-                                                                                 a_raw_base, a_base, scale_lut, 0x300);
+                                                                                 a_raw_base, a_base, 0x300);
             } else {
                 ok = dequant_job<128, C::NBR, C::LBR, C::NB, C::LB, PAIR>(cx, ks * C::UB + (j - C::JA), t, lane, br_full, br_empty, b_full, b_empty,
-                                                                          b_raw_base, b_base, scale_lut, 0x310);
+                                                                          b_raw_base, b_base, 0x310);
             }
             if (!ok) break;
         }

@@ -46,7 +46,6 @@ constexpr uint32_t kEpilogueBoxBytes = 32 * 128;   // 32 rows x 64 bf16 columns
 // for them, and in half-size boxes under 32-row slabs, whose deeper raw ring needs the space.
 constexpr int pair_box_cols(int slab) { return slab >= 64 ? 64 : 32; }
 constexpr uint32_t pair_box_bytes(int slab) { return 32u * pair_box_cols(slab) * 2u; }
-constexpr uint32_t kScaleTableBytes = 256u * 8u;  // per exponent: the scale and its offset, see scale_table_entry
 constexpr uint32_t kSmemBudget = 232448;          // 227 KB of dynamic shared memory per CTA
 #ifdef ATB_TEST_WAIT_NS                             // test build of the timeout path only: a short limit
 constexpr uint64_t kWaitTimeoutNs = ATB_TEST_WAIT_NS;
@@ -78,7 +77,7 @@ struct RingPlan {
 
 constexpr uint32_t ring_smem_bytes(uint32_t b_bytes, uint32_t group_bytes, uint32_t raw_bytes, int acc_bars,
                                    int dqg, int bundle, int b, int g, int n_deq, int r, uint32_t box_bytes = kEpilogueBoxBytes) {
-    const uint32_t bars = 8u * (2 * b + 2 * ring_bars(r, dqg * bundle) + 2 * ring_bars(n_deq, dqg) + 2 * acc_bars) + 16u + kScaleTableBytes;
+    const uint32_t bars = 8u * (2 * b + 2 * ring_bars(r, dqg * bundle) + 2 * ring_bars(n_deq, dqg) + 2 * acc_bars) + 16u;
     return 1024u + b * b_bytes + g * group_bytes + r * raw_bytes + 1024u + 4u * box_bytes + bars;
 }
 
@@ -375,66 +374,64 @@ __device__ __forceinline__ WorkItem work_item(int item, const GemmParams& p) {
 //      (0x64uu = 1024 + u); subtracting 1024 (add.f16x2) normalises them: u as fp16, exact.
 //   2. u is positive and non-zero, so fp16 -> bf16 is pure bit arithmetic: drop 3 mantissa bits
 //      (they are zero: u has at most 8 significant bits) and re-bias the exponent by 112 -
-//      (h >> 3) + 0x3800 per half, done for both halves by one mad.hi.u32 (x * 2^29 >> 32).
-//   3. one fma.rn.bf16x2 forms u * s - 128 * s = m * 2^(E-133) with s = 2^(E-133) and -128 * s from
-//      the block's table entry: both products are exact and so is the result (7 significant bits),
-//      bf16-subnormal results included (s is bf16-subnormal for E < 7; no flush to zero).
-// -128 * s is not a bf16 number for E >= 254: a thread that met such a block converts its slots of
-// the slab once more in the two-step form, add.bf16x2 (u - 128, exact) then mul.bf16x2 by s.
+//      (h >> 3) + 0x3800 per half, done for both halves by one mad.hi.u32 (x * 2^29 >> 32).  Re-biasing
+//      by 6 more gives u / 64 instead of u.
+//   3. one fma.rn.bf16x2 forms (u / 64) * s' - 2 s' = m * 2^(E-133) with s' = 2^(E-127): both products are
+//      exact and so is the result (7 significant bits), bf16-subnormal results included (no flush to zero).
+// The scales need no table: the exponent byte of a block IS the UE8M0 number 2^(E-127), so one
+// cvt.rn.bf16x2.ue8m0x2 turns the two exponent bytes of a slot into the two scales s', a prmt each copies
+// them into both halves, and -2 s' is one bf16x2 multiplication (exact, subnormal s' for E = 0 included).
+// (An earlier version read s = 2^(E-133) and -128 s from a 256-entry table in shared memory: two 8-byte
+// loads per slot, a quarter of the dequantisers' shared-memory wavefronts; without them the single-CTA
+// tilings gained 1-3 %.)
+// -2 s' is not a bf16 number for E >= 254: a thread that met such a block converts its slots of the slab
+// once more in the two-step form, add.bf16x2 (u - 128, exact) then mul.bf16x2 by s = 2^(E-133).
 // Only the prmt runs on the integer ALU pipe; the other operations go to the FMA pipe.
+template <uint32_t kRebias>
 __device__ __forceinline__ uint32_t bf16x2_of_bytes(uint32_t u, uint32_t selector) {
     const uint32_t h2 = __byte_perm(u, 0x64646464u, selector);
     uint32_t t, b;
     asm("add.rn.f16x2 %0, %1, %2;" : "=r"(t) : "r"(h2), "r"(0xE400E400u));          // - 1024
-    asm("mad.hi.u32 %0, %1, %2, %3;" : "=r"(b) : "r"(t), "r"(0x20000000u), "r"(0x38003800u));
+    asm("mad.hi.u32 %0, %1, %2, %3;" : "=r"(b) : "r"(t), "r"(0x20000000u), "r"(kRebias));
     return b;
 }
 __device__ __forceinline__ uint32_t dequant_pair(uint32_t u, uint32_t selector, uint32_t scale2, uint32_t offset2) {
     uint32_t r;
-    asm("fma.rn.bf16x2 %0, %1, %2, %3;" : "=r"(r) : "r"(bf16x2_of_bytes(u, selector)), "r"(scale2), "r"(offset2));
+    asm("fma.rn.bf16x2 %0, %1, %2, %3;" : "=r"(r) : "r"(bf16x2_of_bytes<0x35003500u>(u, selector)), "r"(scale2), "r"(offset2));
     return r;
 }
 __device__ __forceinline__ uint32_t dequant_pair_two_step(uint32_t u, uint32_t selector, uint32_t scale2) {
     uint32_t d, r;
-    asm("add.rn.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(bf16x2_of_bytes(u, selector)), "r"(0xC300C300u));   // - 128
+    asm("add.rn.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(bf16x2_of_bytes<0x38003800u>(u, selector)), "r"(0xC300C300u));   // - 128
     asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(d), "r"(scale2));
     return r;
 }
-
-// Table entry for exponent E, 8 bytes: s = 2^(E-133) as bf16 in both halves of the first word,
-// -128 * s = -2^(E-126) in both halves of the second.  For E >= 254 that number does not exist and
-// the second word is 0: the only entries with bit 31 clear.  (The quantiser never writes E = 255;
-// planes from elsewhere that hold it get m * 2^122 like any other block, +-Inf beyond bf16.)
-__device__ __forceinline__ uint2 scale_table_entry(uint32_t E) {
-    const uint32_t bits = (E >= 7u) ? ((E - 6u) << 7) : (1u << E);
-    uint2 e;
-    e.x = bits * 0x10001u;
-    e.y = E >= 254u ? 0u : (0x8000u | ((E + 1u) << 7)) * 0x10001u;
-    return e;
-}
-__device__ __forceinline__ void store_scale_table_entry(uint32_t scale_lut, uint32_t E) {
-    const uint2 e = scale_table_entry(E);
-    asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(scale_lut + E * 8), "r"(e.x), "r"(e.y) : "memory");
+// s = 2^(E-133) as bf16 in both halves of a word (bf16-subnormal for E < 7).  (E = 255, which the quantiser
+// never writes, gives m * 2^122 like any other block - +-Inf beyond bf16.)
+__device__ __forceinline__ uint32_t scale_bits(uint32_t E) {
+    return ((E >= 7u) ? ((E - 6u) << 7) : (1u << E)) * 0x10001u;
 }
 
 // N slots of one thread: 16 mantissa bytes each (w, two's complement) of two blocks with exponents
 // (e & 0xFF, e >> 8) -> two 16-byte stores of bf16 values per slot (addresses st0[i], st1[i]).
-// FAST: the one-fma form; returns the AND of the offsets used, whose bit 31 is clear when a block
-// had E >= 254 - the caller then converts again in the two-step form (FAST = false) before it hands
-// the operand on.  The test stays off the conversion's dependency chain that way.
+// FAST: the one-fma form; returns a word whose bit 31 is clear when a block had E >= 254 - the caller then
+// converts again in the two-step form (FAST = false) before it hands the operand on.  The test stays off
+// the conversion's dependency chain that way.
 template <int N, bool FAST>
-__device__ __forceinline__ uint32_t dequant_slots(const uint4 (&w)[N], const uint32_t (&e)[N], uint32_t scale_lut,
+__device__ __forceinline__ uint32_t dequant_slots(const uint4 (&w)[N], const uint32_t (&e)[N],
                                                   const uint32_t (&st0)[N], const uint32_t (&st1)[N]) {
-    uint32_t all = 0xFFFFFFFFu;
+    uint32_t mx = 0u;                            // largest 2^(E-127) met, per half
 #pragma unroll
     for (int i = 0; i < N; ++i) {
-        uint32_t s0, c0, s1, c1;
-        asm volatile("ld.shared.v2.b32 {%0, %1}, [%2];" : "=r"(s0), "=r"(c0) : "r"(scale_lut + (e[i] & 0xFFu) * 8));
-        asm volatile("ld.shared.v2.b32 {%0, %1}, [%2];" : "=r"(s1), "=r"(c1) : "r"(scale_lut + (e[i] >> 8) * 8));
-        all &= c0 & c1;
         const uint32_t u0 = w[i].x ^ 0x80808080u, u1 = w[i].y ^ 0x80808080u;
         const uint32_t u2 = w[i].z ^ 0x80808080u, u3 = w[i].w ^ 0x80808080u;
         if constexpr (FAST) {
+            uint32_t sp, c0, c1;
+            asm("cvt.rn.bf16x2.ue8m0x2 %0, %1;" : "=r"(sp) : "h"(static_cast<uint16_t>(e[i])));
+            asm("max.u16x2 %0, %1, %2;" : "=r"(mx) : "r"(mx), "r"(sp));
+            const uint32_t s0 = __byte_perm(sp, 0, 0x1010), s1 = __byte_perm(sp, 0, 0x3232);
+            asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(c0) : "r"(s0), "r"(0xC000C000u));       // -2 s'
+            asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(c1) : "r"(s1), "r"(0xC000C000u));
             asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(st0[i]),
                          "r"(dequant_pair(u0, 0x4140u, s0, c0)), "r"(dequant_pair(u0, 0x4342u, s0, c0)),
                          "r"(dequant_pair(u1, 0x4140u, s0, c0)), "r"(dequant_pair(u1, 0x4342u, s0, c0))
@@ -444,6 +441,7 @@ __device__ __forceinline__ uint32_t dequant_slots(const uint4 (&w)[N], const uin
                          "r"(dequant_pair(u3, 0x4140u, s1, c1)), "r"(dequant_pair(u3, 0x4342u, s1, c1))
                          : "memory");
         } else {
+            const uint32_t s0 = scale_bits(e[i] & 0xFFu), s1 = scale_bits(e[i] >> 8);
             asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(st0[i]),
                          "r"(dequant_pair_two_step(u0, 0x4140u, s0)), "r"(dequant_pair_two_step(u0, 0x4342u, s0)),
                          "r"(dequant_pair_two_step(u1, 0x4140u, s0)), "r"(dequant_pair_two_step(u1, 0x4342u, s0))
@@ -454,7 +452,8 @@ __device__ __forceinline__ uint32_t dequant_slots(const uint4 (&w)[N], const uin
                          : "memory");
         }
     }
-    return all;
+    // a block with E >= 254 has s' >= 2^127 = 0x7F00 as bf16, whose double is not a bf16 number
+    return ((mx + 0x01000100u) & 0x80008000u) ? 0u : 0xFFFFFFFFu;
 }
 
 // Per-thread constants of the dequantiser: thread t of a group owns slot t (16 mantissas = blocks
@@ -477,7 +476,7 @@ struct DequantLane {
 // Dequantises one slab: raw mantissas / exponents in shared memory -> bf16 operand rows starting at
 // row `row_base` (a multiple of 32) of the 128-row groups at dst_base.
 template <class C, bool FAST = true>
-__device__ __forceinline__ void dequant_slab(const DequantLane<C>& ln, uint32_t raw_mant, uint32_t raw_exp, uint32_t scale_lut,
+__device__ __forceinline__ void dequant_slab(const DequantLane<C>& ln, uint32_t raw_mant, uint32_t raw_exp,
                                              uint32_t dst_base, int row_base, int t, int T_MA_rows) {
     static_assert(C::ROWS_PER_ITER % 8 == 0 && 128 % C::ROWS_PER_ITER == 0, "band height");
     const uint32_t ld = raw_mant + ln.ld_off, le = raw_exp + ln.exp_off;
@@ -513,7 +512,7 @@ __device__ __forceinline__ void dequant_slab(const DequantLane<C>& ln, uint32_t 
                 const uint32_t band = static_cast<uint32_t>((i * kBandRows) >> 7) * C::GROUP_BYTES + static_cast<uint32_t>((i * kBandRows) & 127) * 128u;
                 wc[j] = w[i]; ec[j] = e[i]; a0[j] = st0 + band; a1[j] = st1 + band;
             }
-            all &= dequant_slots<CHUNK, FAST>(wc, ec, scale_lut, a0, a1);
+            all &= dequant_slots<CHUNK, FAST>(wc, ec, a0, a1);
         }
     } else {
 #pragma unroll
@@ -522,13 +521,13 @@ __device__ __forceinline__ void dequant_slab(const DequantLane<C>& ln, uint32_t 
                 const uint32_t band = static_cast<uint32_t>((i * kBandRows) >> 7) * C::GROUP_BYTES + static_cast<uint32_t>((i * kBandRows) & 127) * 128u;
                 const uint4 wc[1] = {w[i]};
                 const uint32_t ec[1] = {e[i]}, a0[1] = {st0 + band}, a1[1] = {st1 + band};
-                all &= dequant_slots<1, FAST>(wc, ec, scale_lut, a0, a1);
+                all &= dequant_slots<1, FAST>(wc, ec, a0, a1);
             }
         }
     }
     if constexpr (FAST) {
         if (static_cast<int32_t>(all) >= 0)              // a block with E >= 254: rare
-            dequant_slab<C, false>(ln, raw_mant, raw_exp, scale_lut, dst_base, row_base, t, T_MA_rows);
+            dequant_slab<C, false>(ln, raw_mant, raw_exp, dst_base, row_base, t, T_MA_rows);
     }
 }
 
@@ -537,7 +536,7 @@ __device__ __forceinline__ void dequant_slab(const DequantLane<C>& ln, uint32_t 
 // NS * DQ_ITERS slots in flight exactly as with one 128-row slab.
 template <class C, int NS, bool FAST = true>
 __device__ __forceinline__ void dequant_bundle(const DequantLane<C>& ln, uint32_t raw0, uint32_t raw_stride, uint32_t mant_bytes,
-                                               uint32_t scale_lut, uint32_t dst_base, int row_base0, int t, int slab_rows) {
+                                               uint32_t dst_base, int row_base0, int t, int slab_rows) {
     static_assert(C::SLOTS % C::GROUP_THREADS == 0, "whole iterations");
     const int r0 = t / C::SLOTS_PER_ROW;
     (void)r0;
@@ -571,10 +570,10 @@ __device__ __forceinline__ void dequant_bundle(const DequantLane<C>& ln, uint32_
             a0[s * C::DQ_ITERS + i] = st0 + band; a1[s * C::DQ_ITERS + i] = st1 + band;
         }
     }
-    const uint32_t all = dequant_slots<N, FAST>(wc, ec, scale_lut, a0, a1);
+    const uint32_t all = dequant_slots<N, FAST>(wc, ec, a0, a1);
     if constexpr (FAST) {
         if (static_cast<int32_t>(all) >= 0)              // a block with E >= 254: rare
-            dequant_bundle<C, NS, false>(ln, raw0, raw_stride, mant_bytes, scale_lut, dst_base, row_base0, t, slab_rows);
+            dequant_bundle<C, NS, false>(ln, raw0, raw_stride, mant_bytes, dst_base, row_base0, t, slab_rows);
     }
 }
 
@@ -589,7 +588,7 @@ __device__ __forceinline__ void dequant_bundle(const DequantLane<C>& ln, uint32_
 template <class C, bool PAIR>
 __device__ __forceinline__ void dequantiser_role(const Ctx& cx, int t, int my_group, int warp, int lane, int64_t my_slabs,
                                                  uint32_t raw_full, uint32_t raw_empty, uint32_t deq_full, uint32_t deq_empty,
-                                                 uint32_t raw_base, uint32_t deq_base, uint32_t scale_lut) {
+                                                 uint32_t raw_base, uint32_t deq_base) {
     constexpr int SLAB = C::SLAB_ROWS;
     const DequantLane<C> ln(t, SLAB);
 #ifdef ATB_PROFILE_SKIP_DEQUANT
@@ -616,14 +615,14 @@ __device__ __forceinline__ void dequantiser_role(const Ctx& cx, int t, int my_gr
 #ifndef ATB_PROFILE_SKIP_DEQUANT    // diagnostic: the pipeline without the conversion work (results are wrong)
         // all slots of the bundle in flight at once where that is at most four per thread (registers)
         if constexpr (C::BUNDLE > 1 && C::SLOTS % C::GROUP_THREADS == 0 && C::BUNDLE * C::DQ_ITERS <= 4) {
-            dequant_bundle<C, C::BUNDLE>(ln, raw_base + rr.buf() * C::RAW_BYTES, C::RAW_BYTES, C::RAW_MANT_BYTES, scale_lut,
+            dequant_bundle<C, C::BUNDLE>(ln, raw_base + rr.buf() * C::RAW_BYTES, C::RAW_BYTES, C::RAW_MANT_BYTES,
                                          deq_base + (rd.buf() / C::SPB) * C::GROUP_BYTES, (rd.buf() % C::SPB) * C::BUNDLE * SLAB, t, SLAB);
         } else {
 #pragma unroll
             for (int i = 0; i < C::BUNDLE; ++i) {
                 const uint32_t raw = raw_base + (rr.buf() + i) * C::RAW_BYTES;
                 const uint32_t dst_base = deq_base + (SLAB <= 128 ? rd.buf() / C::SPB : rd.buf() * C::GPS) * C::GROUP_BYTES;
-                dequant_slab<C>(ln, raw, raw + C::RAW_MANT_BYTES, scale_lut, dst_base,
+                dequant_slab<C>(ln, raw, raw + C::RAW_MANT_BYTES, dst_base,
                                 SLAB <= 128 ? ((rd.buf() % C::SPB) * C::BUNDLE + i) * SLAB : 0, t, SLAB);
             }
         }

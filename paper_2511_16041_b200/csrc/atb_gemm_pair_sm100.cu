@@ -95,7 +95,6 @@ atb_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_c
     const uint32_t deq_full = raw_empty + 8 * C::LR, deq_empty = deq_full + 8 * C::LD;
     const uint32_t acc_full = deq_empty + 8 * C::LD, acc_empty = acc_full + 8 * C::N_CHUNKS;
     const uint32_t misc = acc_empty + 8 * C::N_CHUNKS;       // [0]: TMEM base, [1]: abort flag
-    const uint32_t scale_lut = misc + 16;
     volatile uint32_t* const misc_gen = reinterpret_cast<volatile uint32_t*>(smem_gen + (misc - smem_base));
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -120,10 +119,6 @@ atb_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_c
     if (warp == 1) {
         tmem_alloc_pair(misc, 512u);
         tmem_relinquish_pair();
-    }
-    if (threadIdx.x >= kFirstDequantWarp * 32 && threadIdx.x < kFirstDequantWarp * 32 + 256) {
-        const uint32_t E = threadIdx.x - kFirstDequantWarp * 32;
-        store_scale_table_entry(scale_lut, E);
     }
     tcgen05_fence_before_sync();
     __syncthreads();
@@ -264,8 +259,7 @@ atb_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_c
         // slabs arrive in ring order: a group takes every DQ_GROUPS-th slab of this CTA's stream
         int64_t my_slabs = 0;
         for (int tile = cluster_id; tile < total_tiles; tile += n_clusters) my_slabs += static_cast<int64_t>(p.k_steps) * C::SLABS;
-        dequantiser_role<C, true>(cx, t, my_group, warp, lane, my_slabs, raw_full, raw_empty, deq_full, deq_empty, raw_base, deq_base,
-                                  scale_lut);
+        dequantiser_role<C, true>(cx, t, my_group, warp, lane, my_slabs, raw_full, raw_empty, deq_full, deq_empty, raw_base, deq_base);
     }
 
     // ---- teardown: the peer may still arrive on this CTA's barriers until it gets here ----

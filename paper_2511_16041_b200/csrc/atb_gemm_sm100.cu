@@ -108,7 +108,6 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
     const uint32_t deq_full = raw_empty + 8 * C::LR, deq_empty = deq_full + 8 * C::LD;
     const uint32_t acc_full = deq_empty + 8 * C::LD, acc_empty = acc_full + 8 * n_acc;
     const uint32_t misc = acc_empty + 8 * n_acc;             // [0]: TMEM base, [1]: abort flag
-    const uint32_t scale_lut = misc + 16;                    // 256 entries of 8 bytes, see scale_table_entry
     volatile uint32_t* const misc_gen = reinterpret_cast<volatile uint32_t*>(smem_gen + (misc - smem_base));
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -129,10 +128,6 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
     if (warp == 1) {
         tmem_alloc(misc, static_cast<uint32_t>(C::TMEM_COLS));
         tmem_relinquish();
-    }
-    if (threadIdx.x >= kFirstDequantWarp * 32 && threadIdx.x < kFirstDequantWarp * 32 + 256) {
-        const uint32_t E = threadIdx.x - kFirstDequantWarp * 32;
-        store_scale_table_entry(scale_lut, E);
     }
     tcgen05_fence_before_sync();
     __syncthreads();
@@ -323,8 +318,7 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
             const WorkItem w = work_item<SPLIT>(item, p);
             my_slabs += static_cast<int64_t>(w.k_end - w.k_begin) * C::KH * C::RHO;
         }
-        dequantiser_role<C, false>(cx, t, my_group, warp, lane, my_slabs, raw_full, raw_empty, deq_full, deq_empty, raw_base, deq_base,
-                                   scale_lut);
+        dequantiser_role<C, false>(cx, t, my_group, warp, lane, my_slabs, raw_full, raw_empty, deq_full, deq_empty, raw_base, deq_base);
     }
 
     // ---- teardown: on the abort path give copies and MMAs in flight time to land first ----
