@@ -32,7 +32,7 @@
 //   warp 1      UMMA issuer (the leader CTA's, on a pair): 128 (256) x 256 x 16, both operands K-major
 //   warps 2-5   epilogue (BF16 or quantising BFP16, shared with atb_gemm_kernel)
 //   warps 6-21  dequantisers: 4 groups of 4 warps.  The conversion jobs of a K-step - the hand-overs of
-//               A (config 2) followed by this CTA's units of B - form one sequence that the groups take
+//               B that this CTA converts, then the hand-overs of A (config 2) - form one sequence that the groups take
 //               in turn, so the work is spread evenly whatever the mix is.
 // Barriers, bounded waits and the ring cursors are those of atb_gemm_kernel.
 #include "atb_gemm_device.cuh"
@@ -83,6 +83,7 @@ struct CfgK {
     static constexpr int LAR = A_Q ? SPG * stream_bars(NAS / SPG, HA, IPK) : 0;   // ... of the raw A ring (bundles of SPG slabs)
     // A converted B tile is held for a whole K-step, by both row groups: three K-steps of tiles where
     // shared memory allows, two otherwise.
+    // (config 2 on the pair: six units of A with three or two of B measured 6 % slower than four and four)
     static constexpr int NB = PAIR ? 4 : (A_Q ? 4 : 6), NBR = 4;      // operand / raw units of B
     static constexpr int LB = stream_bars(NB, UB, IPK), LBR = stream_bars(NBR, UB, IPK);
     static constexpr int GROUP_WARPS = 4;
@@ -388,9 +389,10 @@ atb_gemm_cfg_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
         if (lane == 0) tma_store_wait_all<0>();
     } else {
         // ================================ dequantisers ================================
-        // The conversion jobs of this CTA in order: per K-step the JA hand-overs of A (config 2), then the UB
-        // units of B.  Group g takes jobs g, g + 4, g + 8, ...; the rings' barrier counts (stream_bars) make
-        // every barrier the business of one group.
+        // The conversion jobs of this CTA in the order the UMMA issuer asks for their results: per K-step the UB
+        // units of B (the issuer waits for the B tile first), then the JA hand-overs of A (config 2).  Group g
+        // takes jobs g, g + 4, g + 8, ...; the rings' barrier counts (stream_bars) make every barrier the business
+        // of one group.
         const int group = (threadIdx.x - kFirstDequantWarp * 32) / 128, t = (threadIdx.x - kFirstDequantWarp * 32) % 128;
         int64_t k_steps_total = 0;                    // K-steps over this CTA's tiles
         for (int tile = first_tile; tile < total_tiles; tile += tile_step) k_steps_total += p.k_steps;
@@ -399,12 +401,12 @@ atb_gemm_cfg_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
             const int64_t ks = n / C::IPK;
             const int j = static_cast<int>(n - ks * C::IPK);
             bool ok = true;
-            if (A_Q && j < C::JA) {
+            if (A_Q && j >= C::UB) {
                 if constexpr (A_Q)
-                    ok = dequant_job<T_MA, C::NAS, C::LAR, C::NAH, C::LAH, PAIR>(cx, ks * C::HA + j, t, lane, ar_full, ar_empty, a_full, a_empty,
-                                                                                 a_raw_base, a_base, 0x300);
+                    ok = dequant_job<T_MA, C::NAS, C::LAR, C::NAH, C::LAH, PAIR>(cx, ks * C::HA + (j - C::UB), t, lane, ar_full, ar_empty, a_full,
+                                                                                 a_empty, a_raw_base, a_base, 0x300);
             } else {
-                ok = dequant_job<128, C::NBR, C::LBR, C::NB, C::LB, PAIR>(cx, ks * C::UB + (j - C::JA), t, lane, br_full, br_empty, b_full, b_empty,
+                ok = dequant_job<128, C::NBR, C::LBR, C::NB, C::LB, PAIR>(cx, ks * C::UB + j, t, lane, br_full, br_empty, b_full, b_empty,
                                                                           b_raw_base, b_base, 0x310);
             }
             if (!ok) break;
@@ -560,3 +562,8 @@ unsigned int take_cfg_error_flag() {
     return flag;
 }
 }  // namespace atb
+
+#ifdef ATB_PROFILE
+// Diagnostic build only: wait-cycle counters of the configuration kernels (16 values), read and cleared.
+extern "C" int atb_debug_read_wait_cycles_cfg(unsigned long long* out16) { return read_wait_cycles(out16); }
+#endif
