@@ -1,6 +1,8 @@
 // atb_gemm: C = dequant(A_bfp16) x B_bf16 with asymmetric tile buffering (Section 3), sm_100a.
 //
-// One persistent CTA per SM walks output tiles of T_MC x T_N.  Per K-step (output-stationary
+// One persistent CTA per SM walks output tiles of T_MC x T_N (bands of 16 tile rows, odd bands with the
+// columns backwards, K upwards in one tile and downwards in the next: tile_coords, serpentine_k - each
+// wave of tiles starts on what the wave before it left in the L2).  Per K-step (output-stationary
 // schedule of Section 3.1) the T_K x T_N tile of B is brought into shared memory ONCE and
 // rho = T_MC / T_MA slabs of A are streamed through it; the FP32 accumulator of the whole
 // T_MC x T_N tile lives in tensor memory and is written out once, after K / T_K steps.
