@@ -210,6 +210,29 @@ def test_leading_dimensions_and_untouched_padding():
     assert torch.all(Cfull[:, N:] == -5.0)
 
 
+def test_leading_dimensions_ragged_edges_every_epilogue():
+    """The two ways C leaves a kernel - TMA stores clipped by the tensor map (single-CTA tilings, the CTA pair
+    under 32-row slabs) and plain 16-byte stores guarded row by row and chunk by chunk (the CTA pair under
+    64- and 128-row slabs) - on a shape whose last tiles are ragged in M and N (N ends 8 columns into a
+    64-column box), with ldb > N and ldc > N: C is right, and not a byte of the padding is touched."""
+    M, N, K = 300, 584, 192
+    A = inputs.make_A("normal", M, K)
+    Bb = inputs.make_B_bits(K, N)
+    mant, exp = oracle.quantize_bfp16(A)
+    md, ed = planes_to_dev(mant, exp)
+    Cr, S = oracle.gemm(mant, exp, Bb)
+    ldb, ldc = 600, 640
+    Bfull = torch.full((K, ldb), 3.0, dtype=torch.bfloat16, device=dev())          # padding must not leak into C
+    Bfull[:, :N] = bf16_bits_to_dev(Bb)
+    for t in [(128, 256, 64, 256), (128, 256, 64, 512), (64, 256, 64, 512), (32, 256, 64, 512), (128, 128, 64, 128)]:
+        Cfull = torch.full((M + 3, ldc), -5.0, dtype=torch.bfloat16, device=dev())  # three guard rows below C
+        atb.atb_gemm(M, N, K, *t, md, ed, Bfull, Cfull, ldb=ldb, ldc=ldc)
+        atb.atb_device_status()
+        bad, ratio = oracle.check_tolerance(bf16_dev_to_bits(Cfull[:M, :N].contiguous()), Cr, S)
+        assert bad == 0 and ratio < 0.75, (t, bad, ratio)
+        assert torch.all(Cfull[:M, N:] == -5.0) and torch.all(Cfull[M:] == -5.0), t
+
+
 def test_tiny_and_degenerate_shapes():
     for (M, N, K) in [(1, 8, 64), (7, 24, 64), (129, 72, 192), (5, 16, 16), (130, 264, 80), (300, 40, 464)]:
         A = inputs.make_A("normal", M, K)
