@@ -41,11 +41,12 @@ DEFAULT_WORKLOAD = "cfg3_8192"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 NOMINAL_BF16_TFLOPS = 2250.0        # NVIDIA's dense BF16 figure for B200 (context beside the measured peak)
 # The asymmetric-buffering ablation: for fixed (T_MC, T_K, T_N) only T_MA moves, the first entry of
-# each family is its symmetric form.  On the CTA pair each SM holds 128 rows of the 256-row tile, so
-# T_MA = 128 is symmetric there.
+# each family is its symmetric form.  On the CTA pair each SM holds 128 rows of the 256-row tile (or its
+# own 128 x 256 tile of a stacked pair of tiles), so T_MA = 128 is symmetric there.
 ABLATION_FAMILIES = {
     "single_cta_256x256": [(256, 256, 64, 256), (128, 256, 64, 256), (64, 256, 64, 256), (32, 256, 64, 256)],
     "cta_pair_256x512": [(128, 256, 64, 512), (64, 256, 64, 512), (32, 256, 64, 512)],
+    "cta_pair_stacked_128x256": [(128, 128, 128, 256), (64, 128, 128, 256), (32, 128, 128, 256)],
 }
 SUSTAINED_SECONDS = 2.2
 
@@ -449,8 +450,10 @@ def run_ours(args):
         value = aggregate_tflops(flops, world, ms_per_step)
         achieved = flops / (gemm_ms * 1e-3) / 1e12
         T_MA, T_MC, T_K, T_N = tiling_used[0]
-        # T_MC = 256, T_K = 64, T_N = 512 is the tiling that runs on a CTA pair, a kernel of its own
-        gemm_kernel = "atb_gemm_pair_kernel" if (T_MC, T_K, T_N) == (256, 64, 512) else "atb_gemm_kernel"
+        # T_MC = 256, T_K = 64, T_N = 512 runs on a CTA pair, a kernel of its own, and so does T_MC = 128, T_K = 128,
+        # T_N = 256 on more than one tile row (two stacked tiles per pair)
+        stacked = (T_MC, T_K, T_N) == (128, 128, 256) and M > 128
+        gemm_kernel = "atb_gemm_pair_kernel" if (T_MC, T_K, T_N) == (256, 64, 512) or stacked else "atb_gemm_kernel"
         line = {
             "metric": METRIC, "value": value, "unit": "TFLOPS", "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
@@ -460,8 +463,10 @@ def run_ours(args):
                        "tiling": {"T_MA": T_MA, "T_MC": T_MC, "T_K": T_K, "T_N": T_N,
                                   "chosen_by": "flag" if args.tiling else "atb_select_tiling",
                                   "rho_per_core": rho_per_core((T_MA, T_MC, T_K, T_N)),
-                                  "note": ("CTA-pair tiling: each SM holds 128 of the 256 rows, so T_MA = 128 buffers "
-                                           "symmetrically per SM and the B tile is shared by two SMs (Eq. 2)")
+                                  "note": ("CTA-pair tiling: two 128 x 256 tiles, one above the other, on the two SMs of a "
+                                           "pair that share their B tiles (Eq. 2); T_MA = 128 buffers symmetrically") if stacked
+                                  else ("CTA-pair tiling: each SM holds 128 of the 256 rows, so T_MA = 128 buffers "
+                                        "symmetrically per SM and the B tile is shared by two SMs (Eq. 2)")
                                   if gemm_kernel == "atb_gemm_pair_kernel" else "single-CTA tiling"},
                        "step": "atb_quantize_bfp16 + atb_select_tiling + atb_gemm",
                        "l2": "inputs larger than L2 (A fp32 %d MB, B %d MB, C %d MB per step)" % (

@@ -94,6 +94,12 @@ atb_status_t atb_quantize_bfp16(const float* A_dev, int64_t M, int64_t K, int64_
  *          (the array-level sharing of Eq. 2).  Per SM - the paper's "core" - the accumulator is 128 rows
  *          tall, so T_MA = 128 is this tiling's SYMMETRIC form (rho per core = 128 / T_MA), only
  *          T_MA in {32, 64} buffer asymmetrically, and T_MA = 256 does not exist (ATB_ERR_BAD_TILING).
+ *          (T_MC, T_K, T_N) = (128, 128, 256) runs on a pair of SMs too where M > 128: the pair computes two
+ *          128 x 256 tiles, one above the other, one per SM, and shares their B tiles between them (Eq. 2 again);
+ *          each SM keeps its 128 x 256 accumulator twice, so the write-out of a tile runs beside the K loop of the
+ *          next one - the tiling of choice where K is shallow or the output is small.  T_MA = 128 is its symmetric
+ *          form, T_MA in {32, 64} buffer asymmetrically.  Where M <= 128 there is one tile row and nothing to share:
+ *          the tiling then runs on single SMs.  atb_tiling_plan() reports the pair's plan.
  * For fixed (T_MC, T_K, T_N) the result is bit-identical for every T_MA, and every call with the same
  * arguments on the same GPU model gives the same bits.  Between different (T_MC, T_K, T_N) results agree
  * within FP32 rounding, not bit for bit: a persistent CTA walks K upwards for one of its tiles and downwards
@@ -324,6 +330,8 @@ atb_status_t atb_score_tiling(const atb_hw_params_t* hw, int64_t K, atb_tiling_t
  * partially filled waves of output tiles over n_units - and returns them best first.  A CTA-pair
  * tiling (T_MC = 256, T_N = 512) is rated per CTA: feasible, buf_bytes_used, acc_bytes_used, eff_core
  * and the compute bound are those of the 128-row half tile one CTA holds, with the B tile shared by two.
+ * The stacked pair tiling (T_MC = 128, T_K = 128, T_N = 256, where M > 128) is rated as it is - a CTA holds a
+ * whole 128 x 256 tile - with the B tile shared by two and the tiles counted in stripes of 256 rows.
  *   hw:       NULL = atb_hw_params_b200().
  *   best:     receives the top feasible tiling (may be NULL).
  *   scores:   optional array of *n_scores entries, filled best first; *n_scores receives the

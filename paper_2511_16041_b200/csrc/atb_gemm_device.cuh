@@ -44,8 +44,8 @@ constexpr int kMaxRingBars = 32;
 constexpr uint32_t kEpilogueBoxBytes = 32 * 128;   // 32 rows x 64 bf16 columns
 // The CTA-pair kernel stages C in full-size boxes (128-byte rows) where 64- and 128-row slabs leave room
 // for them, and in half-size boxes under 32-row slabs, whose deeper raw ring needs the space.
-constexpr int pair_box_cols(int slab) { return slab >= 64 ? 64 : 32; }
-constexpr uint32_t pair_box_bytes(int slab) { return 32u * pair_box_cols(slab) * 2u; }
+constexpr int pair_box_cols(int slab, int T_N = 512) { return (slab >= 64 || T_N == 256) ? 64 : 32; }
+constexpr uint32_t pair_box_bytes(int slab, int T_N = 512) { return 32u * pair_box_cols(slab, T_N) * 2u; }
 constexpr uint32_t kSmemBudget = 232448;          // 227 KB of dynamic shared memory per CTA
 #ifdef ATB_TEST_WAIT_NS                             // test build of the timeout path only: a short limit
 constexpr uint64_t kWaitTimeoutNs = ATB_TEST_WAIT_NS;
@@ -146,19 +146,28 @@ constexpr RingPlan plan_single(int T_MA, int T_MC, int T_K, int T_N) {
     return pl;
 }
 
-// CTA-pair kernel (T_MC = 256, T_N = 512, T_K = 64); `slab` = min(T_MA, 128) rows.
-constexpr RingPlan plan_pair(int slab) {
+// CTA-pair kernel; `slab` = T_MA <= 128 rows.  Two forms:
+//   T_N = 512, T_K = 64: one 256 x 512 tile per pair; each CTA holds a 128 x 512 accumulator (all of its tensor
+//                        memory), one buffer.
+//   T_N = 256, T_K = 128: two 128 x 256 tiles, one above the other, per pair (the tiling 128, 128, 256 on more than
+//                        one tile row): each CTA holds its 128 x 256 accumulator twice, so the epilogue of a tile -
+//                        bound by what one SM can store per unit of time - runs beside the K loop of the next
+//                        tile.  A B stage is 128 rows deep: two 64-column rounds of A per stage keep the K-step
+//                        at 1024 tensor cycles, the rate at which the leader needs both CTAs' operands.
+constexpr RingPlan plan_pair(int slab, int T_N = 512) {
     RingPlan pl;
-    if (!(slab == 32 || slab == 64 || slab == 128)) return pl;
+    if (!(slab == 32 || slab == 64 || slab == 128) || !(T_N == 512 || T_N == 256)) return pl;
     const int slabs = 128 / slab;
+    const bool wide = T_N == 512;
+    // this CTA's half of a B stage: 128 columns of every 256-column chunk, 64 (wide) or 128 rows deep: 32 KB either way
     const uint32_t b_bytes = 4 * 64 * 128, group_bytes = 128 * 64 * 2, raw_bytes = slab * 64 * 9 / 8;
     const int dqg = 4;
     pl.dqg = dqg;
-    pl.acc_bufs = 1;
+    pl.acc_bufs = wide ? 1 : 2;
     pl.tmem_cols = 512;
     const auto total = [=](int b, int g, int r) {
         return ring_smem_bytes(b_bytes, group_bytes, raw_bytes, 2, dqg, slab_bundle(slabs, r, dqg), b, g,
-                               g * (slabs / slab_bundle(slabs, r, dqg)), r, pair_box_bytes(slab));
+                               g * (slabs / slab_bundle(slabs, r, dqg)), r, pair_box_bytes(slab, T_N));
     };
     const auto bars_ok = [=](int g, int r) {
         return ring_bars(r, dqg * slab_bundle(slabs, r, dqg)) <= kMaxRingBars &&

@@ -463,12 +463,14 @@ static void fill_plan(const RingPlan& pl, GemmPlan* plan) {
     plan->smem_bytes = pl.smem_bytes;
 }
 
-bool plan_gemm(int T_MA, int T_MC, int T_K, int T_N, GemmPlan* plan) {
+bool plan_gemm(int T_MA, int T_MC, int T_K, int T_N, GemmPlan* plan, bool single_cta) {
     if (T_MA <= 0 || T_MC <= 0 || T_MA > T_MC) return false;
     // On the CTA pair each SM holds 128 rows of the tile: a slab cannot be taller than that, and
     // T_MA = 128 is the pair's symmetric form.
     if (is_pair_tiling(T_MC, T_K, T_N) && T_MA > 128) return false;
-    const RingPlan pl = is_pair_tiling(T_MC, T_K, T_N) ? plan_pair(T_MA) : plan_single(T_MA, T_MC, T_K, T_N);
+    const RingPlan pl = is_pair_tiling(T_MC, T_K, T_N)                            ? plan_pair(T_MA, 512)
+                        : (is_stacked_pair_tiling(T_MC, T_K, T_N) && !single_cta) ? plan_pair(T_MA, 256)
+                                                                                  : plan_single(T_MA, T_MC, T_K, T_N);
     if (!pl.ok || !(T_MA == 32 || T_MA == 64 || T_MA == 128 || T_MA == 256)) return false;
     fill_plan(pl, plan);
     return true;
@@ -542,8 +544,17 @@ extern "C" atb_status_t atb_gemm(int64_t M, int64_t N, int64_t K, int T_MA, int 
         return atb::fail(ATB_ERR_BAD_SHAPE, "too many output tiles");
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (atb::is_pair_tiling(T_MC, T_K, T_N))
-        return atb::launch_gemm_pair(T_MA, plan, M, N, K, A_mant_dev, A_exp_dev, B_bf16_dev, ldb, C_bf16_dev, ldc,
+        return atb::launch_gemm_pair(T_MA, 512, plan, M, N, K, A_mant_dev, A_exp_dev, B_bf16_dev, ldb, C_bf16_dev, ldc,
                                      dev->num_sms, dev->error_flag, stream);
+    if (atb::is_stacked_pair_tiling(T_MC, T_K, T_N)) {
+        // Two 128 x 256 tiles, one above the other, on a CTA pair that shares their B tiles; a problem of one
+        // tile row has nothing to share and runs on single CTAs.
+        if (M > 128)
+            return atb::launch_gemm_pair(T_MA, 256, plan, M, N, K, A_mant_dev, A_exp_dev, B_bf16_dev, ldb, C_bf16_dev, ldc,
+                                         dev->num_sms, dev->error_flag, stream);
+        if (!atb::plan_gemm(T_MA, T_MC, T_K, T_N, &plan, true))
+            return atb::fail(ATB_ERR_BAD_TILING, "tiling (T_MA=%d, T_MC=%d, T_K=%d, T_N=%d) is not supported", T_MA, T_MC, T_K, T_N);
+    }
 
     switch (T_MC) {
         case 128:
@@ -628,7 +639,7 @@ atb_status_t gemm_splitk_with_workspace(int64_t M, int64_t N, int64_t K, int T_M
                                         const int8_t* mant, const uint8_t* exp, const void* B, int64_t ldb,
                                         void* C, int64_t ldc, int splits, float* ws, void* stream) {
     GemmPlan plan;
-    if (!plan_gemm(T_MA, T_MC, T_K, T_N, &plan))
+    if (!plan_gemm(T_MA, T_MC, T_K, T_N, &plan, true))      // split-K runs on single CTAs
         return fail(ATB_ERR_BAD_TILING, "tiling (T_MA=%d, T_MC=%d, T_K=%d, T_N=%d) is not supported", T_MA, T_MC, T_K, T_N);
     DeviceInfo* dev = nullptr;
     atb_status_t st_dev = device_info(&dev);
@@ -683,7 +694,7 @@ extern "C" atb_status_t atb_gemm_bfp16_out(int64_t M, int64_t N, int64_t K, int 
     if (dev->cc_major != 10 || dev->cc_minor != 0)
         return atb::fail(ATB_ERR_UNSUPPORTED_DEVICE, "compute capability %d.%d; this library runs on 10.0 only", dev->cc_major, dev->cc_minor);
     if (pair)
-        return atb::launch_gemm_pair(T_MA, plan, M, N, K, A_mant_dev, A_exp_dev, B_bf16_dev, ldb, C_mant_dev, N, dev->num_sms,
+        return atb::launch_gemm_pair(T_MA, 512, plan, M, N, K, A_mant_dev, A_exp_dev, B_bf16_dev, ldb, C_mant_dev, N, dev->num_sms,
                                      dev->error_flag, stream, C_exp_dev);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
 #define ATB_QOUT_CASE(TMA_, TMC_, TN_)                                                                       \

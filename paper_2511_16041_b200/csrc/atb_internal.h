@@ -26,11 +26,17 @@ struct GemmPlan {
     int tmem_cols;       // allocated TMEM columns (power of two)
     uint32_t smem_bytes; // dynamic shared memory of the launch
 };
-// Fills `plan`; false if the tiling is not supported or does not fit.
-bool plan_gemm(int T_MA, int T_MC, int T_K, int T_N, GemmPlan* plan);
-// True for the tilings executed by a CTA pair (cluster of 2): T_MC = 256, T_N = 512, T_K = 64.
+// Fills `plan`; false if the tiling is not supported or does not fit.  `single_cta` asks for the one-CTA
+// plan of a tiling that normally runs as stacked tiles on a CTA pair (see is_stacked_pair_tiling).
+bool plan_gemm(int T_MA, int T_MC, int T_K, int T_N, GemmPlan* plan, bool single_cta = false);
+// True for the tiling whose 256 x 512 tile is computed by a CTA pair (cluster of 2): T_MC = 256, T_N = 512, T_K = 64.
 inline bool is_pair_tiling(int T_MC, int T_K, int T_N) { return T_MC == 256 && T_N == 512 && T_K == 64; }
-atb_status_t launch_gemm_pair(int T_MA, const GemmPlan& plan, int64_t M, int64_t N, int64_t K, const int8_t* mant,
+// True for the tiling whose 128 x 256 tiles are computed two at a time, one above the other, by a CTA pair
+// that shares every B tile between them: T_MC = 128, T_N = 256, T_K = 128 (atb_gemm, where M > 128; a problem of
+// one tile row and the split-K and BFP16-output entry points run it on single CTAs).
+inline bool is_stacked_pair_tiling(int T_MC, int T_K, int T_N) { return T_MC == 128 && T_N == 256 && T_K == 128; }
+// T_N = 512: the 256 x 512 pair tile; T_N = 256: two stacked 128 x 256 tiles.
+atb_status_t launch_gemm_pair(int T_MA, int T_N, const GemmPlan& plan, int64_t M, int64_t N, int64_t K, const int8_t* mant,
                               const uint8_t* exp, const void* B, int64_t ldb, void* C, int64_t ldc, int num_sms,
                               unsigned int* error_flag, void* stream, uint8_t* C_exp = nullptr);
 

@@ -154,10 +154,12 @@ atb_status_t atb_select_tiling(int64_t M, int64_t N, int64_t K, const atb_hw_par
     std::vector<atb_tiling_score_t> all;
     for (int mc : kMC) for (int n : kN) for (int k : kK) for (int ma : kMA) {
         atb::GemmPlan plan;
-        if (ma > mc || !atb::plan_gemm(ma, mc, k, n, &plan)) continue;
+        // two stacked 128 x 256 tiles on a CTA pair (where M has more than one tile row), else single CTAs
+        const bool stacked = atb::is_stacked_pair_tiling(mc, k, n) && M > 128;
+        if (ma > mc || !atb::plan_gemm(ma, mc, k, n, &plan, !stacked)) continue;
         const bool pair = atb::is_pair_tiling(mc, k, n);
         atb_hw_params_t h = hw;
-        if (pair) h.share_rows = hw.share_rows * 2;      // the B tile is shared by the two CTAs (Eq. 2)
+        if (pair || stacked) h.share_rows = hw.share_rows * 2;      // the B tile is shared by the two CTAs (Eq. 2)
         // thin slabs get the bundle discount only as far as this tiling's raw ring lets them be bundled
         const int slab = ma;
         if (hw.mma_rows > 0 && slab < hw.mma_rows) {
@@ -179,6 +181,7 @@ atb_status_t atb_select_tiling(int64_t M, int64_t N, int64_t K, const atb_hw_par
             s.acc_bytes_used = half.acc_bytes_used;
             if (hw.pair_efficiency > 0.0) s.compute_bound_flops *= hw.pair_efficiency;
         }
+        if (stacked && hw.pair_efficiency > 0.0) s.compute_bound_flops *= hw.pair_efficiency;
         // Look-ahead of the B ring (Little's law on the buffer of Eq. 1): a stage is busy from the
         // moment its load is issued until its UMMAs have run, so n stages sustain at most
         // n * t_stage / (latency + t_stage) of the UMMA rate.
@@ -209,10 +212,11 @@ atb_status_t atb_select_tiling(int64_t M, int64_t N, int64_t K, const atb_hw_par
         }
         // Wave quantisation: tiles are spread over the units (pairs of units for pair tilings); the
         // last wave may be partly empty and edge tiles compute padding.
-        const double units = pair ? hw.n_units / 2 : hw.n_units;
-        const double tiles = static_cast<double>(atb::ceil_div(M, mc)) * static_cast<double>(atb::ceil_div(N, n));
+        const double units = (pair || stacked) ? hw.n_units / 2 : hw.n_units;
+        const double tile_rows = stacked ? 2.0 * mc : mc;                  // rows a unit (CTA or pair) covers at a time
+        const double tiles = std::ceil(static_cast<double>(M) / tile_rows) * static_cast<double>(atb::ceil_div(N, n));
         const double waves = std::ceil(tiles / units);
-        const double useful = (static_cast<double>(M) * N) / (waves * units * mc * n);
+        const double useful = (static_cast<double>(M) * N) / (waves * units * tile_rows * n);
         s.compute_bound_flops *= useful;
         s.predicted_flops = std::min(s.mem_bound_flops, s.compute_bound_flops);
         if (hw.launch_seconds > 0.0) {

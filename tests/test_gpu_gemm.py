@@ -60,7 +60,7 @@ def test_atb_invariance_bitwise_across_T_MA():
     A = inputs.make_A("outlier", M, K)
     Bb = inputs.make_B_bits(K, N, None)
     mant, exp = oracle.quantize_bfp16(A)
-    for (mc, k, n) in [(256, 64, 256), (256, 128, 128), (128, 64, 128), (256, 64, 512)]:
+    for (mc, k, n) in [(256, 64, 256), (256, 128, 128), (128, 64, 128), (256, 64, 512), (128, 128, 256)]:
         ref = None
         for ma in (32, 64, 128, 256):
             if ma > mc or not atb.atb_tiling_supported(ma, mc, k, n):
@@ -224,7 +224,8 @@ def test_leading_dimensions_ragged_edges_every_epilogue():
     ldb, ldc = 600, 640
     Bfull = torch.full((K, ldb), 3.0, dtype=torch.bfloat16, device=dev())          # padding must not leak into C
     Bfull[:, :N] = bf16_bits_to_dev(Bb)
-    for t in [(128, 256, 64, 256), (128, 256, 64, 512), (64, 256, 64, 512), (32, 256, 64, 512), (128, 128, 64, 128)]:
+    for t in [(128, 256, 64, 256), (128, 256, 64, 512), (64, 256, 64, 512), (32, 256, 64, 512), (128, 128, 64, 128),
+              (128, 128, 128, 256), (32, 128, 128, 256)]:
         Cfull = torch.full((M + 3, ldc), -5.0, dtype=torch.bfloat16, device=dev())  # three guard rows below C
         atb.atb_gemm(M, N, K, *t, md, ed, Bfull, Cfull, ldb=ldb, ldc=ldc)
         atb.atb_device_status()
@@ -241,6 +242,7 @@ def test_tiny_and_degenerate_shapes():
         _check(mant, exp, Bb, (128, 128, 64, 64))
         _check(mant, exp, Bb, (32, 256, 128, 128))
         _check(mant, exp, Bb, (128, 256, 64, 512))       # CTA-pair kernel on a single partial tile
+        _check(mant, exp, Bb, (64, 128, 128, 256))       # stacked pair of tiles (single CTAs where M <= 128)
 
 
 def test_argument_errors():

@@ -119,8 +119,8 @@ def test_b200_refinements_can_be_switched_off():
     _, scores = atb.atb_select_tiling(8192, 8192, 8192, hw)
     for s in scores:
         t = (s.t.T_MA, s.t.T_MC, s.t.T_K, s.t.T_N)
-        if (t[1], t[3]) == (256, 512):
-            continue                                   # pair tilings are scored per CTA
+        if (t[1], t[3]) == (256, 512) or t[1:] == (128, 128, 256):
+            continue                                   # CTA-pair tilings: scored per CTA with the B tile shared by two
         ref = atb.atb_score_tiling(hw, 8192, t)
         tiles = math.ceil(8192 / t[1]) * math.ceil(8192 / t[3])       # edge tiles compute padding
         useful = 8192 * 8192 / (math.ceil(tiles / 148) * 148 * t[1] * t[3])
@@ -161,11 +161,14 @@ def test_per_tile_costs():
 def test_pair_tilings_are_rated_per_cta_and_chosen_at_deep_k():
     """A CTA of the pair holds half of the 256 x 512 tile: Eq. 1's budgets apply to that half (the whole
     accumulator would not fit one SM's tensor memory).  The pair is measured ahead where K is deep and
-    behind where it is shallow (its single accumulator stalls the next tile), and the preset follows."""
+    behind where it is shallow (its single accumulator stalls the next tile); there the stacked pair of
+    128 x 256 tiles, whose accumulators are double-buffered, is ahead, and the preset follows."""
     best, scores = atb.atb_select_tiling(8192, 8192, 8192, max_scores=256)
     by = {(s.t.T_MA, s.t.T_MC, s.t.T_K, s.t.T_N): s for s in scores}
     pair = by[(128, 256, 64, 512)]
     assert pair.feasible == 1 and pair.acc_bytes_used == 128 * 512 * 4
     assert (best.T_MC, best.T_K, best.T_N) == (256, 64, 512)
     shallow, _ = atb.atb_select_tiling(8192, 8192, 1024)
-    assert (shallow.T_MC, shallow.T_K, shallow.T_N) == (256, 64, 256)
+    assert (shallow.T_MC, shallow.T_K, shallow.T_N) == (128, 128, 256)
+    one_row, _ = atb.atb_select_tiling(128, 8192, 8192)          # a single tile row has nothing to share
+    assert atb.atb_tiling_plan(*one_row).acc_buffers in (1, 2)
