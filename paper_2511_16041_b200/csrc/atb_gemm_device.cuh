@@ -680,8 +680,10 @@ __device__ __forceinline__ void dequantiser_role(const Ctx& cx, int t, int my_gr
 // The accumulator is read 32 columns at a time; the load of the next 32 columns is issued as soon as
 // the current ones are packed to bf16, so that its latency passes behind the staging and the stores.
 // Two ways out of the box (measured: the single-CTA kernels are faster with the TMA store - one instruction in a
-// warp that competes with the dequantisers for issue slots -, the CTA-pair kernel, whose 128 x 512 accumulator
-// takes longest to drain, with direct stores: +4 % at K = 1024, +1 % at K = 8192):
+// warp that competes with the dequantisers for issue slots -, and so is the stacked form of the CTA-pair kernel,
+// whose drain runs beside the next tile's K loop; the CTA-pair kernel's 256 x 512 tile, whose 128 x 512 accumulator
+// per SM takes longest to drain and holds up the next tile meanwhile, is faster with direct stores: +4 % at
+// K = 1024, +1 % at K = 8192):
 //   TMA store   one instruction per box; costs about 5.5 cycles per row whatever the row carries (23 B per
 //               cycle and SM at 128-byte rows, half of that at 64-byte rows); edges are clipped by the tensor map.
 //   direct      the warp reads the box back row-wise and writes 16-byte chunks: 8 (4) lanes cover one row
