@@ -618,7 +618,7 @@ __device__ __forceinline__ void dequantiser_role(const Ctx& cx, int t, int my_gr
         bool ok = true;
 #pragma unroll
         for (int i = 0; i < C::BUNDLE; ++i)        // bars and buffers of a bundle are consecutive
-            ok = ok && wait_bar_t<false, PAIR>(cx, raw_full + 8 * (rr.bar + i), rr.phase, 0x301);
+            ok = ok && wait_bar_t<false, false>(cx, raw_full + 8 * (rr.bar + i), rr.phase, 0x301);     // filled by this CTA's own TMA loads
         ok = ok && wait_bar_t<false, PAIR>(cx, deq_empty + 8 * rd.freed_bar(), rd.freed_parity(), 0x302);
         if (!ok) break;
 #ifndef ATB_PROFILE_SKIP_DEQUANT    // diagnostic: the pipeline without the conversion work (results are wrong)

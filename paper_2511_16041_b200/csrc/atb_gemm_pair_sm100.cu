@@ -192,7 +192,7 @@ atb_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_c
                     // (a downward walk keeps the rounds of a B stage in their upward order)
                     const int kh = serpentine_k(it, kh0 / C::KH, 0, p.k_steps) * C::KH + kh0 % C::KH;
                     for (int s = 0; s < C::SLABS; ++s) {
-                        if (!(ok = wait_bar_cl_spin(cx, raw_empty + 8 * rr.freed_bar(), rr.freed_parity(), 0x002))) break;
+                        if (!(ok = wait_bar_spin(cx, raw_empty + 8 * rr.freed_bar(), rr.freed_parity(), 0x002))) break;   // a barrier of this CTA alone
                         const uint32_t fr = raw_full + 8 * rr.bar;
                         const uint32_t dst = raw_base + rr.buf() * C::RAW_BYTES;
                         mbar_arrive_expect_tx(fr, C::RAW_BYTES);
