@@ -393,7 +393,7 @@ def run_ours(args):
     quant_ms = q0.elapsed_time(q1) / 10
 
     # ---------------- the T_MA ablation and a sustained leg (one GPU only) ----------------
-    ablation = sustained = None
+    ablation = sustained = library = None
     if world == 1 and not args.no_ablation:
         def time_gemm(t, reps):
             for _ in range(2):
@@ -406,14 +406,35 @@ def run_ours(args):
             stream.synchronize()
             return min(a.elapsed_time(b) for a, b in evs)
 
-        # every tiling of both families in one process, walked in two opposite orders (what ran just
+        # the library's bf16 GEMM (torch.matmul -> cuBLAS) on operands of the same shape, timed the same way in
+        # the same walk: context for the fraction of the measured peak, which moves from GPU to GPU
+        A_lib = torch.randn((M, K), device=dev, dtype=torch.float32).to(torch.bfloat16)
+        C_lib = torch.empty((M, N), device=dev, dtype=torch.bfloat16)
+
+        def time_library(reps):
+            with torch.cuda.stream(stream):
+                for _ in range(2):
+                    torch.matmul(A_lib, B_dev, out=C_lib)
+                evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+                for a, b in evs:
+                    a.record(stream)
+                    torch.matmul(A_lib, B_dev, out=C_lib)
+                    b.record(stream)
+            stream.synchronize()
+            return min(a.elapsed_time(b) for a, b in evs)
+
+        # every tiling of the families in one process, walked in two opposite orders (what ran just
         # before moves a rate by a few per cent); a tiling keeps its better time
+        t_head = tuple(tiling_used[0])
         walk = [t for fam in ABLATION_FAMILIES.values() for t in fam]
-        best_ms = {}
+        walk += [t_head] if t_head not in walk else []
+        best_ms, lib_ms = {}, []
         for order in (walk, walk[::-1]):
             for t in order:
                 ms = time_gemm(t, 5)
                 best_ms[t] = min(ms, best_ms.get(t, ms))
+                if t == t_head:
+                    lib_ms.append(time_library(5))
         atb.atb_device_status(stream)
         tf = lambda t: 2.0 * M * N * K / (best_ms[t] * 1e-3) / 1e12
         ablation = {"how": "atb_gemm alone on the resident planes; both families interleaved in one process, "
@@ -423,8 +444,12 @@ def run_ours(args):
             ablation["families"][fam] = [{"tiling": list(t), "rho_per_core": rho_per_core(t), "tflops": tf(t)} for t in tilings]
             ablation["atb_over_symmetric"][fam] = max(tf(t) for t in tilings[1:]) / tf(tilings[0])
 
+        library = {"tflops": 2.0 * M * N * K / (min(lib_ms) * 1e-3) / 1e12, "headline_tiling_tflops": tf(t_head),
+                   "how": "torch.matmul (cuBLAS) on bf16 A, B of the same shape, no conversion, timed next to the headline "
+                          "tiling in the ablation walk (best of 2 x 5 launches each)"}
+        library["headline_over_library"] = library["headline_tiling_tflops"] / library["tflops"]
+
         # sustained: the headline GEMM back to back for >= 2 s, so that the GPU settles under its power cap
-        t_head = tiling_used[0]
         n_launch = max(200, int(SUSTAINED_SECONDS * 1e3 / gemm_ms))
         s_sampler = ClockSampler(physical_gpu_index(local_rank))
         s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -438,6 +463,15 @@ def run_ours(args):
         s_clocks = s_sampler.stop()
         atb.atb_device_status(stream)
         s_ms = s0.elapsed_time(s1)
+        # and the library GEMM the same way, for as many launches
+        l0, l1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with torch.cuda.stream(stream):
+            l0.record(stream)
+            for _ in range(n_launch):
+                torch.matmul(A_lib, B_dev, out=C_lib)
+            l1.record(stream)
+        stream.synchronize()
+        library["sustained_tflops"] = 2.0 * M * N * K * n_launch / (l0.elapsed_time(l1) * 1e-3) / 1e12
         sustained = {"launches": n_launch, "seconds": s_ms * 1e-3,
                      "achieved": 2.0 * M * N * K * n_launch / (s_ms * 1e-3) / 1e12, "clocks": s_clocks}
 
@@ -498,6 +532,7 @@ def run_ours(args):
             line["roofline"]["sustained"] = sustained
         if ablation is not None:
             line["ablation"] = ablation
+            line["roofline"]["library_bf16_gemm_same_run"] = library
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_oracle_sample(name, args.cpu_seconds)
         print(json.dumps(line))

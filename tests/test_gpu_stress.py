@@ -124,13 +124,16 @@ def test_soak_cta_pair_against_single_cta_bitwise():
     memory model does not promise to order against the leader's cluster-scope acquire.  Random shapes
     (ragged edges, one to hundreds of K-steps), the three slab heights of the pair and - where no CTA
     computes more than one tile, so that both kernels add the same products in the same order - the
-    single-CTA 256 x 256 tiling: all results must be bit-identical, launch after launch."""
+    single-CTA 256 x 256 tiling: all results must be bit-identical, launch after launch.  The stacked pair
+    (two 128 x 256 tiles on a pair) runs the same hand-over: its three slab heights must agree bit for bit
+    with one another at every size, and with all the others where every kernel has one tile per CTA."""
     import random
     import time
     g = torch.Generator(device=dev())
     g.manual_seed(11)
     rnd = random.Random(5)
     pair_tilings = [(128, 256, 64, 512), (64, 256, 64, 512), (32, 256, 64, 512)]
+    stacked_tilings = [(128, 128, 128, 256), (64, 128, 128, 256), (32, 128, 128, 256)]
     launches, t_end = 0, time.time() + 12.0
     while time.time() < t_end or launches < 400:
         M = rnd.choice([300, 1000, 2048, 4096, 5000])
@@ -138,10 +141,11 @@ def test_soak_cta_pair_against_single_cta_bitwise():
         K = rnd.choice([16, 64, 448, 1024, 1104, 4096])
         one_wave = -(-M // 256) * -(-N // 256) <= 148 and -(-M // 256) * -(-N // 512) <= 74
         tilings = ([(128, 256, 64, 256)] if one_wave else []) + pair_tilings
+        stacked_one_wave = one_wave and -(-M // 256) * -(-N // 256) <= 74
         mant = torch.randint(-127, 128, (M, K), dtype=torch.int8, device=dev(), generator=g)
         plane = torch.randint(100, 150, (atb.atb_bfp16_exp_bytes(M, K),), dtype=torch.uint8, device=dev(), generator=g)
         B = torch.randn((K, N), device=dev(), generator=g).to(torch.bfloat16)
-        ref = None
+        ref = ref_stacked = None
         for rep in range(6):
             for t in tilings:
                 C = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device=dev())
@@ -151,6 +155,14 @@ def test_soak_cta_pair_against_single_cta_bitwise():
                     ref = C.view(torch.int16).clone()
                 else:
                     assert torch.equal(C.view(torch.int16), ref), ((M, N, K), t, rep)
+            if rep < 2:
+                for t in stacked_tilings:
+                    C = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device=dev())
+                    atb.atb_gemm(M, N, K, *t, mant, plane, B, C)
+                    launches += 1
+                    if ref_stacked is None:
+                        ref_stacked = ref if stacked_one_wave else C.view(torch.int16).clone()
+                    assert torch.equal(C.view(torch.int16), ref_stacked), ((M, N, K), t, rep)
         atb.atb_device_status()
         assert bool(torch.isfinite(ref.view(torch.bfloat16).float()).all())
     assert launches >= 400
