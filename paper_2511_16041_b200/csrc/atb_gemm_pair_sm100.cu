@@ -167,10 +167,16 @@ atb_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_c
                     // both halves of the B tile are credited to the leader's barrier
                     if (leader) mbar_arrive_expect_tx(b_full + 8 * rb.stage, 2 * C::B_BYTES);
                     const uint32_t fb = mapa_shared(b_full + 8 * rb.stage, 0);
+#ifdef ATB_PROFILE
+                    const long long issue_t0 = clock64();
+#endif
 #pragma unroll
                     for (int j = 0; j < T_N / 128; ++j)
                         tma_load_2d_pair(b_base + rb.stage * C::B_BYTES + j * C::B_BOX_BYTES, &tm_b,
                                          colb + (j >> 1) * 256 + (j & 1) * 64, k * C::T_K, fb);
+#ifdef ATB_PROFILE      // slot 8: cycles this thread spent issuing the loads of B
+                    atomicAdd(&g_wait_cycles[blockIdx.x & 255][8], static_cast<unsigned long long>(clock64() - issue_t0));
+#endif
                     rb.advance(C::NB);
                 }
             }
@@ -195,6 +201,9 @@ atb_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_c
                         if (!(ok = wait_bar_spin(cx, raw_empty + 8 * rr.freed_bar(), rr.freed_parity(), 0x002))) break;   // a barrier of this CTA alone
                         const uint32_t fr = raw_full + 8 * rr.bar;
                         const uint32_t dst = raw_base + rr.buf() * C::RAW_BYTES;
+#ifdef ATB_PROFILE
+                        const long long issue_t0 = clock64();
+#endif
                         mbar_arrive_expect_tx(fr, C::RAW_BYTES);
 #ifndef ATB_NO_L2_HINTS
                         tma_load_2d_hint(dst, &tm_mant, kh * kKA, row0 + s * SLAB_ROWS, fr, a_policy);
@@ -202,6 +211,9 @@ atb_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_c
 #else
                         tma_load_2d(dst, &tm_mant, kh * kKA, row0 + s * SLAB_ROWS, fr);
                         tma_load_2d(dst + C::RAW_MANT_BYTES, &tm_exp, row0 + s * SLAB_ROWS, kh, fr);
+#endif
+#ifdef ATB_PROFILE      // slot 3: cycles this thread spent issuing the loads of A
+                        atomicAdd(&g_wait_cycles[blockIdx.x & 255][3], static_cast<unsigned long long>(clock64() - issue_t0));
 #endif
                         rr.template advance<1>();
                     }
