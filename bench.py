@@ -568,11 +568,13 @@ def run_entry(args):
         if not args.tiling:         # the selection's pick where this entry has that tiling
             best, _ = atb.atb_select_tiling(M, N, K)
             pick = (best.T_MA, best.T_MC, best.T_K, best.T_N)
-            if pick[2] == 64 and pick[0] in (64, 128) and (pick[1], pick[3]) in ((128, 128), (128, 256), (256, 128), (256, 256), (256, 512)):
+            if pick[0] in (64, 128) and (pick[1:] == (128, 128, 256) or (pick[2] == 64 and (pick[1], pick[3]) in (
+                    (128, 128), (128, 256), (256, 128), (256, 256), (256, 512)))):
                 tiling = pick
         Cm = torch.empty((M, N), dtype=torch.int8, device=dev)
         Ce = torch.empty(atb.atb_bfp16_exp_bytes(M, N), dtype=torch.uint8, device=dev)
-        kname = "atb_gemm_pair_kernel" if tiling[1:] == (256, 64, 512) else "atb_gemm_kernel"
+        on_pair = tiling[1:] == (256, 64, 512) or (tiling[1:] == (128, 128, 256) and M > 128)
+        kname = "atb_gemm_pair_kernel" if on_pair else "atb_gemm_kernel"
         kernel, what = kname + " (quantising epilogue)", "atb_quantize_bfp16 + atb_gemm_bfp16_out"
         quantises = True
         call = lambda: atb.atb_gemm_bfp16_out(M, N, K, *tiling, mant, plane, B_dev, Cm, Ce, stream=stream)

@@ -179,9 +179,10 @@ atb_status_t atb_gemm_splitk_noalloc(int64_t M, int64_t N, int64_t K, int T_MA, 
  *   C_mant_dev: int8 [M][N] row-major (contiguous), 16-byte aligned (written);
  *   C_exp_dev:  exponent plane of atb_bfp16_exp_bytes(M, N) bytes, 16-byte aligned (written; the
  *               plane's padding rows get exponent 0).
- * Shapes: M >= 1, N % 16 == 0, K % 16 == 0.  Tilings: T_K = 64, T_MA in {64, 128}, and T_MC in {128, 256}
- * with T_N in {128, 256} or T_MC = 256 with T_N = 512 (the CTA-pair tiling).  Other arguments, conventions
- * and errors as for atb_gemm. */
+ * Shapes: M >= 1, N % 16 == 0, K % 16 == 0.  Tilings: T_MA in {64, 128} with T_K = 64, T_MC in {128, 256} and
+ * T_N in {128, 256}; with (T_MC, T_K, T_N) = (256, 64, 512), the CTA-pair tiling; and with (128, 128, 256), which
+ * runs as two stacked tiles on a CTA pair where M > 128, as in atb_gemm.  Other arguments, conventions and errors
+ * as for atb_gemm. */
 atb_status_t atb_gemm_bfp16_out(int64_t M, int64_t N, int64_t K, int T_MA, int T_MC, int T_K, int T_N,
                                 const int8_t* A_mant_dev, const uint8_t* A_exp_dev,
                                 const void* B_bf16_dev, int64_t ldb,

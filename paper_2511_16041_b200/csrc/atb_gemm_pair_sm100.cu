@@ -408,7 +408,7 @@ atb_status_t launch_gemm_pair(int T_MA, int T_N, const GemmPlan& plan, int64_t M
     if (T_MA == TMA_ && T_N == TN_)                                                                                    \
         return launch_pair_t<TMA_, TN_, Q_>(plan, M, N, K, mant, exp, B, ldb, C, ldc, num_sms, error_flag, st, C_exp);
     if (C_exp) {       // BFP16 output: C is the int8 mantissa plane
-        ATB_PAIR_CASE(64, 512, true) ATB_PAIR_CASE(128, 512, true)
+        ATB_PAIR_CASE(64, 512, true) ATB_PAIR_CASE(128, 512, true) ATB_PAIR_CASE(64, 256, true) ATB_PAIR_CASE(128, 256, true)
         return atb::fail(ATB_ERR_BAD_TILING, "no pair kernel with the quantising epilogue for T_MA=%d, T_N=%d", T_MA, T_N);
     }
     ATB_PAIR_CASE(32, 512, false) ATB_PAIR_CASE(64, 512, false) ATB_PAIR_CASE(128, 512, false)

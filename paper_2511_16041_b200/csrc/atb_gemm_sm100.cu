@@ -680,29 +680,33 @@ extern "C" atb_status_t atb_gemm_bfp16_out(int64_t M, int64_t N, int64_t K, int 
         return atb::fail(ATB_ERR_BAD_SHAPE, "need M >= 1, N %% 16 == 0, K %% 16 == 0 (got %lld, %lld, %lld)", (long long)M, (long long)N, (long long)K);
     if (ldb < N || ldb % 8 != 0) return atb::fail(ATB_ERR_BAD_SHAPE, "ldb=%lld must be >= N and a multiple of 8", (long long)ldb);
     const bool pair = atb::is_pair_tiling(T_MC, T_K, T_N) && (T_MA == 64 || T_MA == 128);
-    if (!pair && !splitk_tiling_ok(T_MA, T_MC, T_K, T_N))
-        return atb::fail(ATB_ERR_BAD_TILING, "the quantising epilogue supports T_K = 64, T_MA in {64, 128}, and T_MC in {128, 256} with T_N in {128, 256} or T_MC = 256 with T_N = 512");
+    // (T_MA, 128, 128, 256): two stacked tiles on a CTA pair where there is more than one tile row, as in atb_gemm
+    const bool stacked = atb::is_stacked_pair_tiling(T_MC, T_K, T_N) && (T_MA == 64 || T_MA == 128);
+    if (!pair && !stacked && !splitk_tiling_ok(T_MA, T_MC, T_K, T_N))
+        return atb::fail(ATB_ERR_BAD_TILING, "the quantising epilogue supports T_MA in {64, 128} with T_K = 64, T_MC in {128, 256}, T_N in {128, 256}; with (T_MC, T_K, T_N) = (256, 64, 512); and with (128, 128, 256)");
     if (!atb::aligned16(A_mant_dev) || !atb::aligned16(A_exp_dev) || !atb::aligned16(B_bf16_dev) || !atb::aligned16(C_mant_dev) ||
         !atb::aligned16(C_exp_dev))
         return atb::fail(ATB_ERR_MISALIGNED, "all device pointers must be 16-byte aligned");
     atb::GemmPlan plan;
-    if (!atb::plan_gemm(T_MA, T_MC, T_K, T_N, &plan))
+    const bool stacked_pair = stacked && M > 128;
+    if (!atb::plan_gemm(T_MA, T_MC, T_K, T_N, &plan, /*single_cta=*/!stacked_pair))
         return atb::fail(ATB_ERR_BAD_TILING, "tiling (T_MA=%d, T_MC=%d, T_K=%d, T_N=%d) is not supported", T_MA, T_MC, T_K, T_N);
     DeviceInfo* dev = nullptr;
     atb_status_t st_dev = device_info(&dev);
     if (st_dev != ATB_OK) return st_dev;
     if (dev->cc_major != 10 || dev->cc_minor != 0)
         return atb::fail(ATB_ERR_UNSUPPORTED_DEVICE, "compute capability %d.%d; this library runs on 10.0 only", dev->cc_major, dev->cc_minor);
-    if (pair)
-        return atb::launch_gemm_pair(T_MA, 512, plan, M, N, K, A_mant_dev, A_exp_dev, B_bf16_dev, ldb, C_mant_dev, N, dev->num_sms,
-                                     dev->error_flag, stream, C_exp_dev);
+    if (pair || stacked_pair)
+        return atb::launch_gemm_pair(T_MA, pair ? 512 : 256, plan, M, N, K, A_mant_dev, A_exp_dev, B_bf16_dev, ldb, C_mant_dev, N,
+                                     dev->num_sms, dev->error_flag, stream, C_exp_dev);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-#define ATB_QOUT_CASE(TMA_, TMC_, TN_)                                                                       \
-    if (T_MA == TMA_ && T_MC == TMC_ && T_N == TN_)                                                          \
-        return launch<TMA_, TMC_, 64, TN_, false, true>(plan, M, N, K, A_mant_dev, A_exp_dev, B_bf16_dev, ldb, \
-                                                        C_mant_dev, N, dev->num_sms, dev->error_flag, st, 1, C_exp_dev);
-    ATB_QOUT_CASE(64, 128, 128) ATB_QOUT_CASE(128, 128, 128) ATB_QOUT_CASE(64, 128, 256) ATB_QOUT_CASE(128, 128, 256)
-    ATB_QOUT_CASE(64, 256, 128) ATB_QOUT_CASE(128, 256, 128) ATB_QOUT_CASE(64, 256, 256) ATB_QOUT_CASE(128, 256, 256)
+#define ATB_QOUT_CASE(TMA_, TMC_, TK_, TN_)                                                                      \
+    if (T_MA == TMA_ && T_MC == TMC_ && T_K == TK_ && T_N == TN_)                                                \
+        return launch<TMA_, TMC_, TK_, TN_, false, true>(plan, M, N, K, A_mant_dev, A_exp_dev, B_bf16_dev, ldb,  \
+                                                         C_mant_dev, N, dev->num_sms, dev->error_flag, st, 1, C_exp_dev);
+    ATB_QOUT_CASE(64, 128, 64, 128) ATB_QOUT_CASE(128, 128, 64, 128) ATB_QOUT_CASE(64, 128, 64, 256) ATB_QOUT_CASE(128, 128, 64, 256)
+    ATB_QOUT_CASE(64, 256, 64, 128) ATB_QOUT_CASE(128, 256, 64, 128) ATB_QOUT_CASE(64, 256, 64, 256) ATB_QOUT_CASE(128, 256, 64, 256)
+    ATB_QOUT_CASE(64, 128, 128, 256) ATB_QOUT_CASE(128, 128, 128, 256)        // one tile row of the stacked tiling
 #undef ATB_QOUT_CASE
     return atb::fail(ATB_ERR_BAD_TILING, "no kernel for tiling (T_MA=%d, T_MC=%d, T_K=%d, T_N=%d)", T_MA, T_MC, T_K, T_N);
 }

@@ -21,8 +21,9 @@ pytestmark = pytest.mark.gpu
 TILINGS = [(64, 128, 64, 128), (128, 128, 64, 256), (64, 256, 64, 128), (128, 256, 64, 256), (64, 256, 64, 256)]
 # The CTA-pair tilings have no split-K form to read their FP32 accumulators through.  Their UMMAs add the
 # same products in the same order as the single-CTA 256 x 256 tiling, so their planes are compared with
-# that tiling's bit for bit, and with the FP64 oracle like the others.
-PAIR_TILINGS = [(64, 256, 64, 512), (128, 256, 64, 512)]
+# that tiling's bit for bit, and with the FP64 oracle like the others.  The same holds for the stacked pair
+# (two 128 x 256 tiles on a CTA pair, B stages 128 rows deep) on shapes where no CTA has a second tile.
+PAIR_TILINGS = [(64, 256, 64, 512), (128, 256, 64, 512), (64, 128, 128, 256), (128, 128, 128, 256)]
 
 
 def fp32_accumulators(M, N, K, tiling, md, ed, Bd):
@@ -75,6 +76,21 @@ def test_planes_equal_the_quantiser_on_the_fp32_accumulators(shape):
         half_step = np.repeat(np.ldexp(1.0, got_e.astype(np.int64) - 134), 8, axis=1)
         q_err = np.where(np.abs(got_m.astype(np.int64)) == 127, 2.0 * half_step, half_step)
         assert np.all(np.abs(Cq - Cr) <= q_err + S * 2.0 ** -12), tiling
+
+
+def test_stacked_tiling_with_one_tile_row():
+    """(T_MA, 128, 128, 256) on M <= 128 runs on single CTAs (as in atb_gemm): planes equal those of the T_K = 64 form
+    of the same tile, whose UMMAs add the same products in the same order."""
+    M, N, K = 100, 528, 448
+    A = inputs.make_A("laplace", M, K)
+    Bb = inputs.make_B_bits(K, N)
+    mant, exp = oracle.quantize_bfp16(A)
+    md, ed = planes_to_dev(mant, exp)
+    Bd = bf16_bits_to_dev(Bb)
+    ref_m, ref_plane = run_qout(M, N, K, (128, 128, 64, 256), md, ed, Bd)
+    for tiling in [(64, 128, 128, 256), (128, 128, 128, 256)]:
+        got_m, plane = run_qout(M, N, K, tiling, md, ed, Bd)
+        assert np.array_equal(got_m, ref_m) and np.array_equal(plane, ref_plane), tiling
 
 
 def test_output_feeds_the_next_gemm():
