@@ -587,6 +587,54 @@ __device__ __forceinline__ void dequant_bundle(const DequantLane<C>& ln, uint32_
 }
 
 // ---------------------------------------------------------------------------------------------
+// The raw-A producer role of atb_gemm_kernel and atb_gemm_pair_kernel (one elected thread of a warp of its own:
+// the raw slabs feed the dequantisers, which run ahead of the UMMAs, so these loads must not queue behind the
+// wait for a free B stage).  Per work item of the CTA - next_item(it, row0, k_begin, k_end) gives the first row of
+// this CTA's part of the item and its range of K-steps, false when the CTA has no more - it walks the 64-column
+// rounds of the K range (upwards or downwards, see serpentine_k) and loads the C::SLABS slabs of
+// C::SLAB_ROWS rows of each round: mantissa box and exponent box into one raw buffer, under one barrier.
+// ---------------------------------------------------------------------------------------------
+template <class C, class NextItem>
+__device__ __forceinline__ void a_producer_role(const Ctx& cx, const CUtensorMap* tm_mant, const CUtensorMap* tm_exp,
+                                                uint32_t raw_full, uint32_t raw_empty, uint32_t raw_base, NextItem&& next_item) {
+    Cursor<C::NR, C::LR> rr;
+    bool ok = true;
+#ifndef ATB_NO_L2_HINTS
+    // The tile walk keeps a band of A row panels in use wave after wave while the B column panels
+    // change: A is asked to stay in the L2 longest.
+    const uint64_t a_policy = l2_policy_evict_last();
+#endif
+    int row0 = 0, k_begin = 0, k_end = 0;
+    for (int it = 0; ok && next_item(it, row0, k_begin, k_end); ++it) {
+        for (int kh0 = k_begin * C::KH; ok && kh0 < k_end * C::KH; ++kh0) {      // 64-column rounds
+            // (a downward walk keeps the rounds of a T_K = 128 step in their upward order)
+            const int kh = serpentine_k(it, kh0 / C::KH, k_begin, k_end) * C::KH + kh0 % C::KH;
+            for (int s = 0; s < C::SLABS; ++s) {
+                // (a barrier of this CTA alone, on a CTA pair too)
+                if (!(ok = wait_bar_spin(cx, raw_empty + 8 * rr.freed_bar(), rr.freed_parity(), 0x002))) break;
+                const uint32_t fr = raw_full + 8 * rr.bar;
+                const uint32_t dst = raw_base + rr.buf() * C::RAW_BYTES;
+#ifdef ATB_PROFILE
+                const long long issue_t0 = clock64();
+#endif
+                mbar_arrive_expect_tx(fr, C::RAW_BYTES);
+#ifndef ATB_NO_L2_HINTS
+                tma_load_2d_hint(dst, tm_mant, kh * kKA, row0 + s * C::SLAB_ROWS, fr, a_policy);
+                tma_load_2d_hint(dst + C::RAW_MANT_BYTES, tm_exp, row0 + s * C::SLAB_ROWS, kh, fr, a_policy);
+#else
+                tma_load_2d(dst, tm_mant, kh * kKA, row0 + s * C::SLAB_ROWS, fr);
+                tma_load_2d(dst + C::RAW_MANT_BYTES, tm_exp, row0 + s * C::SLAB_ROWS, kh, fr);
+#endif
+#ifdef ATB_PROFILE      // slot 3: cycles this thread spent issuing the loads of A
+                atomicAdd(&g_wait_cycles[blockIdx.x & 255][3], static_cast<unsigned long long>(clock64() - issue_t0));
+#endif
+                rr.template advance<1>();
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
 // The dequantiser role of atb_gemm_kernel and atb_gemm_pair_kernel: one warp of dequantiser group
 // `my_group` (thread `t` of the group).  The group does not need to know tiles or K-steps: slabs arrive in
 // ring order, so it takes every DQ_GROUPS-th bundle of the CTA's stream of `my_slabs` raw slabs, waits for the

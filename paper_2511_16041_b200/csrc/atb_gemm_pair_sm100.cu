@@ -184,41 +184,16 @@ atb_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_c
     } else if (warp == kAProducerWarp) {
         // ================================ TMA producer: raw A slabs ====================
         if (elect_one()) {
-            Cursor<C::NR, C::LR> rr;
-            bool ok = true;
-#ifndef ATB_NO_L2_HINTS
-            const uint64_t a_policy = l2_policy_evict_last();   // a band's A panels serve wave after wave
-#endif
-            int it = 0;
-            for (int tile = cluster_id; ok && tile < total_tiles; tile += n_clusters, ++it) {
-                int mt, nt;
-                tile_coords(tile, p.m_tiles, p.n_tiles, mt, nt);
-                const int row0 = mt * 256 + static_cast<int>(rank) * 128;
-                for (int kh0 = 0; ok && kh0 < p.k_steps * C::KH; ++kh0) {                 // 64-column rounds
-                    // (a downward walk keeps the rounds of a B stage in their upward order)
-                    const int kh = serpentine_k(it, kh0 / C::KH, 0, p.k_steps) * C::KH + kh0 % C::KH;
-                    for (int s = 0; s < C::SLABS; ++s) {
-                        if (!(ok = wait_bar_spin(cx, raw_empty + 8 * rr.freed_bar(), rr.freed_parity(), 0x002))) break;   // a barrier of this CTA alone
-                        const uint32_t fr = raw_full + 8 * rr.bar;
-                        const uint32_t dst = raw_base + rr.buf() * C::RAW_BYTES;
-#ifdef ATB_PROFILE
-                        const long long issue_t0 = clock64();
-#endif
-                        mbar_arrive_expect_tx(fr, C::RAW_BYTES);
-#ifndef ATB_NO_L2_HINTS
-                        tma_load_2d_hint(dst, &tm_mant, kh * kKA, row0 + s * SLAB_ROWS, fr, a_policy);
-                        tma_load_2d_hint(dst + C::RAW_MANT_BYTES, &tm_exp, row0 + s * SLAB_ROWS, kh, fr, a_policy);
-#else
-                        tma_load_2d(dst, &tm_mant, kh * kKA, row0 + s * SLAB_ROWS, fr);
-                        tma_load_2d(dst + C::RAW_MANT_BYTES, &tm_exp, row0 + s * SLAB_ROWS, kh, fr);
-#endif
-#ifdef ATB_PROFILE      // slot 3: cycles this thread spent issuing the loads of A
-                        atomicAdd(&g_wait_cycles[blockIdx.x & 255][3], static_cast<unsigned long long>(clock64() - issue_t0));
-#endif
-                        rr.template advance<1>();
-                    }
-                }
-            }
+            int tile = cluster_id;
+            a_producer_role<C>(cx, &tm_mant, &tm_exp, raw_full, raw_empty, raw_base,
+                               [&](int, int& row0, int& k_begin, int& k_end) {
+                                   if (tile >= total_tiles) return false;
+                                   int mt, nt;
+                                   tile_coords(tile, p.m_tiles, p.n_tiles, mt, nt);
+                                   row0 = mt * 256 + static_cast<int>(rank) * 128; k_begin = 0; k_end = p.k_steps;
+                                   tile += n_clusters;
+                                   return true;
+                               });
         }
     } else if (warp == 1) {
         // ================================ UMMA issuer (leader CTA) ====================

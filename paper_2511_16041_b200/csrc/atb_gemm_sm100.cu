@@ -39,6 +39,7 @@ struct Cfg {
     static constexpr int SLAB_ROWS = T_MA;
     static constexpr int G = T_MC / 128;                       // 128-row groups per output tile
     static constexpr int RHO = T_MC / T_MA;                    // slabs per K-step
+    static constexpr int SLABS = RHO;                          // (per 64-column round, the name the shared roles use)
     static constexpr int SPG = (T_MA < 128) ? 128 / T_MA : 1;  // slabs per group
     static constexpr int GPS = (T_MA > 128) ? T_MA / 128 : 1;  // groups per slab
     static constexpr int N_MMA = T_N > 256 ? 256 : T_N;        // UMMA N extent; T_N / N_MMA instructions side by side
@@ -165,38 +166,16 @@ atb_gemm_kernel(const __grid_constant__ CUtensorMap tm_mant, const __grid_consta
         }
     } else if (warp == kAProducerWarp) {
         // ================================ TMA producer: raw A slabs ====================
-        // A producer of its own: the raw slabs feed the dequantisers, which run ahead of the UMMAs,
-        // so these loads must not queue behind the wait for a free B stage.
         if (elect_one()) {
-            Cursor<C::NR, C::LR> rr;
-            bool ok = true;
-#ifndef ATB_NO_L2_HINTS
-            // The tile walk keeps a band of A row panels in use wave after wave while the B column panels
-            // change: A is asked to stay in the L2 longest.
-            const uint64_t a_policy = l2_policy_evict_last();
-#endif
-            int it = 0;
-            for (int item = blockIdx.x; ok && item < total_items; item += gridDim.x, ++it) {
-                const WorkItem w = work_item<SPLIT>(item, p);
-                for (int kh0 = w.k_begin * C::KH; ok && kh0 < w.k_end * C::KH; ++kh0) {      // 64-column rounds
-                    // (a downward walk keeps the two rounds of a T_K = 128 step in their upward order)
-                    const int kh = serpentine_k(it, kh0 / C::KH, w.k_begin, w.k_end) * C::KH + kh0 % C::KH;
-                    for (int s = 0; s < C::RHO; ++s) {
-                        if (!(ok = wait_bar_spin(cx, raw_empty + 8 * rr.freed_bar(), rr.freed_parity(), 0x002))) break;
-                        const uint32_t fr = raw_full + 8 * rr.bar;
-                        const uint32_t dst = raw_base + rr.buf() * C::RAW_BYTES;
-                        mbar_arrive_expect_tx(fr, C::RAW_BYTES);
-#ifndef ATB_NO_L2_HINTS
-                        tma_load_2d_hint(dst, &tm_mant, kh * kKA, w.mt * T_MC + s * T_MA, fr, a_policy);
-                        tma_load_2d_hint(dst + C::RAW_MANT_BYTES, &tm_exp, w.mt * T_MC + s * T_MA, kh, fr, a_policy);
-#else
-                        tma_load_2d(dst, &tm_mant, kh * kKA, w.mt * T_MC + s * T_MA, fr);
-                        tma_load_2d(dst + C::RAW_MANT_BYTES, &tm_exp, w.mt * T_MC + s * T_MA, kh, fr);
-#endif
-                        rr.template advance<1>();
-                    }
-                }
-            }
+            int item = blockIdx.x;
+            a_producer_role<C>(cx, &tm_mant, &tm_exp, raw_full, raw_empty, raw_base,
+                               [&](int, int& row0, int& k_begin, int& k_end) {
+                                   if (item >= total_items) return false;
+                                   const WorkItem w = work_item<SPLIT>(item, p);
+                                   row0 = w.mt * T_MC; k_begin = w.k_begin; k_end = w.k_end;
+                                   item += gridDim.x;
+                                   return true;
+                               });
         }
     } else if (warp == 1) {
         // ================================ UMMA issuer =================================
