@@ -137,6 +137,8 @@ def test_argument_errors():
     p = t.data_ptr()
     assert lib.atb_gemm_bfp16_out(256, 264, 256, 64, 128, 64, 128, p, p, p, 264, p, p, None) == 2      # N % 16
     assert lib.atb_gemm_bfp16_out(256, 256, 256, 32, 128, 64, 128, p, p, p, 256, p, p, None) == 3      # tiling
+    assert lib.atb_gemm_bfp16_out(256, 256, 256, 32, 128, 128, 256, p, p, p, 256, p, p, None) == 3     # 32-row slabs: none
+    assert lib.atb_gemm_bfp16_out(256, 256, 256, 128, 256, 128, 256, p, p, p, 256, p, p, None) == 3    # T_K = 128 elsewhere
     assert lib.atb_gemm_bfp16_out(256, 256, 256, 64, 128, 64, 128, p, p, p, 256, None, p, None) == 1   # NULL
     assert lib.atb_gemm_bfp16_out(256, 256, 256, 64, 128, 64, 128, p, p, p, 256, p + 8, p, None) == 4  # alignment
 
